@@ -1,0 +1,145 @@
+/*
+ * moe_vqlr — one routed Mixture-of-Experts decode layer (1..16 tokens) whose expert matrices
+ * are stored as a vector-quantised part plus a shared-basis low-rank part, for NVIDIA B200
+ * (sm_100a).  Plain C ABI: integers, sizes and raw pointers only.
+ *
+ * What one call computes (paper: Section 2.1 for the MoE block, Eq. 1 and Section 3.1 for the
+ * representation, Section 4 for the order of the work):
+ *
+ *   logit[t][e] = <router_w[e], x[t]> (+ router_bias[e])
+ *   the k experts with the largest logits per token (ties: lower expert id), affinities a =
+ *       softmax over the k selected logits (or over all E when renorm_topk == 0)
+ *   grouping of the (token, slot) pairs by expert, so each activated expert's payload is read
+ *       once per layer whatever the batch size (Section 5.5)
+ *   per projection P in {gate, up, down}, per activated expert e (Eq. 1, stored transposed):
+ *       W_P,e[o][b*d+j] = codebook_P[ idx_P[e][o][b] ][j] + sum_rho factor_P[e][o][rho]*basis_P[rho][b*d+j]
+ *     evaluated without ever forming W: the VQ part by code-word lookups, the low-rank part as
+ *     factor_P[e] * z with z = basis_P * input computed once per token and shared by all
+ *     experts (Section 3.2, "z = D^T h"); or W_P,e = dense_P[e] for a projection kept in bf16
+ *     (Section 3.1 keeps the down projection uncompressed)
+ *   p = silu(W_gate,e x) * (W_up,e x);   y = W_down,e p                      (SwiGLU expert)
+ *   out[t] = sum_s a[t][s] * y[t][s]  +  sum over the always-on shared experts of y (weight 1)
+ *
+ * Symbols: H hidden size, I expert intermediate size, E routed experts, k experts per token,
+ * S shared experts (ids E..E+S-1), d block length, K code-book size, r rank, T tokens.
+ * bf16 means the 16-bit brain-float format; all matrices are row-major, densely packed.
+ *
+ * Threading: a handle may be used by one host thread at a time.  All work of a call is
+ * enqueued on the given CUDA stream and is asynchronous unless stated otherwise.
+ */
+#ifndef MOE_VQLR_H_
+#define MOE_VQLR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moe_vqlr_handle moe_vqlr_handle; /* opaque, owned by the library */
+
+typedef enum {
+  MOE_VQLR_OK = 0,
+  MOE_VQLR_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, T out of range, ...       */
+  MOE_VQLR_ERR_UNSUPPORTED = 2, /* a shape or option this build has no kernel for            */
+  MOE_VQLR_ERR_CUDA = 3,        /* a CUDA runtime call or a launch failed                     */
+  MOE_VQLR_ERR_OOM = 4,         /* workspace allocation failed                                */
+  MOE_VQLR_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up                         */
+  MOE_VQLR_ERR_BAD_INDEX = 6    /* an index map holds a value >= K (found by validation)      */
+} moe_vqlr_status;
+
+typedef enum {
+  MOE_VQLR_PROJ_VQLR = 0,      /* code book + indices (+ low-rank term when rank > 0)  (Eq. 1)  */
+  MOE_VQLR_PROJ_DENSE_BF16 = 1 /* uncompressed bf16 matrix (Section 3.1, down projection)     */
+} moe_vqlr_proj_kind;
+
+/* One projection.  out x in is I x H for gate and up, H x I for down.  All pointers are DEVICE
+ * pointers borrowed for the lifetime of the handle; the caller keeps them alive and unchanged.
+ * Alignment: every pointer 16-byte aligned.  Pointers of different projections may alias (one
+ * code book or one basis shared by gate and up is detected and staged / projected once). */
+typedef struct {
+  int32_t kind;         /* moe_vqlr_proj_kind                                                  */
+  int32_t reserved;
+  const void* codebook; /* [K][d] bf16                                     (VQLR)             */
+  const void* idx;      /* [E+S][out][in/d], uint8 when K <= 256 else uint16 (VQLR); blocks run
+                           along the contraction dimension `in`                               */
+  const void* basis;    /* [rank][in] bf16 = D^T, shared by all experts   (VQLR, rank > 0)    */
+  const void* factor;   /* [E+S][out][rank] bf16 = C_e^T, expert-private  (VQLR, rank > 0)    */
+  const void* dense;    /* [E+S][out][in] bf16                            (DENSE_BF16)        */
+} moe_vqlr_proj;
+
+enum {
+  MOE_VQLR_FLAG_VALIDATE_INDICES = 1u /* create() scans every index map once and fails with
+                                         BAD_INDEX if a value >= K is found (costs one pass
+                                         over the index maps; never done on the decode path) */
+};
+
+typedef struct {
+  int32_t hidden;        /* H, multiple of vq_dim                                              */
+  int32_t inter;         /* I, multiple of vq_dim                                              */
+  int32_t n_experts;     /* E >= 1                                                             */
+  int32_t top_k;         /* 1 <= k <= E, k <= 32                                               */
+  int32_t n_shared;      /* S >= 0                                                             */
+  int32_t vq_dim;        /* d, must be 8                                                       */
+  int32_t codebook_size; /* K, 1..65536                                                        */
+  int32_t rank;          /* r >= 0                                                             */
+  int32_t max_tokens;    /* largest T a call may pass, 1..16                                   */
+  int32_t renorm_topk;   /* 1: affinities sum to 1 over the selected k;  0: softmax over all E */
+  uint32_t flags;        /* MOE_VQLR_FLAG_*                                                    */
+  int32_t reserved;
+  const void* router_w;     /* [E][H] bf16, device                                             */
+  const float* router_bias; /* [E] fp32, device, or NULL                                       */
+  moe_vqlr_proj gate, up, down;
+} moe_vqlr_config;
+
+/* Optional copies of the routing state, for checking.  Each member is a DEVICE pointer or
+ * NULL; non-null members are filled (on the call's stream) after the layer's kernels.
+ * Shared experts do not appear: these arrays cover the E routed experts only. */
+typedef struct {
+  float* logits;       /* [T][E]                                                              */
+  int32_t* topk_id;    /* [T][k]  slot s = s-th ranked expert (logit descending, id ascending) */
+  float* topk_w;       /* [T][k]  affinities                                                   */
+  int32_t* counts;     /* [E]     pairs per expert                                             */
+  int32_t* offsets;    /* [E+1]   exclusive prefix sum of counts                               */
+  int32_t* pair_token; /* [T*k]   pairs sorted by expert, ascending token within an expert     */
+  int32_t* pair_slot;  /* [T*k]                                                                */
+} moe_vqlr_debug;
+
+/* Validates the configuration, allocates the handle and its device workspace on the CURRENT
+ * CUDA device and returns the handle in *out (NULL on failure).  Synchronous.
+ * Errors: INVALID_ARG, UNSUPPORTED (vq_dim != 8, H or I not a multiple of 8, K > 65536, k > 32,
+ * max_tokens > 16), OOM, CUDA, BAD_INDEX (only with MOE_VQLR_FLAG_VALIDATE_INDICES). */
+int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out);
+
+/* Runs the layer for T tokens.  x: [T][H] bf16, device.  out: [T][H] bf16, device, written with
+ * round-to-nearest-even; must not overlap x.  dbg may be NULL.  cuda_stream is a cudaStream_t
+ * (NULL = the legacy default stream).  Returns after enqueueing; a launch failure gives
+ * ERR_CUDA.  Calls on one handle must not overlap on the device (they share the workspace). */
+int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* out,
+                          const moe_vqlr_debug* dbg, void* cuda_stream);
+
+/* Same layer with HOST buffers: copies x (T*H bf16, host) to the device, runs the layer, copies
+ * out (T*H bf16) back and waits for the stream.  Pinned host memory makes the copies
+ * asynchronous up to the final wait; pageable memory works but is slower.  Weights stay on
+ * the device.  Synchronous on return. */
+int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T, void* out_host,
+                               void* cuda_stream);
+
+/* Frees the workspace and the handle.  The caller must first make sure no call on this handle
+ * is still running on the device.  NULL is accepted. */
+int moe_vqlr_destroy(moe_vqlr_handle* h);
+
+/* Text of the last error on this handle ("" if none); with NULL, of the last failed create()
+ * on this thread.  The string is owned by the library. */
+const char* moe_vqlr_last_error(const moe_vqlr_handle* h);
+
+/* Number of kernel launches this handle has enqueued since create(). */
+int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h);
+
+/* Device workspace the handle owns, in bytes. */
+int64_t moe_vqlr_workspace_bytes(const moe_vqlr_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_VQLR_H_ */

@@ -1,0 +1,213 @@
+"""Thin ctypes binding of the C ABI in ``include/moe_vqlr.h``: argument marshalling only.
+
+Every step of the layer runs in the CUDA library; there is no Python or CPU fallback.  Importing
+this module loads ``csrc/libmoe_vqlr.so`` and raises if it is missing (build it with
+``python -m paper_2609_21137_b200.build``).  PyTorch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_OOM, ERR_TIMEOUT, ERR_BAD_INDEX = range(7)
+PROJ_VQLR, PROJ_DENSE_BF16 = 0, 1
+FLAG_VALIDATE_INDICES = 1
+
+EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
+           "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",
+           "moe_vqlr_workspace_bytes"]
+
+
+class MoeVqlrError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"moe_vqlr status {status}: {message}")
+        self.status = status
+
+
+class _Proj(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("reserved", C.c_int32), ("codebook", C.c_void_p),
+                ("idx", C.c_void_p), ("basis", C.c_void_p), ("factor", C.c_void_p),
+                ("dense", C.c_void_p)]
+
+
+class _Config(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("inter", C.c_int32), ("n_experts", C.c_int32),
+                ("top_k", C.c_int32), ("n_shared", C.c_int32), ("vq_dim", C.c_int32),
+                ("codebook_size", C.c_int32), ("rank", C.c_int32), ("max_tokens", C.c_int32),
+                ("renorm_topk", C.c_int32), ("flags", C.c_uint32), ("reserved", C.c_int32),
+                ("router_w", C.c_void_p), ("router_bias", C.c_void_p),
+                ("gate", _Proj), ("up", _Proj), ("down", _Proj)]
+
+
+class _Debug(C.Structure):
+    _fields_ = [("logits", C.c_void_p), ("topk_id", C.c_void_p), ("topk_w", C.c_void_p),
+                ("counts", C.c_void_p), ("offsets", C.c_void_p), ("pair_token", C.c_void_p),
+                ("pair_slot", C.c_void_p)]
+
+
+def _load():
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: the CUDA library is not built "
+                          "(run `python -m paper_2609_21137_b200.build`); there is no fallback")
+    lib = C.CDLL(path)
+    lib.moe_vqlr_create.restype = C.c_int
+    lib.moe_vqlr_create.argtypes = [C.POINTER(_Config), C.POINTER(C.c_void_p)]
+    lib.moe_vqlr_decode_layer.restype = C.c_int
+    lib.moe_vqlr_decode_layer.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                          C.POINTER(_Debug), C.c_void_p]
+    lib.moe_vqlr_decode_layer_host.restype = C.c_int
+    lib.moe_vqlr_decode_layer_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                               C.c_void_p]
+    lib.moe_vqlr_destroy.restype = C.c_int
+    lib.moe_vqlr_destroy.argtypes = [C.c_void_p]
+    lib.moe_vqlr_last_error.restype = C.c_char_p
+    lib.moe_vqlr_last_error.argtypes = [C.c_void_p]
+    lib.moe_vqlr_launch_count.restype = C.c_int64
+    lib.moe_vqlr_launch_count.argtypes = [C.c_void_p]
+    lib.moe_vqlr_workspace_bytes.restype = C.c_int64
+    lib.moe_vqlr_workspace_bytes.argtypes = [C.c_void_p]
+    return lib
+
+
+_lib = _load()
+
+
+def library():
+    return _lib
+
+
+def bits_to_device(a: Optional[np.ndarray], device) -> Optional[torch.Tensor]:
+    """numpy array (bf16 bit patterns as uint16, uint8/uint16 indices, float32) -> device tensor
+    holding the same bytes."""
+    if a is None:
+        return None
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).to(device)
+    return torch.from_numpy(a).to(device)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+class MoeVqlrLayer:
+    """One layer handle.  Weights are torch tensors on the GPU (any 2-byte dtype for bf16 data,
+    uint8 / 2-byte for indices); the handle borrows their storage, this object keeps them alive.
+
+    ``gate``/``up``/``down`` are dicts with keys among codebook, idx, basis, factor, dense.
+    """
+
+    def __init__(self, *, H, I, E, k, S=0, d=8, K=0, r=0, max_tokens=16, router_w, router_bias=None,
+                 gate, up, down, renorm_topk=True, flags=0):
+        self.H, self.I, self.E, self.k, self.S, self.K, self.r = H, I, E, k, S, K, r
+        self.max_tokens = max_tokens
+        self._keep = [router_w, router_bias, gate, up, down]
+        self.device = router_w.device
+        cfg = _Config()
+        cfg.hidden, cfg.inter, cfg.n_experts, cfg.top_k, cfg.n_shared = H, I, E, k, S
+        cfg.vq_dim, cfg.codebook_size, cfg.rank, cfg.max_tokens = d, K, r, max_tokens
+        cfg.renorm_topk = 1 if renorm_topk else 0
+        cfg.flags = flags
+        cfg.router_w = router_w.data_ptr()
+        cfg.router_bias = None if router_bias is None else router_bias.data_ptr()
+        for name, p in (("gate", gate), ("up", up), ("down", down)):
+            P = getattr(cfg, name)
+            dense = p.get("dense")
+            P.kind = PROJ_DENSE_BF16 if dense is not None else PROJ_VQLR
+            for key in ("codebook", "idx", "basis", "factor", "dense"):
+                t = p.get(key)
+                setattr(P, key, None if t is None else t.data_ptr())
+        self._cfg = cfg
+        handle = C.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = _lib.moe_vqlr_create(C.byref(cfg), C.byref(handle))
+        if rc != OK:
+            raise MoeVqlrError(rc, _lib.moe_vqlr_last_error(None).decode())
+        self._h = handle
+
+    @classmethod
+    def from_synth(cls, layer, device="cuda", max_tokens=None, flags=0, renorm_topk=True):
+        """Upload a ``synth.Layer`` (numpy bit patterns) and create a handle on it."""
+        s = layer.shape
+        cache = {}
+
+        def up(a):
+            if a is None:
+                return None
+            if id(a) not in cache:          # aliased arrays stay aliased on the device
+                cache[id(a)] = bits_to_device(a, device)
+            return cache[id(a)]
+
+        def proj(p):
+            return dict(codebook=up(p.codebook), idx=up(p.idx), basis=up(p.basis),
+                        factor=up(p.factor), dense=up(p.dense))
+
+        return cls(H=s.H, I=s.I, E=s.E, k=s.k, S=s.S, d=s.d, K=s.K, r=s.r,
+                   max_tokens=max_tokens or max(s.T, 1), router_w=up(layer.router_w),
+                   router_bias=up(layer.router_bias), gate=proj(layer.gate), up=proj(layer.up),
+                   down=proj(layer.down), renorm_topk=renorm_topk, flags=flags)
+
+    # -----------------------------------------------------------------------------------
+    def _check(self, rc):
+        if rc != OK:
+            raise MoeVqlrError(rc, _lib.moe_vqlr_last_error(self._h).decode())
+
+    def decode(self, x: torch.Tensor, out: Optional[torch.Tensor] = None, debug: bool = False,
+               stream: Optional[torch.cuda.Stream] = None):
+        """x: [T][H] 2-byte tensor holding bf16 on the GPU.  Returns out ([T][H] bf16), or
+        (out, dict of routing tensors) with ``debug=True``."""
+        T = x.shape[0]
+        if out is None:
+            out = torch.empty((T, self.H), dtype=torch.bfloat16, device=x.device)
+        st = stream or torch.cuda.current_stream(x.device)
+        dbg = None
+        tensors = None
+        if debug:
+            i32 = dict(dtype=torch.int32, device=x.device)
+            tensors = dict(logits=torch.empty((T, self.E), dtype=torch.float32, device=x.device),
+                           topk_id=torch.empty((T, self.k), **i32),
+                           topk_w=torch.empty((T, self.k), dtype=torch.float32, device=x.device),
+                           counts=torch.empty(self.E, **i32), offsets=torch.empty(self.E + 1, **i32),
+                           pair_token=torch.empty(T * self.k, **i32),
+                           pair_slot=torch.empty(T * self.k, **i32))
+            dbg = _Debug(**{k: v.data_ptr() for k, v in tensors.items()})
+        self._check(_lib.moe_vqlr_decode_layer(self._h, _ptr(x), T, _ptr(out),
+                                               None if dbg is None else C.byref(dbg),
+                                               C.c_void_p(st.cuda_stream)))
+        return (out, tensors) if debug else out
+
+    def decode_host(self, x_host: torch.Tensor, out_host: torch.Tensor,
+                    stream: Optional[torch.cuda.Stream] = None):
+        """Host buffers in and out (pinned recommended); returns when the result is in out_host."""
+        T = x_host.shape[0]
+        st = stream or torch.cuda.current_stream(self.device)
+        self._check(_lib.moe_vqlr_decode_layer_host(self._h, _ptr(x_host), T, _ptr(out_host),
+                                                    C.c_void_p(st.cuda_stream)))
+        return out_host
+
+    @property
+    def launch_count(self) -> int:
+        return int(_lib.moe_vqlr_launch_count(self._h))
+
+    @property
+    def workspace_bytes(self) -> int:
+        return int(_lib.moe_vqlr_workspace_bytes(self._h))
+
+    def close(self):
+        if getattr(self, "_h", None):
+            _lib.moe_vqlr_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

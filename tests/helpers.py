@@ -1,0 +1,82 @@
+"""Shared comparison code of the GPU parity tests: runs the oracle and the CUDA library on the
+same seeded layer and checks the acceptance bars.
+
+Bars: routing ids and grouping bit-exact; affinities to 2e-6; bf16 outputs against the fp64
+oracle with (i) elementwise |err| / max(|y|, 1e-3 * max|y|) <= 2e-2, (ii) max|err| / max|y| <=
+2e-2, (iii) mean |err| <= 1e-3 + mean|bf16(y) - y| (the second term is the rounding error any
+bf16 output carries).
+"""
+import numpy as np
+import torch
+
+import oracle
+from paper_2609_21137_b200 import synth
+
+MIN_LOGIT_GAP = 1e-5      # fp32 logits must order like the fp64 oracle's: reject closer seeds
+REL_TOL = 2e-2
+MAE_TOL = 1e-3
+
+
+def logit_gaps(res, k):
+    srt = -np.sort(-res.logits, axis=1)
+    kk = min(k + 1, srt.shape[1])
+    return float(np.min(srt[:, :kk - 1] - srt[:, 1:kk])) if kk > 1 else np.inf
+
+
+def make_checked_layer(shp, seed=0, max_tries=20, tie=None, **oracle_kw):
+    """Returns (layer, oracle result, seed used): the first seed >= `seed` whose logits are
+    separated by more than MIN_LOGIT_GAP around and inside the top-k."""
+    for s in range(seed, seed + max_tries):
+        layer = synth.make_layer(shp, seed=s)
+        if tie is not None:
+            synth.duplicate_router_rows(layer, *tie)
+        res = oracle.OracleLayer.from_synth(layer, **oracle_kw).decode_layer(layer.x)
+        if tie is not None:
+            return layer, res, s
+        if shp.k == shp.E or logit_gaps(res, shp.k) > MIN_LOGIT_GAP:
+            return layer, res, s
+    raise RuntimeError("no seed with separated logits")
+
+
+def bf16_tensor_to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def output_metrics(out_gpu: np.ndarray, ref: np.ndarray) -> dict:
+    err = np.abs(out_gpu - ref)
+    ymax = float(np.max(np.abs(ref)))
+    floor = 1e-3 * ymax
+    ref_bf16 = synth.bf16_bits_to_f64(synth.f32_to_bf16_bits(ref.astype(np.float32)))
+    return dict(max_rel=float(np.max(err / np.maximum(np.abs(ref), floor))),
+                norm_max=float(np.max(err) / ymax), mae=float(np.mean(err)),
+                mae_format=float(np.mean(np.abs(ref_bf16 - ref))),
+                mae_vs_bf16_oracle=float(np.mean(np.abs(out_gpu - ref_bf16))), ymax=ymax)
+
+
+def assert_output(out_gpu: np.ndarray, ref: np.ndarray, what=""):
+    m = output_metrics(out_gpu, ref)
+    assert m["max_rel"] <= REL_TOL, (what, m)
+    assert m["norm_max"] <= REL_TOL, (what, m)
+    assert m["mae"] <= MAE_TOL + m["mae_format"], (what, m)
+    return m
+
+
+def assert_routing(dbg: dict, res, check_ids=True):
+    ids = dbg["topk_id"].cpu().numpy()
+    if check_ids:
+        np.testing.assert_array_equal(ids, res.topk_id)
+        np.testing.assert_array_equal(dbg["counts"].cpu().numpy(), res.counts)
+        np.testing.assert_array_equal(dbg["offsets"].cpu().numpy(), res.offsets)
+        np.testing.assert_array_equal(dbg["pair_token"].cpu().numpy(), res.pair_token)
+        np.testing.assert_array_equal(dbg["pair_slot"].cpu().numpy(), res.pair_slot)
+        np.testing.assert_allclose(dbg["topk_w"].cpu().numpy(), res.topk_w, rtol=0, atol=2e-6)
+    np.testing.assert_allclose(dbg["logits"].cpu().numpy(), res.logits, rtol=0, atol=2e-5)
+
+
+def run_gpu(layer, T=None, debug=True, **kw):
+    from paper_2609_21137_b200 import binding
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", **kw)
+    x = binding.bits_to_device(layer.x if T is None else layer.x[:T], "cuda")
+    result = mod.decode(x, debug=debug)
+    torch.cuda.synchronize()
+    return mod, result
