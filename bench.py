@@ -1,0 +1,396 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE decode layer on VQ + shared-basis low-rank expert weights.
+
+A step is ONE call of the whole layer (router, top-k, grouping, gate/up, SwiGLU, down, weighted
+sum) on one batch of tokens.  Steps rotate over L distinct synthetic layers so that every call
+reads its weights from HBM, not from L2.  Metric: microseconds per MoE layer per token.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload qwen3|qwen3_b16|dsv2lite|dsv2lite_b8|mixtral|...] [--mode full|paper|dense]
+
+N > 1 (launched with torch.distributed.run) runs independent replicas, one per GPU: the path
+has no exchange step, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=960)
+    ap.add_argument("--warmup", type=int, default=96)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3")
+    ap.add_argument("--mode", default="full", choices=["full", "paper", "dense"])
+    ap.add_argument("--layers", type=int, default=0, help="distinct layers to rotate over (0 = auto)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the secondary measurements")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self._stop = threading.Event()
+        self._thr = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}",
+                                      "--format=csv,noheader,nounits"], capture_output=True,
+                                     text=True, timeout=5).stdout.strip()
+                if out:
+                    self.rows.append([c.strip() for c in out.splitlines()[0].split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thr.join(timeout=6)
+
+    def summary(self) -> dict:
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+# ------------------------------------------------------------------------------------------
+def oracle_timing(workload: str, mode: str, budget_s: float, max_steps: int, warmup: int = 1):
+    """Times full oracle layer calls (fp64, dense reconstruction) on a numpy-generated layer of
+    the same shape; stops after `max_steps` calls or when `budget_s` of CPU time is used."""
+    import oracle
+    from paper_2609_21137_b200 import synth
+    shp = synth.shape(workload, mode=mode)
+    layer = synth.make_layer(shp, seed=0)
+    orc = oracle.OracleLayer.from_synth(layer)
+    for _ in range(warmup):
+        orc.decode_layer(layer.x)
+    times = []
+    t_start = time.perf_counter()
+    while len(times) < max_steps and (time.perf_counter() - t_start) < budget_s:
+        t0 = time.perf_counter()
+        orc.decode_layer(layer.x)
+        times.append(time.perf_counter() - t0)
+    mean_s = sum(times) / len(times)
+    return dict(us_per_layer_per_token=mean_s * 1e6 / shp.T, calls=len(times), cores=oracle.threads(),
+                T=shp.T, mean_s=mean_s)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    r = oracle_timing(args.workload, args.mode, budget_s=150.0, max_steps=max(1, args.steps),
+                      warmup=min(max(args.warmup, 1), 2))
+    sample = (f"{r['calls']} full fp64 oracle layer calls of the {args.workload} shape (mode {args.mode}, "
+              f"T={r['T']}, seed 0) on the host cores; {args.steps} steps requested, capped at 150 s")
+    line = {"impl": "reference", "metric": "us_per_moe_layer_per_token", "value": r["us_per_layer_per_token"],
+            "unit": "us", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": r["mean_s"] * 1e3, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{args.workload} T={r['T']} mode={args.mode}"},
+            "cpu_baseline": {"value": r["us_per_layer_per_token"], "unit": "us", "cores": r["cores"],
+                             "kind": "oracle", "sample": sample},
+            "e2e": {"value": r["us_per_layer_per_token"], "unit": "us", "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------
+class Workload:
+    """L distinct layers of one shape on the GPU, with per-layer token batches."""
+
+    def __init__(self, name: str, mode: str, n_layers: int, device):
+        import torch
+        from paper_2609_21137_b200 import accounting, binding, devsynth, synth
+        self.torch = torch
+        self.shp = synth.shape(name, mode=mode)
+        self.name, self.mode, self.device = name, mode, device
+        shp = self.shp
+        probe = accounting.layer_bytes(H=shp.H, I=shp.I, E=shp.E, d=shp.d, K=shp.K, r=shp.r, T=shp.T,
+                                       mode=mode, n_active=shp.k + shp.S)
+        if n_layers <= 0:       # enough distinct layers that one rotation touches > 2.5x L2
+            n_layers = max(4, min(64, -(-int(2.5 * L2_BYTES) // max(probe.total, 1))))
+        self.layers, self.xs, self.outs = [], [], []
+        for i in range(n_layers):
+            kw = devsynth.make_device_layer(shp, seed=1000 + i, device=device)
+            x = kw.pop("x")
+            self.layers.append(binding.MoeVqlrLayer(**kw))
+            self.xs.append(x)
+            self.outs.append(torch.empty_like(x))
+        torch.cuda.synchronize(device)
+        # routing of every layer (distinct activated experts) for the byte accounting
+        self.bytes = []
+        for lay, x in zip(self.layers, self.xs):
+            _, dbg = lay.decode(x, debug=True)
+            n_act = int((dbg["counts"] > 0).sum().item()) + shp.S
+            self.bytes.append(accounting.layer_bytes(H=shp.H, I=shp.I, E=shp.E, d=shp.d, K=shp.K, r=shp.r,
+                                                     T=shp.T, mode=mode, n_active=n_act))
+        torch.cuda.synchronize(device)
+        self.mean_bytes = sum(b.total for b in self.bytes) / len(self.bytes)
+        self.mean_active = sum(b.n_active for b in self.bytes) / len(self.bytes)
+
+    def step(self, i: int):
+        j = i % len(self.layers)
+        self.layers[j].decode(self.xs[j], out=self.outs[j])
+
+    def launches(self) -> int:
+        return sum(l.launch_count for l in self.layers)
+
+    def run_timed(self, steps: int, warmup: int):
+        """Device time of `steps` back-to-back calls in milliseconds (CUDA events on the stream)."""
+        torch = self.torch
+        for i in range(warmup):
+            self.step(i)
+        torch.cuda.synchronize(self.device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = self.launches()
+        e0.record()
+        for i in range(steps):
+            self.step(warmup + i)
+        e1.record()
+        torch.cuda.synchronize(self.device)
+        return e0.elapsed_time(e1), self.launches() - n0
+
+    def run_stage_profile(self, steps: int, warmup: int) -> dict:
+        """Average device time per stage (ms) over `steps` profiled calls."""
+        torch = self.torch
+        for lay in self.layers:
+            lay.set_profiling(True)
+        sums, n = {}, 0
+        for i in range(warmup + steps):
+            j = i % len(self.layers)
+            self.step(i)
+            if i >= warmup:
+                for k_, v in self.layers[j].last_stage_times_ms().items():
+                    sums[k_] = sums.get(k_, 0.0) + v
+                n += 1
+        for lay in self.layers:
+            lay.set_profiling(False)
+        torch.cuda.synchronize(self.device)
+        return {k_: v / n for k_, v in sums.items()}
+
+    def run_e2e(self, steps: int, warmup: int):
+        """Host buffers in and out through moe_vqlr_decode_layer_host; ms for `steps` calls."""
+        torch = self.torch
+        shp = self.shp
+        xh = [x.cpu().pin_memory() for x in self.xs]
+        oh = [torch.empty((shp.T, shp.H), dtype=torch.bfloat16).pin_memory() for _ in self.xs]
+        for i in range(warmup):
+            j = i % len(self.layers)
+            self.layers[j].decode_host(xh[j], oh[j])
+        torch.cuda.synchronize(self.device)
+        t0 = time.perf_counter()
+        for i in range(steps):
+            j = (warmup + i) % len(self.layers)
+            self.layers[j].decode_host(xh[j], oh[j])
+        torch.cuda.synchronize(self.device)
+        ms = (time.perf_counter() - t0) * 1e3
+        nbytes = shp.T * shp.H * 2
+        return ms, nbytes, nbytes
+
+    def close(self):
+        for lay in self.layers:
+            lay.close()
+        self.layers, self.xs, self.outs = [], [], []
+        self.torch.cuda.empty_cache()
+
+
+def measure(name, mode, steps, warmup, device, n_layers=0):
+    wl = Workload(name, mode, n_layers, device)
+    ms, launches = wl.run_timed(steps, warmup)
+    us_layer = ms * 1e3 / steps
+    res = dict(workload=name, mode=mode, T=wl.shp.T, layers=len(wl.layers), us_per_layer=us_layer,
+               us_per_layer_per_token=us_layer / wl.shp.T, algorithmic_bytes=wl.mean_bytes,
+               distinct_experts=wl.mean_active, gbs=wl.mean_bytes / (us_layer * 1e-6) / 1e9,
+               launches=launches)
+    return wl, res, ms
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_21137_b200 import accounting  # noqa: F401
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    peak, peak_kind = measured_peak()
+    wl = Workload(args.workload, args.mode, args.layers, device)
+
+    # ---- the timed region: W warm-up steps, then exactly K steps ---------------------------
+    for i in range(args.warmup):
+        wl.step(i)
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = wl.launches()
+        e0.record()
+        for i in range(args.steps):
+            wl.step(args.warmup + i)
+        e1.record()
+        torch.cuda.synchronize(device)
+        ms = e0.elapsed_time(e1)
+        launches = wl.launches() - n0
+        barrier()
+        if ms < 400:      # keep the sampler alive long enough to see the clocks
+            t_end = time.time() + 0.6
+            i = 0
+            while time.time() < t_end:
+                wl.step(i)
+                i += 1
+            torch.cuda.synchronize(device)
+    if world > 1:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    shp = wl.shp
+    ms_per_step = ms / args.steps
+    us_per_layer_token = ms_per_step * 1e3 / (shp.T * world)
+    layer_gbs = wl.mean_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- per-stage profile for the roofline of the dominant kernel -------------------------
+    stage_ms = wl.run_stage_profile(min(args.steps, 4 * len(wl.layers)), 8)
+    gu_bytes = sum(b.gateup_kernel for b in wl.bytes) / len(wl.bytes)
+    dn_bytes = sum(b.down_kernel for b in wl.bytes) / len(wl.bytes)
+    stage_bytes = {"gateup": gu_bytes, "down": dn_bytes}
+    dominant = max(stage_bytes, key=lambda s: stage_ms.get(s, 0.0))
+    dom_ms = stage_ms[dominant]
+    achieved = stage_bytes[dominant] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": f"k_{dominant}", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": None, "algorithmic_bytes_per_launch": stage_bytes[dominant],
+                "us_per_launch": dom_ms * 1e3,
+                "stage_us": {k_: v * 1e3 for k_, v in stage_ms.items()},
+                "layer": {"algorithmic_bytes": wl.mean_bytes, "gbs": layer_gbs, "frac_of_measured": layer_gbs / peak,
+                          "frac_of_nominal_8TBs": layer_gbs / NOMINAL_HBM_GBS}}
+
+    # ---- end to end through host buffers --------------------------------------------------
+    e2e_steps = min(args.steps, 400)
+    e2e_ms, h2d, d2h = wl.run_e2e(e2e_steps, max(3, min(args.warmup, 20)))
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = {"value": e2e_ms * 1e3 / e2e_steps / (shp.T * world), "unit": "us", "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+    n_layers = len(wl.layers)
+    wl.close()
+
+    extras = []
+    if rank == 0 and world == 1 and not args.no_extras:
+        todo = [("qwen3", "paper"), ("qwen3", "dense"), ("qwen3_b16", "full"), ("qwen3_b16", "paper"),
+                ("qwen3_b16", "dense")]
+        todo = [t_ for t_ in todo if t_ != (args.workload, args.mode)]
+        for name, mode in todo:
+            try:
+                w2, r2, _ = measure(name, mode, 240, 24, device)
+                r2["frac_of_measured"] = r2["gbs"] / peak
+                r2["frac_of_nominal_8TBs"] = r2["gbs"] / NOMINAL_HBM_GBS
+                w2.close()
+                extras.append(r2)
+            except Exception as exc:   # an extra must never take the headline down
+                extras.append({"workload": name, "mode": mode, "error": str(exc)[:200]})
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        r = oracle_timing(args.workload, args.mode, budget_s=20.0, max_steps=64)
+        cpu = {"value": r["us_per_layer_per_token"], "unit": "us", "cores": r["cores"], "kind": "oracle",
+               "sample": f"{r['calls']} full fp64 oracle layer calls of the same shape (numpy-seeded layer, T={r['T']})"}
+
+    if rank == 0:
+        line = {"metric": "us_per_moe_layer_per_token", "value": us_per_layer_token, "unit": "us",
+                "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+                "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic",
+                "config": {"workload": f"{args.workload} (H={shp.H} I={shp.I} E={shp.E} k={shp.k} S={shp.S} "
+                                       f"K={shp.K} r={shp.r}) T={shp.T} mode={args.mode}",
+                           "distinct_layers": n_layers,
+                           "l2": f"rotation over {n_layers} distinct layers touches "
+                                 f"{n_layers * wl.mean_bytes / 1e6:.0f} MB per pass, larger than the 126 MB L2",
+                           "parallelism": "replicas only" if world > 1 else "single GPU"},
+                "tokens_per_s_per_layer": shp.T * world / (ms_per_step * 1e-3),
+                "hbm_gbs": layer_gbs, "hbm_frac_of_measured": layer_gbs / peak,
+                "hbm_frac_of_nominal_8TBs": layer_gbs / NOMINAL_HBM_GBS,
+                "algorithmic_bytes_per_layer": wl.mean_bytes, "distinct_experts_per_layer": wl.mean_active,
+                "gpu_launches": launches, "clocks": clocks.summary(), "roofline": roofline, "e2e": e2e,
+                "cpu_baseline": cpu, "extras": extras}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -133,6 +133,22 @@ int moe_vqlr_destroy(moe_vqlr_handle* h);
  * on this thread.  The string is owned by the library. */
 const char* moe_vqlr_last_error(const moe_vqlr_handle* h);
 
+/* Measurement aid (no counterpart in the paper; its profiles come from the Neuron tools,
+ * Section 5.1).  With profiling on, every decode call records a CUDA event on the call's
+ * stream before and after each stage.  Stages, in order: router_z, route, gateup, zdown, down
+ * (moe_vqlr_stage_count() of them, named by moe_vqlr_stage_name()).  The events sit between
+ * the kernels, so a profiled call can run slightly slower than an unprofiled one. */
+int moe_vqlr_set_profiling(moe_vqlr_handle* h, int32_t on);
+
+/* Waits for the last profiled call on this handle and writes the device time of each stage in
+ * milliseconds to ms_out[0..stage_count) (0 for a stage the configuration does not run).
+ * cap = capacity of ms_out, at least moe_vqlr_stage_count().  INVALID_ARG when the last call
+ * was not profiled. */
+int moe_vqlr_last_stage_times(moe_vqlr_handle* h, float* ms_out, int32_t cap);
+
+int moe_vqlr_stage_count(void);
+const char* moe_vqlr_stage_name(int32_t i);
+
 /* Number of kernel launches this handle has enqueued since create(). */
 int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h);
 

@@ -21,7 +21,8 @@ FLAG_VALIDATE_INDICES = 1
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",
-           "moe_vqlr_workspace_bytes"]
+           "moe_vqlr_workspace_bytes", "moe_vqlr_set_profiling", "moe_vqlr_last_stage_times",
+           "moe_vqlr_stage_count", "moe_vqlr_stage_name"]
 
 
 class MoeVqlrError(RuntimeError):
@@ -73,6 +74,14 @@ def _load():
     lib.moe_vqlr_launch_count.argtypes = [C.c_void_p]
     lib.moe_vqlr_workspace_bytes.restype = C.c_int64
     lib.moe_vqlr_workspace_bytes.argtypes = [C.c_void_p]
+    lib.moe_vqlr_set_profiling.restype = C.c_int
+    lib.moe_vqlr_set_profiling.argtypes = [C.c_void_p, C.c_int32]
+    lib.moe_vqlr_last_stage_times.restype = C.c_int
+    lib.moe_vqlr_last_stage_times.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int32]
+    lib.moe_vqlr_stage_count.restype = C.c_int
+    lib.moe_vqlr_stage_count.argtypes = []
+    lib.moe_vqlr_stage_name.restype = C.c_char_p
+    lib.moe_vqlr_stage_name.argtypes = [C.c_int32]
     return lib
 
 
@@ -192,6 +201,15 @@ class MoeVqlrLayer:
         self._check(_lib.moe_vqlr_decode_layer_host(self._h, _ptr(x_host), T, _ptr(out_host),
                                                     C.c_void_p(st.cuda_stream)))
         return out_host
+
+    def set_profiling(self, on: bool) -> None:
+        self._check(_lib.moe_vqlr_set_profiling(self._h, 1 if on else 0))
+
+    def last_stage_times_ms(self) -> dict:
+        n = _lib.moe_vqlr_stage_count()
+        buf = (C.c_float * n)()
+        self._check(_lib.moe_vqlr_last_stage_times(self._h, buf, n))
+        return {_lib.moe_vqlr_stage_name(i).decode(): float(buf[i]) for i in range(n)}
 
     @property
     def launch_count(self) -> int:

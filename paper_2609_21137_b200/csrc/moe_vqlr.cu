@@ -26,6 +26,8 @@ constexpr int kMaxT = 16;      // tokens per call
 constexpr int kMaxK = 32;      // experts per token
 constexpr int kD = 8;          // VQ block length (one code word = 16 bytes of bf16)
 constexpr int kTokGroup = 4;   // tokens of one expert handled per pass over its row
+constexpr int kStages = 5;     // router_z, route, gateup, zdown, down
+const char* const kStageNames[kStages] = {"router_z", "route", "gateup", "zdown", "down"};
 
 typedef __nv_bfloat16 bf16;
 
@@ -557,6 +559,10 @@ struct moe_vqlr_handle {
   bf16* x_stage;     // [maxT][H] device staging for the host-buffer entry point
   bf16* out_stage;   // [maxT][H]
   int64_t launches;
+  int profiling;             // record an event after every stage of a call
+  cudaEvent_t ev[kStages + 1];
+  bool ev_valid;
+  bool stage_ran[kStages];
   std::string error;
 };
 
@@ -642,6 +648,9 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   h->cfg = *cfg;
   h->launches = 0;
   h->workspace = nullptr;
+  h->profiling = 0;
+  h->ev_valid = false;
+  for (auto& e : h->ev) e = nullptr;
   h->idx_bytes = K <= 256 ? 1 : 2;
   cudaError_t ce = cudaGetDevice(&h->device);
   cudaDeviceProp prop;
@@ -773,32 +782,47 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
   const bf16* xb = static_cast<const bf16*>(x);
   bf16* ob = static_cast<bf16*>(out);
 
+  const bool prof = h->profiling != 0;
+  auto mark = [&](int i) { if (prof) cudaEventRecord(h->ev[i], st); };
+  for (int i = 0; i < kStages; ++i) h->stage_ran[i] = false;
+  mark(0);
   {
     const int rows = P.E + P.n_zrows;
     k_router_z<<<(rows + 7) / 8, 256, 0, st>>>(P, xb, T);
+    h->stage_ran[0] = true;
   }
+  mark(1);
   {
     const size_t smem = (size_t)T * P.E * 4 + (2 * (size_t)P.E + 1) * 4;
     k_route<<<1, 32 * T, smem, st>>>(P, T);
+    h->stage_ran[1] = true;
   }
+  mark(2);
   {
     const size_t smem = h->smem_gateup_fixed + h->smem_gateup_per_token * T;
     const int grid = h->sm_count;
     if (h->idx_bytes == 1) k_gateup<uint8_t><<<grid, 512, smem, st>>>(P, xb, T, h->two_books);
     else k_gateup<uint16_t><<<grid, 512, smem, st>>>(P, xb, T, h->two_books);
+    h->stage_ran[2] = true;
   }
+  mark(3);
   h->launches += 3;
   if (P.down.kind == MOE_VQLR_PROJ_VQLR && P.r > 0) {
     const int n_pos = T * (P.k + P.S);
     k_zdown<<<(n_pos * P.r + 7) / 8, 256, 0, st>>>(P, n_pos);
     h->launches += 1;
+    h->stage_ran[3] = true;
   }
+  mark(4);
   {
     const int grid = min(h->sm_count, (P.H + 15) / 16);
     if (h->idx_bytes == 1) k_down<uint8_t><<<grid, 512, h->smem_down, st>>>(P, ob, T);
     else k_down<uint16_t><<<grid, 512, h->smem_down, st>>>(P, ob, T);
     h->launches += 1;
+    h->stage_ran[4] = true;
   }
+  mark(5);
+  h->ev_valid = prof;
   cudaError_t ce = cudaGetLastError();
   if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "launch: %s", cudaGetErrorString(ce));
 
@@ -837,6 +861,8 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
 
 int moe_vqlr_destroy(moe_vqlr_handle* h) {
   if (!h) return MOE_VQLR_OK;
+  for (auto& e : h->ev)
+    if (e) cudaEventDestroy(e);
   cudaError_t ce = cudaFree(h->workspace);
   delete h;
   return ce == cudaSuccess ? MOE_VQLR_OK : MOE_VQLR_ERR_CUDA;
@@ -844,6 +870,38 @@ int moe_vqlr_destroy(moe_vqlr_handle* h) {
 
 const char* moe_vqlr_last_error(const moe_vqlr_handle* h) {
   return h ? h->error.c_str() : g_create_error.c_str();
+}
+
+int moe_vqlr_set_profiling(moe_vqlr_handle* h, int32_t on) {
+  if (!h) return MOE_VQLR_ERR_INVALID_ARG;
+  if (on && !h->ev[0]) {
+    for (auto& e : h->ev) {
+      cudaError_t ce = cudaEventCreate(&e);
+      if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "cudaEventCreate: %s", cudaGetErrorString(ce));
+    }
+  }
+  h->profiling = on ? 1 : 0;
+  h->ev_valid = false;
+  return MOE_VQLR_OK;
+}
+
+int moe_vqlr_stage_count(void) { return kStages; }
+
+const char* moe_vqlr_stage_name(int32_t i) { return (i >= 0 && i < kStages) ? kStageNames[i] : ""; }
+
+int moe_vqlr_last_stage_times(moe_vqlr_handle* h, float* ms_out, int32_t cap) {
+  if (!h || !ms_out || cap < kStages) return h ? fail(h, MOE_VQLR_ERR_INVALID_ARG, "ms_out null or cap < %d", kStages) : MOE_VQLR_ERR_INVALID_ARG;
+  if (!h->ev_valid) return fail(h, MOE_VQLR_ERR_INVALID_ARG, "no profiled call to report");
+  cudaError_t ce = cudaEventSynchronize(h->ev[kStages]);
+  if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "event sync: %s", cudaGetErrorString(ce));
+  for (int i = 0; i < kStages; ++i) {
+    ms_out[i] = 0.f;
+    if (h->stage_ran[i]) {
+      ce = cudaEventElapsedTime(&ms_out[i], h->ev[i], h->ev[i + 1]);
+      if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "elapsed: %s", cudaGetErrorString(ce));
+    }
+  }
+  return MOE_VQLR_OK;
 }
 
 int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h) { return h ? h->launches : 0; }
