@@ -155,6 +155,30 @@ int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h);
 /* Device workspace the handle owns, in bytes. */
 int64_t moe_vqlr_workspace_bytes(const moe_vqlr_handle* h);
 
+/* Routing step only, for callers that must not allocate device memory (no counterpart in the
+ * paper: it exists for processes where a memory pool or the host application owns every
+ * allocation, so moe_vqlr_create(), which allocates a workspace, is off limits).  Computes
+ *   logit[t][e] = <router_w[e], x[t]> (+ router_bias[e]),  the k best experts per token (ties:
+ *   lower id) and their affinities, exactly as moe_vqlr_decode_layer does,
+ * and writes topk_id[T][k] (int32) and topk_w[T][k] (fp32).  All pointers are DEVICE pointers;
+ * x [T][H] bf16 and router_w [E][H] bf16 must be 16-byte aligned, H a multiple of 8;
+ * router_bias [E] fp32 may be NULL.  Asynchronous on cuda_stream.
+ *
+ * The only scratch, the [T][E] fp32 logits, lives in a fixed 64 KiB array inside the library's
+ * device image (held by every GPU that loads the library until the process exits).  Hence:
+ *   - limits: T <= 16, E <= 1024, k <= 32; anything larger returns MOE_VQLR_ERR_UNSUPPORTED and
+ *     launches nothing;
+ *   - no cudaMalloc / cudaFree / allocating library call is made, ever;
+ *   - all calls on one device share the array: calls that overlap on the GPU race, so keep them
+ *     on one stream or order them yourself.  Each call rewrites every entry it reads; nothing
+ *     carried over from an earlier call is used;
+ *   - the first call on each device resolves the array's device address (with that device
+ *     current); issue that first call outside any stream capture.
+ * Returns MOE_VQLR_OK, ERR_INVALID_ARG, ERR_UNSUPPORTED or ERR_CUDA. */
+int moe_vqlr_route_noalloc(const void* x, const void* router_w, const float* router_bias,
+                           int32_t T, int32_t E, int32_t H, int32_t k, int32_t renorm_topk,
+                           int32_t* topk_id, float* topk_w, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,7 @@ FLAG_VALIDATE_INDICES = 1
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",
            "moe_vqlr_workspace_bytes", "moe_vqlr_set_profiling", "moe_vqlr_last_stage_times",
-           "moe_vqlr_stage_count", "moe_vqlr_stage_name"]
+           "moe_vqlr_stage_count", "moe_vqlr_stage_name", "moe_vqlr_route_noalloc"]
 
 
 class MoeVqlrError(RuntimeError):
@@ -82,6 +82,9 @@ def _load():
     lib.moe_vqlr_stage_count.argtypes = []
     lib.moe_vqlr_stage_name.restype = C.c_char_p
     lib.moe_vqlr_stage_name.argtypes = [C.c_int32]
+    lib.moe_vqlr_route_noalloc.restype = C.c_int
+    lib.moe_vqlr_route_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 5 + \
+                                          [C.c_void_p, C.c_void_p, C.c_void_p]
     return lib
 
 
@@ -105,6 +108,23 @@ def bits_to_device(a: Optional[np.ndarray], device) -> Optional[torch.Tensor]:
 
 def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def route_noalloc(x: torch.Tensor, router_w: torch.Tensor, router_bias: Optional[torch.Tensor],
+                  k: int, topk_id: torch.Tensor, topk_w: torch.Tensor, renorm_topk: bool = True,
+                  stream: Optional[torch.cuda.Stream] = None) -> int:
+    """Routing only, for callers that must not allocate on the device: the library keeps the
+    logits in a fixed array of its own and makes no allocation.  The caller supplies the output
+    tensors (topk_id [T][k] int32, topk_w [T][k] float32).  Limits: T <= 16, E <= 1024, k <= 32;
+    calls on one device must not overlap.  Returns the status code (no exception), so that the
+    caller can test the limits."""
+    T, H = x.shape
+    E = router_w.shape[0]
+    st = stream or torch.cuda.current_stream(x.device)
+    with torch.cuda.device(x.device):
+        return int(_lib.moe_vqlr_route_noalloc(_ptr(x), _ptr(router_w), _ptr(router_bias), T, E, H, k,
+                                               1 if renorm_topk else 0, _ptr(topk_id), _ptr(topk_w),
+                                               C.c_void_p(st.cuda_stream)))
 
 
 class MoeVqlrLayer:
