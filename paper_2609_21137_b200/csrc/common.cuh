@@ -1,0 +1,82 @@
+// Shared definitions of the CUDA kernels: parameter block, bf16 helpers, warp reductions.
+#pragma once
+#include "moe_vqlr.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace {
+
+constexpr int kMaxT = 16;      // tokens per call
+constexpr int kMaxK = 32;      // experts per token
+constexpr int kD = 8;          // VQ block length (one code word = 16 bytes of bf16)
+constexpr int kTokGroup = 4;   // tokens of one expert handled per pass over its row
+constexpr int kStages = 6;     // router_z, route, gateup, zdown, down, combine
+const char* const kStageNames[kStages] = {"router_z", "route", "gateup", "zdown", "down", "combine"};
+
+typedef __nv_bfloat16 bf16;
+
+struct ProjDev {
+  int kind;
+  int out_dim, in_dim;
+  int zslot;               // which z slot feeds the low-rank term (gate/up), -1 if none
+  const uint4* codebook;   // [K] code words of 8 bf16
+  const void* idx;
+  const bf16* basis;
+  const bf16* factor;
+  const bf16* dense;
+};
+
+struct Params {
+  int H, I, E, k, S, K, r, renorm;
+  int n_zrows;             // rows of the stacked basis projection: (distinct gate/up bases) * r
+  const bf16* router_w;
+  const float* router_bias;
+  ProjDev gate, up, down;
+  // workspace
+  float* logits;           // [maxT][E]
+  float* z;                // [maxT][2][r]
+  int* topk_id;            // [maxT][k]
+  float* topk_w;           // [maxT][k]
+  int* counts;             // [E]
+  int* offsets;            // [E+1]
+  int* pair_token;         // [maxT*(k+S)]  routed pairs sorted by expert, then shared experts' pairs
+  int* pair_slot;          // [maxT*(k+S)]
+  float* pair_w;           // [maxT*(k+S)]
+  int* act_n;              // [1] number of active experts (routed with >=1 pair, then shared)
+  int* act_e;              // [E+S] expert id
+  int* act_off;            // [E+S] first pair position
+  int* act_cnt;            // [E+S] pairs
+  float* p;                // [maxT*(k+S)][I]   SwiGLU intermediate per pair position
+  float* zd;               // [maxT*(k+S)][r]   basis_down * p per pair position
+  float* y;                // [maxT][k+S][H]    expert outputs before the weighted sum
+  int* status;             // [1]
+};
+
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  f[0] = bf_lo(v.x); f[1] = bf_hi(v.x); f[2] = bf_lo(v.y); f[3] = bf_hi(v.y);
+  f[4] = bf_lo(v.z); f[5] = bf_hi(v.z); f[6] = bf_lo(v.w); f[7] = bf_hi(v.w);
+}
+
+__device__ __forceinline__ float dot8(const float (&a)[8], const float (&b)[8], float acc) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc = fmaf(a[j], b[j], acc);
+  return acc;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Position of 16-byte block b of an activation row in shared memory.  Lane l of a warp walks
+// blocks 8l..8l+7; XOR-ing the low three bits with l keeps the eight lanes of a quarter warp on
+// distinct bank groups.
+__device__ __forceinline__ int swz(int b) { return b ^ ((b >> 3) & 7); }
+
+}  // namespace

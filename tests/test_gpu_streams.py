@@ -1,0 +1,83 @@
+"""The same layer through the other launch routes: a side stream (kernels chained by
+programmatic dependent launch), a captured CUDA graph, and the generic kernels forced on a
+shape the tensor-core kernels would normally take."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_21137_b200 import synth
+
+from helpers import assert_output, assert_routing, bf16_tensor_to_f64, make_checked_layer
+
+pytestmark = pytest.mark.gpu
+
+CASES = [synth.shape("tiny", T=3), synth.shape("qwen3", E=16), synth.shape("qwen3_b16", E=32),
+         synth.shape("qwen3", E=16, mode="paper"), synth.shape("dsv2lite_b8", E=16),
+         synth.shape("tiny", T=2, mode="dense")]
+
+
+@pytest.mark.parametrize("shp", CASES, ids=lambda s: f"{s.name}-{s.mode}")
+def test_side_stream_back_to_back(shp):
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    x = binding.bits_to_device(layer.x, "cuda")
+    st = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(st):
+        outs = [mod.decode(x, stream=st) for _ in range(3)]      # three chained calls
+        out, dbg = mod.decode(x, debug=True, stream=st)
+    st.synchronize()
+    assert_routing(dbg, res)
+    ref = bf16_tensor_to_f64(out)
+    assert_output(ref, res.out)
+    for o in outs:
+        assert torch.equal(o.view(torch.int16), out.view(torch.int16))
+    mod.close()
+
+
+def test_graph_capture_replay():
+    from paper_2609_21137_b200 import binding
+    shapes = [synth.shape("qwen3", E=16), synth.shape("qwen3_b16", E=32, mode="paper")]
+    mods, xs, outs, refs = [], [], [], []
+    for shp in shapes:
+        layer, res, _ = make_checked_layer(shp, 0)
+        mods.append(binding.MoeVqlrLayer.from_synth(layer, device="cuda"))
+        xs.append(binding.bits_to_device(layer.x, "cuda"))
+        outs.append(torch.zeros((shp.T, shp.H), dtype=torch.bfloat16, device="cuda"))
+        refs.append(res.out)
+    graph = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph):
+        for _ in range(2):
+            for m, x, o in zip(mods, xs, outs):
+                m.decode(x, out=o)
+    for _ in range(2):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for o, ref in zip(outs, refs):
+            assert_output(bf16_tensor_to_f64(o), ref)
+    for m in mods:
+        m.close()
+
+
+@pytest.mark.parametrize("shp", [synth.shape("tiny", T=5), synth.shape("qwen3", E=16, T=3, mode="paper")],
+                         ids=lambda s: f"{s.name}-{s.mode}")
+def test_generic_kernels_forced(shp):
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    os.environ["MOE_VQLR_FORCE_GENERIC"] = "1"
+    try:
+        mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    finally:
+        del os.environ["MOE_VQLR_FORCE_GENERIC"]
+    x = binding.bits_to_device(layer.x, "cuda")
+    out, dbg = mod.decode(x, debug=True)
+    torch.cuda.synchronize()
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out)
+    mod.close()
