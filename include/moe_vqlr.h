@@ -121,7 +121,9 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
 /* Same layer with HOST buffers: copies x (T*H bf16, host) to the device, runs the layer, copies
  * out (T*H bf16) back and waits for the stream.  Pinned host memory makes the copies
  * asynchronous up to the final wait; pageable memory works but is slower.  Weights stay on
- * the device.  Synchronous on return. */
+ * the device.  Synchronous on return.  The first call for each T captures the kernel chain into
+ * a CUDA graph owned by the handle (later calls replay it), so that first call is slower and
+ * must not itself run inside a stream capture. */
 int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T, void* out_host,
                                void* cuda_stream);
 
@@ -148,6 +150,14 @@ int moe_vqlr_last_stage_times(moe_vqlr_handle* h, float* ms_out, int32_t cap);
 
 int moe_vqlr_stage_count(void);
 const char* moe_vqlr_stage_name(int32_t i);
+
+/* Measurement aid (no counterpart in the paper): enqueues the kernel of ONE stage of the layer
+ * on cuda_stream, with the same arguments as moe_vqlr_decode_layer, reading whatever the
+ * previous stages of an earlier full call on this handle (same x, same T) left in the
+ * workspace.  Lets a benchmark time a single kernel back to back, e.g. inside a captured graph.
+ * A stage the configuration does not have enqueues nothing and returns MOE_VQLR_OK. */
+int moe_vqlr_run_stage(moe_vqlr_handle* h, int32_t stage, const void* x, int32_t T, void* out,
+                       void* cuda_stream);
 
 /* Number of kernel launches this handle has enqueued since create(). */
 int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h);

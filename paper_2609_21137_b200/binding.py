@@ -22,7 +22,8 @@ FLAG_VALIDATE_INDICES = 1
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",
            "moe_vqlr_workspace_bytes", "moe_vqlr_set_profiling", "moe_vqlr_last_stage_times",
-           "moe_vqlr_stage_count", "moe_vqlr_stage_name", "moe_vqlr_route_noalloc"]
+           "moe_vqlr_stage_count", "moe_vqlr_stage_name", "moe_vqlr_route_noalloc",
+           "moe_vqlr_run_stage"]
 
 
 class MoeVqlrError(RuntimeError):
@@ -82,6 +83,8 @@ def _load():
     lib.moe_vqlr_stage_count.argtypes = []
     lib.moe_vqlr_stage_name.restype = C.c_char_p
     lib.moe_vqlr_stage_name.argtypes = [C.c_int32]
+    lib.moe_vqlr_run_stage.restype = C.c_int
+    lib.moe_vqlr_run_stage.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     lib.moe_vqlr_route_noalloc.restype = C.c_int
     lib.moe_vqlr_route_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 5 + \
                                           [C.c_void_p, C.c_void_p, C.c_void_p]
@@ -221,6 +224,14 @@ class MoeVqlrLayer:
         self._check(_lib.moe_vqlr_decode_layer_host(self._h, _ptr(x_host), T, _ptr(out_host),
                                                     C.c_void_p(st.cuda_stream)))
         return out_host
+
+    def run_stage(self, stage: str, x: torch.Tensor, out: torch.Tensor,
+                  stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Enqueue one stage's kernel only (measurement aid; needs an earlier full call)."""
+        names = [_lib.moe_vqlr_stage_name(i).decode() for i in range(_lib.moe_vqlr_stage_count())]
+        st = stream or torch.cuda.current_stream(x.device)
+        self._check(_lib.moe_vqlr_run_stage(self._h, names.index(stage), _ptr(x), x.shape[0], _ptr(out),
+                                            C.c_void_p(st.cuda_stream)))
 
     def set_profiling(self, on: bool) -> None:
         self._check(_lib.moe_vqlr_set_profiling(self._h, 1 if on else 0))

@@ -27,7 +27,8 @@
 namespace {
 
 constexpr int kFastThreads = 512;
-constexpr int kDenseThreads = 384;   // dense weight tiles in flight need more registers per thread
+constexpr int kDenseThreads = 384;   // dense gate/up: weight tiles in flight need more registers per thread
+constexpr int kDownThreads = 384;    // down: hi + lo activation fragments need 64 registers per thread
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -100,6 +101,7 @@ struct StagePlan {
   int n_teams;     // teams per block
   int tiles;       // row tiles per expert = out_dim / 8
   int n_lr;        // groups of 32 ranks = ceil(r / 32), 0 without a low-rank term
+  int depth;       // tiles each warp keeps in flight in its shared-memory ring (2..4)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -243,14 +245,22 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
 }
 
 // ---------------------------------------------------------------------------------------------
-// k_router_z_pdl: same arithmetic and summation order as k_router_z, as the head of the chain.
+// k_router_z_pdl: head of the chain.  One warp per (row of [router_w ; basis_gate ; basis_up],
+// group of four tokens).  Per (row, token) the summation order is the one of k_router_z
+// (lane-strided 16-byte chunks, sequential FMAs inside a chunk, xor butterfly), so identical
+// router rows give bitwise identical logits.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
+constexpr int kRouterWarps = 2;
+
+__global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
   pdl_wait();      // the previous call's kernels may still read logits / z
   pdl_launch();
   const int lane = threadIdx.x & 31;
-  const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  if (row >= P.E + P.n_zrows) return;
+  const int unit = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
+  const int n_rows = P.E + P.n_zrows;
+  const int n_groups = (T + kTokGroup - 1) / kTokGroup;
+  if (unit >= n_rows * n_groups) return;
+  const int row = unit / n_groups, t0 = (unit - row * n_groups) * kTokGroup;
   const bf16* wrow;
   float* dst;
   int dst_stride;
@@ -270,54 +280,116 @@ __global__ void __launch_bounds__(256) k_router_z_pdl(const Params P, const bf16
   }
   const int nchunk = P.H / 8;
   const uint4* w4 = reinterpret_cast<const uint4*>(wrow);
-  for (int t0 = 0; t0 < T; t0 += kTokGroup) {
-    float acc[kTokGroup] = {0.f, 0.f, 0.f, 0.f};
-    for (int c = lane; c < nchunk; c += 32) {
-      float wf[8];
-      unpack8(__ldg(w4 + c), wf);
+  const int nt = min(kTokGroup, T - t0);
+  float acc[kTokGroup] = {0.f, 0.f, 0.f, 0.f};
+  for (int c0 = 0; c0 < nchunk; c0 += 32 * 4) {          // four chunks per lane in flight
+    uint4 wv[4], xv[4][kTokGroup];
 #pragma unroll
-      for (int tt = 0; tt < kTokGroup; ++tt) {
-        if (t0 + tt < T) {
+    for (int q = 0; q < 4; ++q) {
+      const int c = c0 + q * 32 + lane;
+      wv[q] = c < nchunk ? __ldg(w4 + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int tt = 0; tt < kTokGroup; ++tt)
+        xv[q][tt] = (c < nchunk && tt < nt) ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(t0 + tt) * P.H) + c)
+                                            : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (c0 + q * 32 + lane < nchunk) {
+        float wf[8];
+        unpack8(wv[q], wf);
+#pragma unroll
+        for (int tt = 0; tt < kTokGroup; ++tt) {
           float xf[8];
-          unpack8(__ldg(reinterpret_cast<const uint4*>(x + (size_t)(t0 + tt) * P.H) + c), xf);
+          unpack8(xv[q][tt], xf);
           acc[tt] = dot8(wf, xf, acc[tt]);
         }
       }
     }
+  }
 #pragma unroll
-    for (int tt = 0; tt < kTokGroup; ++tt) {
-      const float s = warp_sum(acc[tt]);
-      if (lane == 0 && t0 + tt < T) dst[(size_t)(t0 + tt) * dst_stride] = s + bias;
-    }
+  for (int tt = 0; tt < kTokGroup; ++tt) {
+    const float sum = warp_sum(acc[tt]);
+    if (lane == 0 && tt < nt) dst[(size_t)(t0 + tt) * dst_stride] = sum + bias;
   }
 }
 
 // ---------------------------------------------------------------------------------------------
-// k_gateup_mma
+// Asynchronous copies: every warp streams the bytes it will need (indices, factor rows, dense
+// weight rows) into a private shared-memory ring several tiles ahead, so that HBM latency is
+// hidden without holding the data in registers.
 // ---------------------------------------------------------------------------------------------
-__host__ __device__ inline size_t gu_part_bytes(const StagePlan& pl) {
-  // [buffer 2][team][projection 2][warp][lane 32] float2
-  return (size_t)2 * pl.n_teams * 2 * pl.team_warps * 32 * 8;
+__device__ __forceinline__ void cp_async16(void* smem, const void* gptr) {
+  const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* smem, const void* gptr) {
+  const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(sa), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// waits until at most `pending` of this thread's copy groups are still in flight
+__device__ __forceinline__ void cp_async_wait_pending(int pending) {
+  switch (pending) {
+    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+  }
+}
+template <typename IdxT>
+__device__ __forceinline__ void cp_async_idx8(uint4* smem, const IdxT* gptr) {
+  if (sizeof(IdxT) == 2) cp_async16(smem, gptr); else cp_async8(smem, gptr);
+}
+template <typename IdxT>
+__device__ __forceinline__ uint4 ring_idx8(const uint4* smem) {
+  if (sizeof(IdxT) == 2) return *smem;
+  const uint2 v = *reinterpret_cast<const uint2*>(smem);
+  return make_uint4(v.x, v.y, 0u, 0u);
 }
 
-__host__ __device__ inline size_t gu_smem_bytes(int K, int n_books, int T, int H, const StagePlan& pl,
-                                                int E, int k, int S) {
-  return (size_t)n_books * K * 16 + (size_t)T * (H / 8 + 1) * 16 + gu_part_bytes(pl) +
-         route_smem_bytes(T, E, k, S);
+constexpr int kMaxDepth = 4;
+
+// ---------------------------------------------------------------------------------------------
+// k_gateup_mma
+// ---------------------------------------------------------------------------------------------
+struct GuLayout {         // byte offsets into dynamic shared memory
+  size_t cb_u, x, ring, fring, z, part, route, total;
+};
+
+__host__ __device__ inline GuLayout gu_layout(int K, int n_books, int T, int H, int r, const StagePlan& pl,
+                                              int warps, int E, int k, int S) {
+  GuLayout L;
+  size_t o = 0;
+  L.cb_u = n_books == 2 ? (size_t)K * 16 : 0;
+  o = (size_t)n_books * K * 16;
+  L.x = o;      o += (size_t)T * (H / 8 + 1) * 16;
+  L.ring = o;   o += (size_t)warps * pl.depth * 2 * 32 * 16;
+  L.fring = o;  o += (size_t)pl.n_teams * (pl.n_lr > 0 ? pl.n_lr : 0) * pl.depth * 2 * 32 * 16;
+  L.z = o;      o += (size_t)2 * T * 2 * ((r + 7) / 8) * 16;            // hi and lo blocks of z
+  L.part = o;   o += (size_t)2 * pl.n_teams * 2 * pl.team_warps * 32 * 8;
+  L.route = o;  o += route_smem_bytes(T, E, k, S);
+  L.total = o;
+  return L;
 }
 
 template <typename IdxT, bool DENSE>
 __global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
 k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books) {
   extern __shared__ uint4 s_u4[];
+  char* s_base = reinterpret_cast<char*>(s_u4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, c = lane & 3;
-  const int nb = pl.nb, xs = nb + 1;
+  const int nb = pl.nb, xs = nb + 1, D = pl.depth, rb = (P.r + 7) / 8;
+  const GuLayout L = gu_layout(P.K, n_books, T, P.H, P.r, pl, blockDim.x >> 5, P.E, P.k, P.S);
   uint4* s_cb_g = s_u4;
-  uint4* s_cb_u = n_books == 2 ? s_u4 + P.K : s_u4;
-  uint4* s_x = s_u4 + (size_t)n_books * P.K;
-  float2* s_part = reinterpret_cast<float2*>(s_x + (size_t)T * xs);
-  char* s_route = reinterpret_cast<char*>(s_part) + gu_part_bytes(pl);
-  const RouteSmem R = carve_route(s_route, T, P.E, P.k, P.S);
+  uint4* s_cb_u = reinterpret_cast<uint4*>(s_base + L.cb_u);
+  uint4* s_x = reinterpret_cast<uint4*>(s_base + L.x);
+  uint4* s_ring = reinterpret_cast<uint4*>(s_base + L.ring);
+  uint4* s_fring = reinterpret_cast<uint4*>(s_base + L.fring);
+  uint4* s_zh = reinterpret_cast<uint4*>(s_base + L.z);          // [T][2][rb]
+  uint4* s_zl = s_zh + (size_t)T * 2 * rb;
+  float2* s_part = reinterpret_cast<float2*>(s_base + L.part);
+  const RouteSmem R = carve_route(s_base + L.route, T, P.E, P.k, P.S);
 
   // ---- prologue that does not depend on the routing: code books and tokens -------------------
   if (!DENSE) {
@@ -333,6 +405,11 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
     }
   }
   pdl_wait();      // logits and z of this call are complete
+  if (pl.n_lr > 0)
+    for (int i = tid; i < T * 2 * rb; i += blockDim.x) {      // z as bf16 hi / lo blocks
+      const float* zp = P.z + (size_t)i * 8;                   // z is [T][2][r], r a multiple of 8
+      split_hi_lo(*reinterpret_cast<const float4*>(zp), *reinterpret_cast<const float4*>(zp + 4), s_zh[i], s_zl[i]);
+    }
   route_in_block(P, T, R, blockIdx.x == 0);
   pdl_launch();
 
@@ -342,40 +419,68 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   const int n_act = *R.n_act;
   const long long U = (long long)n_act * pl.tiles;
   const long long G = (long long)gridDim.x * pl.n_teams, tau = (long long)blockIdx.x * pl.n_teams + team;
-  const long long u_begin = tau * U / G, u_end = (tau + 1) * U / G;
-  const int spw_one = pl.n_slices <= pl.team_warps;          // one slice per warp: fragments stay put
+  const long long u_begin = tau * U / G;
+  const int n_my = team < pl.n_teams ? (int)((tau + 1) * U / G - u_begin) : 0;
+  const bool spw_one = pl.n_slices <= pl.team_warps;         // one slice per warp: fragments stay put
+  const bool ringed = !DENSE && spw_one;
   // low-rank group handled by this warp (groups are dealt from the last warp of the team down)
   const int lr_group = pl.team_warps - 1 - wi;
-  const bool has_lr = lr_group < pl.n_lr;   // n_lr is 0 for a dense projection
-
-  uint4 fx[8];                       // activation fragments of the current slice
-  uint4 zgh = {0, 0, 0, 0}, zgl = {0, 0, 0, 0}, zuh = {0, 0, 0, 0}, zul = {0, 0, 0, 0};
-  int frag_a = -1, frag_pass = -1, frag_slice = -1, z_a = -1, z_pass = -1, z_lg = -1;
-  int buf = 0;
+  const bool has_lr = lr_group < pl.n_lr;                    // n_lr is 0 for a dense projection
+  const int b_first = wi * 32 + 8 * c, rho_first = lr_group * 32 + 8 * c;
+  const bool idx_live = b_first < nb, fac_live = has_lr && rho_first < P.r;
 
   const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
   const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx);
+  uint4* ring = s_ring + (size_t)warp * D * 2 * 32;                                   // [slot][proj][lane]
+  uint4* fring = s_fring + (size_t)(team * pl.n_lr + (has_lr ? lr_group : 0)) * D * 2 * 32;
 
-  for (long long u = u_begin; u < u_end; ++u) {
+  auto tile_row = [&](int i) -> size_t {                     // this lane's weight row of the team's i-th tile
+    const long long u = u_begin + i;
+    const int a = (int)(u / pl.tiles), jt = (int)(u - (long long)a * pl.tiles);
+    return (size_t)R.act_e[a] * P.I + jt * 8 + g;
+  };
+  auto issue = [&](int i) {
+    const size_t row = tile_row(i);
+    const int slot = i % D;
+    if (ringed && idx_live) {
+      cp_async_idx8<IdxT>(ring + (slot * 2 + 0) * 32 + lane, idx_g + row * nb + b_first);
+      cp_async_idx8<IdxT>(ring + (slot * 2 + 1) * 32 + lane, idx_u + row * nb + b_first);
+    }
+    if (fac_live) {
+      cp_async16(fring + (slot * 2 + 0) * 32 + lane, P.gate.factor + row * P.r + rho_first);
+      cp_async16(fring + (slot * 2 + 1) * 32 + lane, P.up.factor + row * P.r + rho_first);
+    }
+  };
+
+  uint4 fx[8];                       // activation fragments of the current slice
+  int frag_a = -1, frag_pass = -1, frag_slice = -1;
+  int buf = 0;
+
+  for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(i); cp_async_commit(); }
+  for (int i = 0; i < n_my; ++i) {
+    if (i + D - 1 < n_my) issue(i + D - 1);
+    cp_async_commit();
+    cp_async_wait_pending(D - 1);
+    const long long u = u_begin + i;
     const int a = (int)(u / pl.tiles), jt = (int)(u - (long long)a * pl.tiles);
     const int e = R.act_e[a], off = R.act_off[a], cnt = R.act_cnt[a];
     const size_t row = (size_t)e * P.I + jt * 8 + g;       // this lane's weight row
-    // index registers of the first slice are fetched once per tile and reused by every pass
+    const int slot = i % D;
     uint4 raw_g = {0, 0, 0, 0}, raw_u = {0, 0, 0, 0};
     uint4 fac_g = {0, 0, 0, 0}, fac_u = {0, 0, 0, 0};
-    const int b_first = wi * 32 + 8 * c;
-    if (!DENSE && spw_one && b_first < nb) {
-      raw_g = load_idx_raw<IdxT>(idx_g + row * nb + b_first);
-      raw_u = load_idx_raw<IdxT>(idx_u + row * nb + b_first);
+    if (ringed && idx_live) {
+      raw_g = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32 + lane);
+      raw_u = ring_idx8<IdxT>(ring + (slot * 2 + 1) * 32 + lane);
     }
-    if (has_lr && lr_group * 32 + 8 * c < P.r) {
-      fac_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + row * P.r + lr_group * 32 + 8 * c));
-      fac_u = __ldg(reinterpret_cast<const uint4*>(P.up.factor + row * P.r + lr_group * 32 + 8 * c));
+    if (fac_live) {
+      fac_g = fring[(slot * 2 + 0) * 32 + lane];
+      fac_u = fring[(slot * 2 + 1) * 32 + lane];
     }
     for (int pass = 0; pass * 8 < cnt; ++pass) {
       const int n_tok = min(8, cnt - pass * 8);
       const int tok = g < n_tok ? R.pair_token[off + pass * 8 + g] : -1;
-      float acc_g[4] = {0.f, 0.f, 0.f, 0.f}, acc_u[4] = {0.f, 0.f, 0.f, 0.f};
+      float acc_g[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      float acc_u[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
       for (int sl = wi; sl < pl.n_slices; sl += pl.team_warps) {
         const int b0 = sl * 32 + (DENSE ? c : 8 * c);
         if (frag_a != a || frag_pass != pass || frag_slice != sl) {
@@ -397,9 +502,9 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
             vu[j] = b < nb ? __ldg(wu + b) : make_uint4(0, 0, 0, 0);
           }
 #pragma unroll
-          for (int j = 0; j < 8; ++j) { mma_block(acc_g, fx[j], vg[j]); mma_block(acc_u, fx[j], vu[j]); }
+          for (int j = 0; j < 8; ++j) { mma_block(acc_g[j & 1], fx[j], vg[j]); mma_block(acc_u[j & 1], fx[j], vu[j]); }
         } else {
-          if (!spw_one) {
+          if (!ringed) {
             if (b0 < nb) {
               raw_g = load_idx_raw<IdxT>(idx_g + row * nb + b0);
               raw_u = load_idx_raw<IdxT>(idx_u + row * nb + b0);
@@ -414,8 +519,8 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
           unpack_idx8<IdxT>(raw_u, iu);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            mma_block(acc_g, fx[j], s_cb_g[ig[j]]);
-            mma_block(acc_u, fx[j], s_cb_u[iu[j]]);
+            mma_block(acc_g[j & 1], fx[j], s_cb_g[ig[j]]);
+            mma_block(acc_u[j & 1], fx[j], s_cb_u[iu[j]]);
           }
         }
       }
@@ -430,24 +535,18 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
             fu = __ldg(reinterpret_cast<const uint4*>(P.up.factor + row * P.r + rho0));
           }
         }
-        if (z_a != a || z_pass != pass || z_lg != lg) {
-          if (tok >= 0 && rho0 < P.r) {
-            const float* zg = P.z + ((size_t)tok * 2 + P.gate.zslot) * P.r + rho0;
-            const float* zu = P.z + ((size_t)tok * 2 + P.up.zslot) * P.r + rho0;
-            split_hi_lo(*reinterpret_cast<const float4*>(zg), *reinterpret_cast<const float4*>(zg + 4), zgh, zgl);
-            split_hi_lo(*reinterpret_cast<const float4*>(zu), *reinterpret_cast<const float4*>(zu + 4), zuh, zul);
-          } else {
-            zgh = zgl = zuh = zul = make_uint4(0, 0, 0, 0);
-          }
-          z_a = a; z_pass = pass; z_lg = lg;
+        uint4 zgh = {0, 0, 0, 0}, zgl = {0, 0, 0, 0}, zuh = {0, 0, 0, 0}, zul = {0, 0, 0, 0};
+        if (tok >= 0 && rho0 < P.r) {
+          const int ig2 = (tok * 2 + P.gate.zslot) * rb + (rho0 >> 3), iu2 = (tok * 2 + P.up.zslot) * rb + (rho0 >> 3);
+          zgh = s_zh[ig2]; zgl = s_zl[ig2]; zuh = s_zh[iu2]; zul = s_zl[iu2];
         }
-        mma_block(acc_g, zgh, fg); mma_block(acc_g, zgl, fg);
-        mma_block(acc_u, zuh, fu); mma_block(acc_u, zul, fu);
+        mma_block(acc_g[0], zgh, fg); mma_block(acc_g[1], zgl, fg);
+        mma_block(acc_u[0], zuh, fu); mma_block(acc_u[1], zul, fu);
       }
       // ---- add the team's partial tiles and apply SwiGLU -----------------------------------
       float2* part = s_part + ((size_t)(buf * pl.n_teams + team) * 2) * pl.team_warps * 32;
-      part[(0 * pl.team_warps + wi) * 32 + lane] = make_float2(acc_g[0], acc_g[1]);
-      part[(1 * pl.team_warps + wi) * 32 + lane] = make_float2(acc_u[0], acc_u[1]);
+      part[(0 * pl.team_warps + wi) * 32 + lane] = make_float2(acc_g[0][0] + acc_g[1][0], acc_g[0][1] + acc_g[1][1]);
+      part[(1 * pl.team_warps + wi) * 32 + lane] = make_float2(acc_u[0][0] + acc_u[1][0], acc_u[0][1] + acc_u[1][1]);
       if (pl.team_warps > 1) team_sync(1 + team, team_threads); else __syncwarp();
       for (int q = tid_team; q < 64; q += team_threads) {
         const int m = q >> 3, n = q & 7;                      // token m of this pass, row n of the tile
@@ -466,28 +565,43 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
       buf ^= 1;
     }
   }
+  cp_async_wait_pending(0);
 }
 
 // ---------------------------------------------------------------------------------------------
 // k_down_mma: y[token][slot][h] for every (expert, 8-row tile of H); activations are the fp32
 // intermediates p split into bf16 hi + lo fragments.
 // ---------------------------------------------------------------------------------------------
-__host__ __device__ inline size_t dn_part_bytes(const StagePlan& pl) {
-  return (size_t)2 * pl.n_teams * pl.team_warps * 32 * 8;
-}
+struct DnLayout {
+  size_t ring, fring, part, yrow, total;
+  int slot_u4;      // uint4 per lane per ring slot: 1 (indices) or 8 (a dense 256-value slice of a row)
+};
 
-__host__ __device__ inline size_t dn_smem_bytes(int K, bool vq, const StagePlan& pl) {
-  return (vq ? (size_t)K * 16 : 0) + dn_part_bytes(pl);
+__host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& pl, int warps) {
+  DnLayout L;
+  size_t o = vq ? (size_t)K * 16 : 0;
+  L.slot_u4 = vq ? 1 : 8;
+  L.ring = o;   o += (size_t)warps * pl.depth * L.slot_u4 * 32 * 16;
+  L.fring = o;  o += (size_t)pl.n_teams * (pl.n_lr > 0 ? pl.n_lr : 0) * pl.depth * 32 * 16;
+  L.part = o;   o += (size_t)2 * pl.n_teams * pl.team_warps * 32 * 8;
+  L.yrow = o;   o += (size_t)2 * pl.n_teams * 8 * 8;
+  L.total = o;
+  return L;
 }
 
 template <typename IdxT, bool DENSE>
-__global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
+__global__ void __launch_bounds__(kDownThreads, 1)
 k_down_mma(const Params P, int T, const StagePlan pl) {
   extern __shared__ uint4 s_u4[];
+  char* s_base = reinterpret_cast<char*>(s_u4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, c = lane & 3;
-  const int nb = pl.nb;
+  const int nb = pl.nb, D = pl.depth;
+  const DnLayout L = dn_layout(P.K, !DENSE, pl, blockDim.x >> 5);
   uint4* s_cb = s_u4;
-  float2* s_part = reinterpret_cast<float2*>(s_u4 + (DENSE ? 0 : P.K));
+  uint4* s_ring = reinterpret_cast<uint4*>(s_base + L.ring);
+  uint4* s_fring = reinterpret_cast<uint4*>(s_base + L.fring);
+  float2* s_part = reinterpret_cast<float2*>(s_base + L.part);
+  long long* s_yrow = reinterpret_cast<long long*>(s_base + L.yrow);   // [buf][team][8] output row offsets
   if (!DENSE)
     for (int i = tid; i < P.K; i += blockDim.x) s_cb[i] = __ldg(P.down.codebook + i);
   pdl_wait();      // p (and z_d) and the routing lists are complete
@@ -501,30 +615,59 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   const int n_slots = P.k + P.S;
   const long long U = (long long)n_act * pl.tiles;
   const long long G = (long long)gridDim.x * pl.n_teams, tau = (long long)blockIdx.x * pl.n_teams + team;
-  const long long u_begin = tau * U / G, u_end = (tau + 1) * U / G;
-  const int spw_one = pl.n_slices <= pl.team_warps;
+  const long long u_begin = tau * U / G;
+  const int n_my = team < pl.n_teams ? (int)((tau + 1) * U / G - u_begin) : 0;
+  const bool spw_one = pl.n_slices <= pl.team_warps;
+  const bool ringed = spw_one;
   const int lr_group = pl.team_warps - 1 - wi;
   const bool has_lr = lr_group < pl.n_lr;
+  const int b_first = wi * 32 + (DENSE ? c : 8 * c), rho_first = lr_group * 32 + 8 * c;
+  const bool idx_live = DENSE ? (wi * 32 < nb) : (b_first < nb), fac_live = has_lr && rho_first < P.r;
+
+  const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
+  uint4* ring = s_ring + (size_t)warp * D * L.slot_u4 * 32;                        // [slot][chunk][lane]
+  uint4* fring = s_fring + (size_t)(team * pl.n_lr + (has_lr ? lr_group : 0)) * D * 32;
+
+  auto issue = [&](int i) {
+    const long long u = u_begin + i;
+    const int a = (int)(u / pl.tiles), jt = (int)(u - (long long)a * pl.tiles);
+    const size_t row = (size_t)P.act_e[a] * P.H + jt * 8 + g;
+    const int slot = i % D;
+    if (ringed && idx_live) {
+      if (DENSE) {
+        const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (b_first + 4 * j < nb) cp_async16(ring + (slot * 8 + j) * 32 + lane, wd + b_first + 4 * j);
+      } else {
+        cp_async_idx8<IdxT>(ring + slot * 32 + lane, idx_d + row * nb + b_first);
+      }
+    }
+    if (fac_live) cp_async16(fring + slot * 32 + lane, P.down.factor + row * P.r + rho_first);
+  };
 
   uint4 fh[8], fl[8];
   uint4 zh = {0, 0, 0, 0}, zl = {0, 0, 0, 0};
   int frag_a = -1, frag_pass = -1, frag_slice = -1, z_a = -1, z_pass = -1, z_lg = -1;
   int buf = 0;
-  const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
 
-  for (long long u = u_begin; u < u_end; ++u) {
+  for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(i); cp_async_commit(); }
+  for (int i = 0; i < n_my; ++i) {
+    if (i + D - 1 < n_my) issue(i + D - 1);
+    cp_async_commit();
+    cp_async_wait_pending(D - 1);
+    const long long u = u_begin + i;
     const int a = (int)(u / pl.tiles), jt = (int)(u - (long long)a * pl.tiles);
     const int e = P.act_e[a], off = P.act_off[a], cnt = P.act_cnt[a];
     const size_t row = (size_t)e * P.H + jt * 8 + g;
+    const int slot = i % D;
     uint4 raw = {0, 0, 0, 0}, fac = {0, 0, 0, 0};
-    const int b_first = wi * 32 + 8 * c;
-    if (!DENSE && spw_one && b_first < nb) raw = load_idx_raw<IdxT>(idx_d + row * nb + b_first);
-    if (has_lr && lr_group * 32 + 8 * c < P.r)
-      fac = __ldg(reinterpret_cast<const uint4*>(P.down.factor + row * P.r + lr_group * 32 + 8 * c));
+    if (!DENSE && ringed && idx_live) raw = ring_idx8<IdxT>(ring + slot * 32 + lane);
+    if (fac_live) fac = fring[slot * 32 + lane];
     for (int pass = 0; pass * 8 < cnt; ++pass) {
       const int n_tok = min(8, cnt - pass * 8);
       const int pos = g < n_tok ? off + pass * 8 + g : -1;
-      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
       for (int sl = wi; sl < pl.n_slices; sl += pl.team_warps) {
         const int b0 = sl * 32 + (DENSE ? c : 8 * c);
         if (frag_a != a || frag_pass != pass || frag_slice != sl) {
@@ -542,23 +685,23 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
         }
         if (DENSE) {
           const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I);
-          uint4 v[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const int b = b0 + 4 * j;
-            v[j] = b < nb ? __ldg(wd + b) : make_uint4(0, 0, 0, 0);
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (b < nb) v = ringed ? ring[(slot * 8 + j) * 32 + lane] : __ldg(wd + b);
+            mma_block(acc[0], fh[j], v);
+            mma_block(acc[1], fl[j], v);
           }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) { mma_block(acc, fh[j], v[j]); mma_block(acc, fl[j], v[j]); }
         } else {
-          if (!spw_one) raw = b0 < nb ? load_idx_raw<IdxT>(idx_d + row * nb + b0) : make_uint4(0, 0, 0, 0);
+          if (!ringed) raw = b0 < nb ? load_idx_raw<IdxT>(idx_d + row * nb + b0) : make_uint4(0, 0, 0, 0);
           uint32_t id[8];                      // out-of-range groups: index 0, zero fragments
           unpack_idx8<IdxT>(raw, id);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const uint4 w = s_cb[id[j]];
-            mma_block(acc, fh[j], w);
-            mma_block(acc, fl[j], w);
+            mma_block(acc[0], fh[j], w);
+            mma_block(acc[1], fl[j], w);
           }
         }
       }
@@ -576,28 +719,33 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
           }
           z_a = a; z_pass = pass; z_lg = lg;
         }
-        mma_block(acc, zh, f);
-        mma_block(acc, zl, f);
+        mma_block(acc[0], zh, f);
+        mma_block(acc[1], zl, f);
       }
       float2* part = s_part + (size_t)(buf * pl.n_teams + team) * pl.team_warps * 32;
-      part[wi * 32 + lane] = make_float2(acc[0], acc[1]);
+      long long* yrow = s_yrow + (size_t)(buf * pl.n_teams + team) * 8;
+      part[wi * 32 + lane] = make_float2(acc[0][0] + acc[1][0], acc[0][1] + acc[1][1]);
+      if (tid_team < n_tok) {                    // output rows of this pass's tokens
+        const int ps = off + pass * 8 + tid_team;
+        yrow[tid_team] = ((long long)P.pair_token[ps] * n_slots + P.pair_slot[ps]) * P.H;
+      }
       if (pl.team_warps > 1) team_sync(1 + team, team_threads); else __syncwarp();
       for (int q = tid_team; q < 64; q += team_threads) {
         const int m = q >> 3, n = q & 7;
         if (m < n_tok) {
           const int src = 4 * m + (n >> 1);
-          float s = 0.f;
+          float sum = 0.f;
           for (int w = 0; w < pl.team_warps; ++w) {
             const float2 v = part[w * 32 + src];
-            s += (n & 1) ? v.y : v.x;
+            sum += (n & 1) ? v.y : v.x;
           }
-          const int ps = off + pass * 8 + m;
-          P.y[((size_t)P.pair_token[ps] * n_slots + P.pair_slot[ps]) * P.H + jt * 8 + n] = s;
+          P.y[yrow[m] + jt * 8 + n] = sum;
         }
       }
       buf ^= 1;
     }
   }
+  cp_async_wait_pending(0);
 }
 
 // z_d[pos][rho] = <basis_down[rho], p[pos]> (link of the chain between gate/up and down).

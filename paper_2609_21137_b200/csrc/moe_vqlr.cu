@@ -46,6 +46,9 @@ struct moe_vqlr_handle {
   size_t workspace_bytes;
   bf16* x_stage;     // [maxT][H] device staging for the host-buffer entry point
   bf16* out_stage;   // [maxT][H]
+  cudaStream_t cap_stream;                 // only ever used to capture the graphs below
+  cudaGraphExec_t host_graph[kMaxT + 1];   // kernel chain x_stage -> out_stage for T tokens
+  int host_graph_launches;                 // kernels in one such graph
   int64_t launches;
   int profiling;             // record an event after every stage of a call
   cudaEvent_t ev[kStages + 1];
@@ -75,12 +78,12 @@ StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense, int warps) {
   StagePlan pl;
   pl.nb = in_dim / kD;
   pl.n_slices = (pl.nb + 31) / 32;
-  const int max_team = warps >= 16 ? 16 : 4;
-  pl.team_warps = next_pow2(pl.n_slices) < max_team ? next_pow2(pl.n_slices) : max_team;
+  pl.team_warps = pl.n_slices < warps ? pl.n_slices : warps;   // one warp per slice when they fit
   pl.n_teams = warps / pl.team_warps;
   if (pl.n_teams > 15 && pl.team_warps > 1) pl.n_teams = 15;   // named barriers 1..15
   pl.tiles = out_dim / 8;
   pl.n_lr = (!dense && r > 0) ? (r + 31) / 32 : 0;
+  pl.depth = 2;
   return pl;
 }
 
@@ -140,6 +143,86 @@ T* carve(char*& cur, size_t n) {
   return p;
 }
 
+// Enqueues the kernel of one stage (nothing for a stage this configuration does not have).
+cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, bf16* ob, cudaStream_t st) {
+  const Params& P = h->P;
+  cudaError_t le = cudaSuccess;
+  bool ran = false;
+  const int n_pos = T * (P.k + P.S);
+  if (h->fast) {
+    switch (stage) {
+      case 0:
+        le = launch_pdl(k_router_z_pdl, ((P.E + P.n_zrows) * ((T + kTokGroup - 1) / kTokGroup) + kRouterWarps - 1) / kRouterWarps,
+                        32 * kRouterWarps, 0, st, P, xb, T);
+        ran = true;
+        break;
+      case 2: {
+        const size_t smem = gu_layout(P.K, h->n_books, T, P.H, P.r, h->plan_gu, (h->gu_dense ? kDenseThreads : kFastThreads) / 32, P.E, P.k, P.S).total;
+        if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, h->plan_gu, h->n_books);
+        else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, h->plan_gu, h->n_books);
+        else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, h->plan_gu, h->n_books);
+        ran = true;
+        break;
+      }
+      case 3:
+        if (!h->dn_dense && P.r > 0) {
+          le = launch_pdl(k_zdown_pdl, (n_pos * P.r + 7) / 8, 256, 0, st, P, n_pos);
+          ran = true;
+        }
+        break;
+      case 4:
+        if (h->dn_dense) le = launch_pdl(k_down_mma<uint16_t, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, h->plan_dn);
+        else if (h->idx_bytes == 1) le = launch_pdl(k_down_mma<uint8_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, h->plan_dn);
+        else le = launch_pdl(k_down_mma<uint16_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, h->plan_dn);
+        ran = true;
+        break;
+      case 5: {
+        int grid = (T * P.H / 2 + 255) / 256;
+        if (grid > h->sm_count) grid = h->sm_count;
+        le = launch_pdl(k_combine, grid, 256, 0, st, P, ob, T);
+        ran = true;
+        break;
+      }
+      default: break;
+    }
+  } else {
+    switch (stage) {
+      case 0:
+        k_router_z<<<(P.E + P.n_zrows + 7) / 8, 256, 0, st>>>(P, xb, T);
+        ran = true;
+        break;
+      case 1:
+        k_route<<<1, 32 * T, (size_t)T * P.E * 4 + (2 * (size_t)P.E + 1) * 4, st>>>(P, T);
+        ran = true;
+        break;
+      case 2: {
+        const size_t smem = h->smem_gateup_fixed + h->smem_gateup_per_token * T;
+        if (h->idx_bytes == 1) k_gateup<uint8_t><<<h->sm_count, 512, smem, st>>>(P, xb, T, h->two_books);
+        else k_gateup<uint16_t><<<h->sm_count, 512, smem, st>>>(P, xb, T, h->two_books);
+        ran = true;
+        break;
+      }
+      case 3:
+        if (P.down.kind == MOE_VQLR_PROJ_VQLR && P.r > 0) {
+          k_zdown<<<(n_pos * P.r + 7) / 8, 256, 0, st>>>(P, n_pos);
+          ran = true;
+        }
+        break;
+      case 4: {
+        const int grid = min(h->sm_count, (P.H + 15) / 16);
+        if (h->idx_bytes == 1) k_down<uint8_t><<<grid, 512, h->smem_down, st>>>(P, ob, T);
+        else k_down<uint16_t><<<grid, 512, h->smem_down, st>>>(P, ob, T);
+        ran = true;
+        break;
+      }
+      default: break;
+    }
+    if (ran) le = cudaGetLastError();
+  }
+  if (ran) { h->launches += 1; h->stage_ran[stage] = true; }
+  return le;
+}
+
 }  // namespace
 
 extern "C" {
@@ -172,6 +255,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   h->launches = 0;
   h->workspace = nullptr;
   h->profiling = 0;
+  h->cap_stream = nullptr;
+  for (auto& g : h->host_graph) g = nullptr;
   h->ev_valid = false;
   for (auto& e : h->ev) e = nullptr;
   h->idx_bytes = K <= 256 ? 1 : 2;
@@ -240,10 +325,21 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     if (gu_vq && r > 0 && (P.gate.zslot < 0 || P.up.zslot < 0)) ok = false;
     h->n_books = gu_vq ? (h->two_books ? 2 : 1) : 0;
     h->plan_gu = plan_stage(I, H, r, gu_dn, (gu_dn ? kDenseThreads : kFastThreads) / 32);
-    h->plan_dn = plan_stage(H, I, r, h->dn_dense, (h->dn_dense ? kDenseThreads : kFastThreads) / 32);
-    const size_t smem_gu = gu_smem_bytes(K, h->n_books, maxT, H, h->plan_gu, E, k, S);
-    h->smem_fast_dn = dn_smem_bytes(K, !h->dn_dense, h->plan_dn);
-    if (smem_gu > (size_t)prop.sharedMemPerBlockOptin || h->smem_fast_dn > (size_t)prop.sharedMemPerBlockOptin) ok = false;
+    h->plan_dn = plan_stage(H, I, r, h->dn_dense, kDownThreads / 32);
+    // deepest rings that still fit the shared memory of one block
+    const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
+    const int gu_warps = (gu_dn ? kDenseThreads : kFastThreads) / 32;
+    for (int d = kMaxDepth; d >= 2; --d) {
+      h->plan_gu.depth = d;
+      if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total <= limit) break;
+    }
+    for (int d = kMaxDepth; d >= 2; --d) {
+      h->plan_dn.depth = d;
+      if (dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32).total <= limit) break;
+    }
+    const size_t smem_gu = gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total;
+    h->smem_fast_dn = dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32).total;
+    if (smem_gu > limit || h->smem_fast_dn > limit) ok = false;
     const char* force = getenv("MOE_VQLR_FORCE_GENERIC");
     if (force && force[0] == '1') ok = false;
     h->fast = ok;
@@ -339,92 +435,13 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
   bf16* ob = static_cast<bf16*>(out);
 
   const bool prof = h->profiling != 0;
-  auto mark = [&](int i) { if (prof) cudaEventRecord(h->ev[i], st); };
   for (int i = 0; i < kStages; ++i) h->stage_ran[i] = false;
-  if (h->fast) {
-    cudaError_t le = cudaSuccess;
-    auto keep = [&](cudaError_t e) { if (le == cudaSuccess) le = e; };
-    mark(0);
-    {
-      const int rows = P.E + P.n_zrows;
-      keep(launch_pdl(k_router_z_pdl, (rows + 7) / 8, 256, 0, st, P, xb, (int)T));
-      h->stage_ran[0] = true;
-    }
-    mark(1);
-    mark(2);
-    {
-      const size_t smem = gu_smem_bytes(P.K, h->n_books, T, P.H, h->plan_gu, P.E, P.k, P.S);
-      if (h->gu_dense) keep(launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, (int)T, h->plan_gu, h->n_books));
-      else if (h->idx_bytes == 1) keep(launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, (int)T, h->plan_gu, h->n_books));
-      else keep(launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, (int)T, h->plan_gu, h->n_books));
-      h->stage_ran[2] = true;
-    }
-    mark(3);
-    h->launches += 2;
-    if (!h->dn_dense && P.r > 0) {
-      const int n_pos = T * (P.k + P.S);
-      keep(launch_pdl(k_zdown_pdl, (n_pos * P.r + 7) / 8, 256, 0, st, P, n_pos));
-      h->launches += 1;
-      h->stage_ran[3] = true;
-    }
-    mark(4);
-    {
-      if (h->dn_dense) keep(launch_pdl(k_down_mma<uint16_t, true>, h->sm_count, kDenseThreads, h->smem_fast_dn, st, P, (int)T, h->plan_dn));
-      else if (h->idx_bytes == 1) keep(launch_pdl(k_down_mma<uint8_t, false>, h->sm_count, kFastThreads, h->smem_fast_dn, st, P, (int)T, h->plan_dn));
-      else keep(launch_pdl(k_down_mma<uint16_t, false>, h->sm_count, kFastThreads, h->smem_fast_dn, st, P, (int)T, h->plan_dn));
-      h->stage_ran[4] = true;
-    }
-    mark(5);
-    {
-      const int work = T * P.H / 2;
-      int grid = (work + 255) / 256;
-      if (grid > h->sm_count) grid = h->sm_count;
-      keep(launch_pdl(k_combine, grid, 256, 0, st, P, ob, (int)T));
-      h->stage_ran[5] = true;
-    }
-    mark(6);
-    h->launches += 2;
-    if (le != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "launch: %s", cudaGetErrorString(le));
-  } else {
-  mark(0);
-  {
-    const int rows = P.E + P.n_zrows;
-    k_router_z<<<(rows + 7) / 8, 256, 0, st>>>(P, xb, T);
-    h->stage_ran[0] = true;
+  for (int stage = 0; stage < kStages; ++stage) {
+    if (prof) cudaEventRecord(h->ev[stage], st);
+    const cudaError_t le = launch_stage(h, stage, xb, T, ob, st);
+    if (le != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "launch of stage %s: %s", kStageNames[stage], cudaGetErrorString(le));
   }
-  mark(1);
-  {
-    const size_t smem = (size_t)T * P.E * 4 + (2 * (size_t)P.E + 1) * 4;
-    k_route<<<1, 32 * T, smem, st>>>(P, T);
-    h->stage_ran[1] = true;
-  }
-  mark(2);
-  {
-    const size_t smem = h->smem_gateup_fixed + h->smem_gateup_per_token * T;
-    const int grid = h->sm_count;
-    if (h->idx_bytes == 1) k_gateup<uint8_t><<<grid, 512, smem, st>>>(P, xb, T, h->two_books);
-    else k_gateup<uint16_t><<<grid, 512, smem, st>>>(P, xb, T, h->two_books);
-    h->stage_ran[2] = true;
-  }
-  mark(3);
-  h->launches += 3;
-  if (P.down.kind == MOE_VQLR_PROJ_VQLR && P.r > 0) {
-    const int n_pos = T * (P.k + P.S);
-    k_zdown<<<(n_pos * P.r + 7) / 8, 256, 0, st>>>(P, n_pos);
-    h->launches += 1;
-    h->stage_ran[3] = true;
-  }
-  mark(4);
-  {
-    const int grid = min(h->sm_count, (P.H + 15) / 16);
-    if (h->idx_bytes == 1) k_down<uint8_t><<<grid, 512, h->smem_down, st>>>(P, ob, T);
-    else k_down<uint16_t><<<grid, 512, h->smem_down, st>>>(P, ob, T);
-    h->launches += 1;
-    h->stage_ran[4] = true;
-  }
-  mark(5);
-  mark(6);
-  }
+  if (prof) cudaEventRecord(h->ev[kStages], st);
   h->ev_valid = prof;
   cudaError_t ce = cudaGetLastError();
   if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "launch: %s", cudaGetErrorString(ce));
@@ -452,10 +469,39 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
   if (T < 1 || T > h->cfg.max_tokens) return fail(h, MOE_VQLR_ERR_INVALID_ARG, "T=%d outside 1..%d", T, h->cfg.max_tokens);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t bytes = (size_t)T * h->P.H * sizeof(bf16);
+  // The kernel chain between the two staging buffers never changes for a given T, so it is
+  // captured once into a graph and replayed: one launch instead of five.
+  if (!h->host_graph[T] && !h->profiling) {
+    cudaError_t ge = cudaSuccess;
+    if (!h->cap_stream) ge = cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking);
+    cudaGraph_t graph = nullptr;
+    if (ge == cudaSuccess) ge = cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal);
+    if (ge == cudaSuccess) {
+      const int64_t before = h->launches;
+      const int rc = moe_vqlr_decode_layer(h, h->x_stage, T, h->out_stage, nullptr, h->cap_stream);
+      h->host_graph_launches = (int)(h->launches - before);
+      h->launches = before;
+      ge = cudaStreamEndCapture(h->cap_stream, &graph);
+      if (rc != MOE_VQLR_OK && ge == cudaSuccess) ge = cudaErrorUnknown;
+    }
+    if (ge == cudaSuccess) ge = cudaGraphInstantiate(&h->host_graph[T], graph, 0);
+    if (graph) cudaGraphDestroy(graph);
+    if (ge != cudaSuccess) {
+      cudaGetLastError();
+      h->host_graph[T] = nullptr;
+      return fail(h, MOE_VQLR_ERR_CUDA, "graph capture of the layer: %s", cudaGetErrorString(ge));
+    }
+  }
   cudaError_t ce = cudaMemcpyAsync(h->x_stage, x_host, bytes, cudaMemcpyHostToDevice, st);
   if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "copy in: %s", cudaGetErrorString(ce));
-  const int rc = moe_vqlr_decode_layer(h, h->x_stage, T, h->out_stage, nullptr, cuda_stream);
-  if (rc != MOE_VQLR_OK) return rc;
+  if (h->host_graph[T] && !h->profiling) {
+    ce = cudaGraphLaunch(h->host_graph[T], st);
+    if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "graph launch: %s", cudaGetErrorString(ce));
+    h->launches += h->host_graph_launches;
+  } else {
+    const int rc = moe_vqlr_decode_layer(h, h->x_stage, T, h->out_stage, nullptr, cuda_stream);
+    if (rc != MOE_VQLR_OK) return rc;
+  }
   ce = cudaMemcpyAsync(out_host, h->out_stage, bytes, cudaMemcpyDeviceToHost, st);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
   if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "copy out: %s", cudaGetErrorString(ce));
@@ -466,6 +512,9 @@ int moe_vqlr_destroy(moe_vqlr_handle* h) {
   if (!h) return MOE_VQLR_OK;
   for (auto& e : h->ev)
     if (e) cudaEventDestroy(e);
+  for (auto& g : h->host_graph)
+    if (g) cudaGraphExecDestroy(g);
+  if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
   cudaError_t ce = cudaFree(h->workspace);
   delete h;
   return ce == cudaSuccess ? MOE_VQLR_OK : MOE_VQLR_ERR_CUDA;
@@ -473,6 +522,16 @@ int moe_vqlr_destroy(moe_vqlr_handle* h) {
 
 const char* moe_vqlr_last_error(const moe_vqlr_handle* h) {
   return h ? h->error.c_str() : g_create_error.c_str();
+}
+
+int moe_vqlr_run_stage(moe_vqlr_handle* h, int32_t stage, const void* x, int32_t T, void* out, void* cuda_stream) {
+  if (!h) return MOE_VQLR_ERR_INVALID_ARG;
+  if (stage < 0 || stage >= kStages || !x || !out || T < 1 || T > h->cfg.max_tokens)
+    return fail(h, MOE_VQLR_ERR_INVALID_ARG, "run_stage: bad stage, pointer or T");
+  const cudaError_t le = launch_stage(h, stage, static_cast<const bf16*>(x), T, static_cast<bf16*>(out),
+                                      static_cast<cudaStream_t>(cuda_stream));
+  if (le != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "launch of stage %s: %s", kStageNames[stage], cudaGetErrorString(le));
+  return MOE_VQLR_OK;
 }
 
 int moe_vqlr_set_profiling(moe_vqlr_handle* h, int32_t on) {
