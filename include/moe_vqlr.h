@@ -159,6 +159,13 @@ const char* moe_vqlr_stage_name(int32_t i);
 int moe_vqlr_run_stage(moe_vqlr_handle* h, int32_t stage, const void* x, int32_t T, void* out,
                        void* cuda_stream);
 
+/* Tracing aid (no counterpart in the paper).  When the environment variable
+ * MOE_VQLR_PHASE_CLOCKS=1 is set at create(), the tensor-core gate/up kernel stores SM clock
+ * readings at its phase boundaries: [kernel 4][block][warp 16][stamp 16] int64.  With out == NULL
+ * returns the number of values; otherwise synchronously copies them to the HOST buffer out
+ * (cap = its capacity in values) and returns the count, -1 on error, 0 when tracing is off. */
+int64_t moe_vqlr_phase_clocks(moe_vqlr_handle* h, int64_t* out, int64_t cap);
+
 /* Number of kernel launches this handle has enqueued since create(). */
 int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h);
 

@@ -23,7 +23,7 @@ EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_ho
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",
            "moe_vqlr_workspace_bytes", "moe_vqlr_set_profiling", "moe_vqlr_last_stage_times",
            "moe_vqlr_stage_count", "moe_vqlr_stage_name", "moe_vqlr_route_noalloc",
-           "moe_vqlr_run_stage"]
+           "moe_vqlr_run_stage", "moe_vqlr_phase_clocks"]
 
 
 class MoeVqlrError(RuntimeError):
@@ -85,6 +85,8 @@ def _load():
     lib.moe_vqlr_stage_name.argtypes = [C.c_int32]
     lib.moe_vqlr_run_stage.restype = C.c_int
     lib.moe_vqlr_run_stage.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    lib.moe_vqlr_phase_clocks.restype = C.c_int64
+    lib.moe_vqlr_phase_clocks.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
     lib.moe_vqlr_route_noalloc.restype = C.c_int
     lib.moe_vqlr_route_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 5 + \
                                           [C.c_void_p, C.c_void_p, C.c_void_p]
@@ -232,6 +234,16 @@ class MoeVqlrLayer:
         st = stream or torch.cuda.current_stream(x.device)
         self._check(_lib.moe_vqlr_run_stage(self._h, names.index(stage), _ptr(x), x.shape[0], _ptr(out),
                                             C.c_void_p(st.cuda_stream)))
+
+    def phase_clocks(self):
+        """Phase stamps of the last call as an int64 array [4][blocks][16][16], or None when the
+        handle was not created with MOE_VQLR_PHASE_CLOCKS=1."""
+        n = int(_lib.moe_vqlr_phase_clocks(self._h, None, 0))
+        if n <= 0:
+            return None
+        buf = np.zeros(n, np.int64)
+        got = int(_lib.moe_vqlr_phase_clocks(self._h, buf.ctypes.data_as(C.c_void_p), n))
+        return buf.reshape(4, -1, 16, 16) if got == n else None
 
     def set_profiling(self, on: bool) -> None:
         self._check(_lib.moe_vqlr_set_profiling(self._h, 1 if on else 0))

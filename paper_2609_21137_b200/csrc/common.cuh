@@ -48,11 +48,27 @@ struct Params {
   int* act_e;              // [E+S] expert id
   int* act_off;            // [E+S] first pair position
   int* act_cnt;            // [E+S] pairs
+  int* grp_n;              // [1] work groups of the tensor-core chain: (expert, first pair, <= 8 pairs)
+  int* grp_e;              // [maxT*(k+S)]
+  int* grp_off;            // [maxT*(k+S)]
+  int* grp_cnt;            // [maxT*(k+S)]
   float* p;                // [maxT*(k+S)][I]   SwiGLU intermediate per pair position
+  bf16* p_hi;              // [maxT*(k+S)][I]   p rounded to bf16 ...
+  bf16* p_lo;              // [maxT*(k+S)][I]   ... and the bf16 remainder (p = hi + lo to 2^-17)
   float* zd;               // [maxT*(k+S)][r]   basis_down * p per pair position
-  float* y;                // [maxT][k+S][H]    expert outputs before the weighted sum
+  float* y;                // [maxT*(k+S)][H]   expert outputs before the weighted sum, by pair position
+  int* inv_pos;            // [maxT][k+S]       pair position of (token, slot)
   int* status;             // [1]
+  long long* clk;          // optional phase stamps [kernel 4][block][warp 16][stamp 16], or NULL
+  int clk_blocks;
 };
+
+// Optional tracing: lane 0 of a warp stores clock64() at phase `k` of kernel `kern`.
+__device__ __forceinline__ void stamp(const long long* base_c, int clk_blocks, int kern, int k) {
+  long long* base = const_cast<long long*>(base_c);
+  if (base && (threadIdx.x & 31) == 0 && k < 16 && (int)blockIdx.x < clk_blocks && (threadIdx.x >> 5) < 16)
+    base[(((size_t)kern * clk_blocks + blockIdx.x) * 16 + (threadIdx.x >> 5)) * 16 + k] = clock64();
+}
 
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }

@@ -38,6 +38,7 @@ struct moe_vqlr_handle {
   int two_books;
   size_t smem_gateup_per_token, smem_gateup_fixed, smem_down;
   bool fast;                 // tensor-core chain eligible for this configuration
+  int want_dbg;              // the running call asked for counts / offsets
   bool gu_dense, dn_dense;
   int n_books;               // distinct gate/up code books staged by k_gateup_mma
   StagePlan plan_gu, plan_dn;
@@ -71,7 +72,6 @@ int fail(moe_vqlr_handle* h, int code, const char* fmt, ...) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int next_pow2(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
 // Cuts one projection stage into slices and teams for `warps` warps per block.
 StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense, int warps) {
@@ -84,6 +84,7 @@ StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense, int warps) {
   pl.tiles = out_dim / 8;
   pl.n_lr = (!dense && r > 0) ? (r + 31) / 32 : 0;
   pl.depth = 2;
+  pl.batch = 1;
   return pl;
 }
 
@@ -158,9 +159,9 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         break;
       case 2: {
         const size_t smem = gu_layout(P.K, h->n_books, T, P.H, P.r, h->plan_gu, (h->gu_dense ? kDenseThreads : kFastThreads) / 32, P.E, P.k, P.S).total;
-        if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, h->plan_gu, h->n_books);
-        else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, h->plan_gu, h->n_books);
-        else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, h->plan_gu, h->n_books);
+        if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, h->plan_gu, h->n_books, h->want_dbg);
+        else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, h->plan_gu, h->n_books, h->want_dbg);
+        else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, h->plan_gu, h->n_books, h->want_dbg);
         ran = true;
         break;
       }
@@ -253,6 +254,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   if (!h) return fail(nullptr, MOE_VQLR_ERR_OOM, "host allocation failed");
   h->cfg = *cfg;
   h->launches = 0;
+  h->want_dbg = 0;
   h->workspace = nullptr;
   h->profiling = 0;
   h->cap_stream = nullptr;
@@ -329,16 +331,25 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     // deepest rings that still fit the shared memory of one block
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
     const int gu_warps = (gu_dn ? kDenseThreads : kFastThreads) / 32;
-    for (int d = kMaxDepth; d >= 2; --d) {
-      h->plan_gu.depth = d;
-      if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total <= limit) break;
-    }
-    for (int d = kMaxDepth; d >= 2; --d) {
-      h->plan_dn.depth = d;
-      if (dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32).total <= limit) break;
+    // deepest rings and largest tile batches that fit: batch first (it removes barriers), then depth
+    {
+      bool found = false;
+      for (int bt = 4; bt >= 1 && !found; --bt)
+        for (int d = kMaxDepth; d >= 2 && !found; --d) {
+          h->plan_gu.batch = bt;
+          h->plan_gu.depth = d;
+          found = gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total <= limit;
+        }
+      found = false;
+      for (int bt = 4; bt >= 1 && !found; --bt)
+        for (int d = kMaxDepth; d >= 2 && !found; --d) {
+          h->plan_dn.batch = bt;
+          h->plan_dn.depth = d;
+          found = dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total <= limit;
+        }
     }
     const size_t smem_gu = gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total;
-    h->smem_fast_dn = dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32).total;
+    h->smem_fast_dn = dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total;
     if (smem_gu > limit || h->smem_fast_dn > limit) ok = false;
     const char* force = getenv("MOE_VQLR_FORCE_GENERIC");
     if (force && force[0] == '1') ok = false;
@@ -357,6 +368,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   }
 
   // workspace
+  const char* clk_env = getenv("MOE_VQLR_PHASE_CLOCKS");
+  const bool want_clk = clk_env && clk_env[0] == '1';
   const size_t n_pos = (size_t)maxT * (k + S);
   auto plan = [&](char* base) {
     char* cur = base;
@@ -373,10 +386,18 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     P.act_e = carve<int>(cur, E + S);
     P.act_off = carve<int>(cur, E + S);
     P.act_cnt = carve<int>(cur, E + S);
+    P.grp_n = carve<int>(cur, 1);
+    P.grp_e = carve<int>(cur, n_pos);
+    P.grp_off = carve<int>(cur, n_pos);
+    P.grp_cnt = carve<int>(cur, n_pos);
     P.p = carve<float>(cur, n_pos * I);
+    P.p_hi = carve<bf16>(cur, n_pos * I);
+    P.p_lo = carve<bf16>(cur, n_pos * I);
     P.zd = carve<float>(cur, n_pos * (r > 0 ? r : 1));
     P.y = carve<float>(cur, n_pos * H);
+    P.inv_pos = carve<int>(cur, n_pos);
     P.status = carve<int>(cur, 1);
+    if (want_clk) { P.clk = carve<long long>(cur, (size_t)4 * h->sm_count * 16 * 16); P.clk_blocks = h->sm_count; }
     h->x_stage = carve<bf16>(cur, (size_t)maxT * H);
     h->out_stage = carve<bf16>(cur, (size_t)maxT * H);
     return (size_t)(cur - base);
@@ -435,6 +456,7 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
   bf16* ob = static_cast<bf16*>(out);
 
   const bool prof = h->profiling != 0;
+  h->want_dbg = (dbg && (dbg->counts || dbg->offsets)) ? 1 : 0;
   for (int i = 0; i < kStages; ++i) h->stage_ran[i] = false;
   for (int stage = 0; stage < kStages; ++stage) {
     if (prof) cudaEventRecord(h->ev[stage], st);
@@ -564,6 +586,15 @@ int moe_vqlr_last_stage_times(moe_vqlr_handle* h, float* ms_out, int32_t cap) {
     }
   }
   return MOE_VQLR_OK;
+}
+
+int64_t moe_vqlr_phase_clocks(moe_vqlr_handle* h, int64_t* out, int64_t cap) {
+  if (!h || !h->P.clk) return 0;
+  const int64_t n = (int64_t)4 * h->P.clk_blocks * 16 * 16;
+  if (!out) return n;
+  if (cap < n) return -1;
+  if (cudaMemcpy(out, h->P.clk, (size_t)n * 8, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  return n;
 }
 
 int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h) { return h ? h->launches : 0; }
