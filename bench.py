@@ -54,6 +54,17 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def max_over_ranks(value: float, world: int, device="cuda") -> float:
+    """Maximum of a per-rank scalar over all ranks (replicas report the slowest rank's time)."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -346,10 +357,7 @@ def main():
         while time.time() < t_end:
             wl.g_full.replay()
             torch.cuda.synchronize(device)
-    if world > 1:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, device)
     shp = wl.shp
     ms_per_step = ms / args.steps
     us_per_layer_token = ms_per_step * 1e3 / (shp.T * world)
@@ -375,10 +383,7 @@ def main():
     # ---- end to end through host buffers --------------------------------------------------
     e2e_steps = min(args.steps, 400)
     e2e_ms, h2d, d2h = wl.run_e2e(e2e_steps, max(3, min(args.warmup, 20)))
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, device)
     e2e = {"value": e2e_ms * 1e3 / e2e_steps / (shp.T * world), "unit": "us", "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps}
     n_layers = len(wl.layers)

@@ -1,0 +1,110 @@
+"""Larger and odder shapes: Mixtral-shaped layers at full size (outputs sampled, the oracle
+computes only the sampled down rows), a shape with more slices than warps, error codes."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_21137_b200 import synth
+
+from helpers import (assert_output, assert_routing, bf16_tensor_to_f64, logit_gaps, MIN_LOGIT_GAP)
+
+pytestmark = pytest.mark.gpu
+
+
+def _sampled_check(shp, rows, seed=0):
+    from paper_2609_21137_b200 import binding
+    for s in range(seed, seed + 10):
+        layer = synth.make_layer(shp, seed=s)
+        res = oracle.OracleLayer.from_synth(layer).decode_layer(layer.x, down_rows=rows)
+        if logit_gaps(res, shp.k) > MIN_LOGIT_GAP or shp.k == shp.E:
+            break
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    x = binding.bits_to_device(layer.x, "cuda")
+    out, dbg = mod.decode(x, debug=True)
+    torch.cuda.synchronize()
+    assert_routing(dbg, res)
+    got = bf16_tensor_to_f64(out)[:, rows]
+    m = assert_output(got, res.out, what=shp.name)
+    mod.close()
+    del layer
+    return m
+
+
+@pytest.mark.parametrize("mode", ["full", "paper"])
+def test_mixtral_full_size_b1_sampled_rows(mode):
+    shp = synth.shape("mixtral", mode=mode)
+    rows = sorted(set(np.random.default_rng(1).integers(0, shp.H, 96).tolist()) | {0, shp.H - 1})
+    _sampled_check(shp, rows)
+
+
+def test_more_slices_than_warps_b16():
+    # I = 3584 -> 14 slices of the down contraction for 12 warps; every expert active at T = 16
+    shp = synth.shape("mixtral_b16", I=3584)
+    rows = sorted(set(np.random.default_rng(2).integers(0, shp.H, 64).tolist()) | {0, shp.H - 1})
+    _sampled_check(shp, rows)
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    from paper_2609_21137_b200 import binding
+    shp = synth.shape("qwen3_b16", E=32)
+    layer = synth.make_layer(shp, seed=0)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    x = binding.bits_to_device(layer.x, "cuda")
+    ref = mod.decode(x)
+    torch.cuda.synchronize()
+    xh = x.cpu().pin_memory()
+    oh = torch.zeros((shp.T, shp.H), dtype=torch.int16).pin_memory()
+    for _ in range(2):                     # the second call replays the captured graph
+        oh.zero_()
+        mod.decode_host(xh, oh)
+        assert torch.equal(oh, ref.view(torch.int16).cpu())
+    # fewer tokens than max_tokens through the same handle
+    mod.decode_host(xh[:3].contiguous().pin_memory(), oh[:3])
+    ref3 = mod.decode(x[:3].contiguous())
+    torch.cuda.synchronize()
+    assert torch.equal(oh[:3], ref3.view(torch.int16).cpu())
+    mod.close()
+
+
+def test_error_codes():
+    from paper_2609_21137_b200 import binding
+    layer = synth.make_layer(synth.shape("tiny", T=4), seed=0)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", max_tokens=4)
+    x = binding.bits_to_device(layer.x, "cuda")
+    lib = binding.library()
+    out = torch.empty((8, 256), dtype=torch.bfloat16, device="cuda")
+    big = torch.zeros((8, 256), dtype=torch.bfloat16, device="cuda")
+    st = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert lib.moe_vqlr_decode_layer(mod._h, big.data_ptr(), 5, out.data_ptr(), None, st) == binding.ERR_INVALID_ARG
+    assert b"T=5" in lib.moe_vqlr_last_error(mod._h)
+    assert lib.moe_vqlr_decode_layer(mod._h, big.data_ptr(), 0, out.data_ptr(), None, st) == binding.ERR_INVALID_ARG
+    assert lib.moe_vqlr_decode_layer(mod._h, None, 1, out.data_ptr(), None, st) == binding.ERR_INVALID_ARG
+    assert lib.moe_vqlr_decode_layer(mod._h, big.data_ptr() + 2, 1, out.data_ptr(), None, st) == binding.ERR_INVALID_ARG
+    assert b"aligned" in lib.moe_vqlr_last_error(mod._h)
+    mod.decode(x)                          # the handle still works after rejected calls
+    torch.cuda.synchronize()
+    mod.close()
+    # unsupported shapes and options
+    for kw, code in ((dict(d=4), binding.ERR_UNSUPPORTED), (dict(max_tokens=17), binding.ERR_UNSUPPORTED),
+                     (dict(k=9), binding.ERR_INVALID_ARG), (dict(H=260), binding.ERR_UNSUPPORTED)):
+        with pytest.raises(binding.MoeVqlrError) as err:
+            args = dict(H=256, I=128, E=8, k=2, S=0, d=8, K=256, r=16, max_tokens=4)
+            args.update(kw)
+            up = lambda a: binding.bits_to_device(a, "cuda")   # noqa: E731
+            proj = lambda p: dict(codebook=up(p.codebook), idx=up(p.idx), basis=up(p.basis), factor=up(p.factor))  # noqa: E731
+            binding.MoeVqlrLayer(router_w=up(layer.router_w), gate=proj(layer.gate), up=proj(layer.up),
+                                 down=proj(layer.down), **args)
+        assert err.value.status == code, kw
+
+
+def test_index_validation_flag_finds_bad_index():
+    from paper_2609_21137_b200 import binding
+    layer = synth.make_layer(synth.shape("tiny", K=200), seed=0)
+    binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_VALIDATE_INDICES).close()
+    layer.up.idx[3, 7, 5] = 200
+    with pytest.raises(binding.MoeVqlrError) as err:
+        binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_VALIDATE_INDICES)
+    assert err.value.status == binding.ERR_BAD_INDEX
