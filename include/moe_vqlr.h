@@ -160,8 +160,8 @@ int moe_vqlr_run_stage(moe_vqlr_handle* h, int32_t stage, const void* x, int32_t
                        void* cuda_stream);
 
 /* Tracing aid (no counterpart in the paper).  When the environment variable
- * MOE_VQLR_PHASE_CLOCKS=1 is set at create(), the tensor-core gate/up kernel stores SM clock
- * readings at its phase boundaries: [kernel 4][block][warp 16][stamp 16] int64.  With out == NULL
+ * MOE_VQLR_PHASE_CLOCKS=1 is set at create() and the library was built with -DMOE_VQLR_TRACE,
+ * the tensor-core kernels store SM clock readings at their phase boundaries: [kernel 4][block][warp 16][stamp 16] int64.  With out == NULL
  * returns the number of values; otherwise synchronously copies them to the HOST buffer out
  * (cap = its capacity in values) and returns the count, -1 on error, 0 when tracing is off. */
 int64_t moe_vqlr_phase_clocks(moe_vqlr_handle* h, int64_t* out, int64_t cap);

@@ -31,7 +31,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
-        cmd = [nvcc] + flags + (["-Xptxas", "-v"] if verbose else []) + \
+        extra = os.environ.get("MOE_VQLR_NVCC_EXTRA", "").split()      # e.g. -DMOE_VQLR_TRACE
+        cmd = [nvcc] + flags + extra + (["-Xptxas", "-v"] if verbose else []) + \
               ["-I", INCLUDE, "-o", LIB_PATH] + sources()
         subprocess.run(cmd, check=True)
     return LIB_PATH

@@ -33,6 +33,14 @@ constexpr int kDownThreads = 384;    // down: hi + lo activation fragments need 
 constexpr int kGroupTokens = 8;      // tokens of one work group = live rows of the m16 tile
 constexpr int kMaxDepth = 4;
 
+// Phase stamps cost instructions in the tile loops, so they are compiled in only for tracing builds
+// (nvcc -DMOE_VQLR_TRACE); the phase-clock query then returns real data.
+#ifdef MOE_VQLR_TRACE
+#define TRACE_STAMP(kern, k) stamp(P.clk, P.clk_blocks, kern, k)
+#else
+#define TRACE_STAMP(kern, k) ((void)0)
+#endif
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -203,10 +211,10 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
   const int E = P.E, k = P.k, S = P.S;
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
   const int n_pairs = T * k;
-  stamp(P.clk, P.clk_blocks, 1, 0);
+  TRACE_STAMP(1, 0);
   for (int i = tid; i < T * E; i += nthr) R.logit[i] = __ldcg(P.logits + i);
   __syncthreads();
-  stamp(P.clk, P.clk_blocks, 1, 1);
+  TRACE_STAMP(1, 1);
   // ---- top-k and affinities, one warp per token -------------------------------------------
   // Logits become order-preserving unsigned keys, so that one redux.sync finds the warp maximum
   // and a second one the lowest expert id among the lanes that hold it.
@@ -300,7 +308,7 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
     }
     return;
   }
-  stamp(P.clk, P.clk_blocks, 1, 2);
+  TRACE_STAMP(1, 2);
   // ---- sort the pairs by (expert, token): four lanes share a pair and scan a quarter each ---
   for (int q0 = 0; q0 < n_pairs; q0 += nthr >> 2) {       // uniform trip count for the shuffles
     const int q = q0 + (tid >> 2);
@@ -332,7 +340,7 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
     }
   }
   __syncthreads();
-  stamp(P.clk, P.clk_blocks, 1, 3);
+  TRACE_STAMP(1, 3);
   // ---- work groups: a new group starts at every eighth pair of an expert's run -------------
   int base = 0;
   for (int p0 = 0; p0 < n_pairs; p0 += nthr) {
@@ -361,7 +369,7 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
   }
   if (tid == 0) *R.n_grp = base + S * sh_groups;
   __syncthreads();
-  stamp(P.clk, P.clk_blocks, 1, 4);
+  TRACE_STAMP(1, 4);
   if (write_global) {
     const int n_grp = *R.n_grp;
     for (int i = tid; i < n_pairs; i += nthr) { P.topk_id[i] = R.sel_id[i]; P.topk_w[i] = R.w[i]; }
@@ -500,7 +508,7 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   int4* s_meta = reinterpret_cast<int4*>(s_base + L.meta);     // [buf][team][tile of the batch] (pair offset, tile, tokens)
   const RouteSmem R = carve_route(s_base + L.route, T, P.E, P.k, P.S);
 
-  stamp(P.clk, P.clk_blocks, 0, 0);
+  TRACE_STAMP(0, 0);
   // ---- routing-independent prologue: code books and tokens start streaming into shared memory
   if (!DENSE) {
     for (int i = tid; i < P.K; i += blockDim.x) cp_async16(s_cb_g + i, P.gate.codebook + i);
@@ -515,20 +523,20 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
     }
   }
   cp_async_commit();
-  stamp(P.clk, P.clk_blocks, 0, 1);
+  TRACE_STAMP(0, 1);
   pdl_wait();      // logits and z of this call are complete
-  stamp(P.clk, P.clk_blocks, 0, 2);
+  TRACE_STAMP(0, 2);
   if (pl.n_lr > 0)
     for (int i = tid; i < T * 2 * rb; i += blockDim.x) {      // z as bf16 hi / lo blocks
       const float* zp = P.z + (size_t)i * 8;                   // z is [T][2][r], r a multiple of 8
       split_hi_lo(__ldcg(reinterpret_cast<const float4*>(zp)), __ldcg(reinterpret_cast<const float4*>(zp + 4)), s_zh[i], s_zl[i]);
     }
   route_in_block(P, T, R, blockIdx.x == 0, want_dbg != 0);
-  stamp(P.clk, P.clk_blocks, 1, 5);
+  TRACE_STAMP(1, 5);
   pdl_launch();
   cp_async_wait_pending(0);       // this thread's share of code book and tokens has landed ...
   __syncthreads();                // ... and so has everybody else's
-  stamp(P.clk, P.clk_blocks, 0, 3);
+  TRACE_STAMP(0, 3);
 
   const int team = warp / pl.team_warps, wi = warp - team * pl.team_warps;
   const int team_threads = pl.team_warps * 32;
@@ -545,56 +553,60 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   const int b_first = wi * 32 + 8 * c, rho_first = lr_group * 32 + 8 * c;
   const bool idx_live = b_first < nb, fac_live = has_lr && rho_first < P.r;
 
-  const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
-  const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx);
-  uint4* ring = s_ring + (size_t)warp * D * 2 * 32;                                   // [slot][proj][lane]
-  uint4* fring = s_fring + (size_t)(team * pl.n_lr + (has_lr ? lr_group : 0)) * D * 2 * 32;
+  // per-lane bases: row g of a tile, this warp's first block group / rank group
+  const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx) + (size_t)g * nb + b_first;
+  const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx) + (size_t)g * nb + b_first;
+  const bf16* fac_gp = P.gate.factor + (size_t)g * P.r + rho_first;
+  const bf16* fac_up = P.up.factor + (size_t)g * P.r + rho_first;
+  uint4* ring = s_ring + (size_t)warp * D * 2 * 32 + lane;                            // [slot][proj][lane]
+  uint4* fring = s_fring + (size_t)(team * pl.n_lr + (has_lr ? lr_group : 0)) * D * 2 * 32 + lane;
 
   // (group, tile) of the next tile to prefetch and of the tile being computed advance in step
   int pf_grp = n_my > 0 ? u_begin / pl.tiles : 0, pf_jt = n_my > 0 ? u_begin - pf_grp * pl.tiles : 0;
   int cur_grp = pf_grp, cur_jt = pf_jt;
-  auto issue = [&](int i) {
-    const size_t row = (size_t)R.grp_e[pf_grp] * P.I + pf_jt * 8 + g;
-    const int slot = i % D;
+  int pf_slot = 0, cur_slot = 0;
+  auto issue = [&]() {
+    const size_t row0 = (size_t)R.grp_e[pf_grp] * P.I + pf_jt * 8;     // first row of the tile
     if (ringed && idx_live) {
-      cp_async_idx8<IdxT>(ring + (slot * 2 + 0) * 32 + lane, idx_g + row * nb + b_first);
-      cp_async_idx8<IdxT>(ring + (slot * 2 + 1) * 32 + lane, idx_u + row * nb + b_first);
+      cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 0) * 32, idx_g + row0 * nb);
+      cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 1) * 32, idx_u + row0 * nb);
     }
     if (fac_live) {
-      cp_async16(fring + (slot * 2 + 0) * 32 + lane, P.gate.factor + row * P.r + rho_first);
-      cp_async16(fring + (slot * 2 + 1) * 32 + lane, P.up.factor + row * P.r + rho_first);
+      cp_async16(fring + (pf_slot * 2 + 0) * 32, fac_gp + row0 * P.r);
+      cp_async16(fring + (pf_slot * 2 + 1) * 32, fac_up + row0 * P.r);
     }
     if (++pf_jt == pl.tiles) { pf_jt = 0; ++pf_grp; }
+    if (++pf_slot == D) pf_slot = 0;
   };
 
-  stamp(P.clk, P.clk_blocks, 1, 6);
+  TRACE_STAMP(1, 6);
   uint4 fx[8];                       // activation fragments of the current slice
   int frag_grp = -1, frag_slice = -1;
   int buf = 0, r_in = 0;
   const int tid_team = tid - team * team_threads;
 
-  for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(i); cp_async_commit(); }
-  stamp(P.clk, P.clk_blocks, 1, 7);
+  for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(); cp_async_commit(); }
+  TRACE_STAMP(1, 7);
   for (int i = 0; i < n_my; ++i) {
-    if (i + D - 1 < n_my) issue(i + D - 1);
+    if (i + D - 1 < n_my) issue();
     cp_async_commit();
-    stamp(P.clk, P.clk_blocks, 0, 4 + 3 * i);
+    TRACE_STAMP(0, 4 + 3 * i);
     cp_async_wait_pending(D - 1);
-    stamp(P.clk, P.clk_blocks, 0, 5 + 3 * i);
-    const int grp = cur_grp, jt = cur_jt;
+    TRACE_STAMP(0, 5 + 3 * i);
+    const int grp = cur_grp, jt = cur_jt, slot = cur_slot;
     if (++cur_jt == pl.tiles) { cur_jt = 0; ++cur_grp; }
+    if (++cur_slot == D) cur_slot = 0;
     const int e = R.grp_e[grp], off = R.grp_off[grp], n_tok = R.grp_cnt[grp];
     const size_t row = (size_t)e * P.I + jt * 8 + g;       // this lane's weight row
-    const int slot = i % D;
     uint4 raw_g = {0, 0, 0, 0}, raw_u = {0, 0, 0, 0};
     uint4 fac_g = {0, 0, 0, 0}, fac_u = {0, 0, 0, 0};
     if (ringed && idx_live) {
-      raw_g = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32 + lane);
-      raw_u = ring_idx8<IdxT>(ring + (slot * 2 + 1) * 32 + lane);
+      raw_g = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32);
+      raw_u = ring_idx8<IdxT>(ring + (slot * 2 + 1) * 32);
     }
     if (fac_live) {
-      fac_g = fring[(slot * 2 + 0) * 32 + lane];
-      fac_u = fring[(slot * 2 + 1) * 32 + lane];
+      fac_g = fring[(slot * 2 + 0) * 32];
+      fac_u = fring[(slot * 2 + 1) * 32];
     }
     const int tok = g < n_tok ? R.pair_token[off + g] : -1;
     float acc_g[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -624,8 +636,8 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
       } else {
         if (!ringed) {
           if (b0 < nb) {
-            raw_g = load_idx_raw<IdxT>(idx_g + row * nb + b0);
-            raw_u = load_idx_raw<IdxT>(idx_u + row * nb + b0);
+            raw_g = load_idx_raw<IdxT>(static_cast<const IdxT*>(P.gate.idx) + row * nb + b0);
+            raw_u = load_idx_raw<IdxT>(static_cast<const IdxT*>(P.up.idx) + row * nb + b0);
           } else {
             raw_g = raw_u = make_uint4(0, 0, 0, 0);
           }
@@ -662,7 +674,7 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
       mma_block(acc_u[0], zuh, fu); mma_block(acc_u[1], zul, fu);
     }
     // ---- add the team's partial tiles and apply SwiGLU -----------------------------------
-    stamp(P.clk, P.clk_blocks, 0, 6 + 3 * i);
+    TRACE_STAMP(0, 6 + 3 * i);
     const int bslot = (buf * pl.n_teams + team) * pl.batch + r_in;
     float2* part = s_part + (size_t)bslot * 2 * pl.team_warps * 32;
     part[(0 * pl.team_warps + wi) * 32 + lane] = make_float2(acc_g[0][0] + acc_g[1][0], acc_g[0][1] + acc_g[1][1]);
@@ -680,6 +692,7 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
           const float2* pt = s_part + (size_t)(bbase + rt) * 2 * pl.team_warps * 32;
           const int src = 4 * m + (n >> 1);
           float gs = 0.f, us = 0.f;
+#pragma unroll 4
           for (int w = 0; w < pl.team_warps; ++w) {
             const float2 pg = pt[(0 * pl.team_warps + w) * 32 + src];
             const float2 pu = pt[(1 * pl.team_warps + w) * 32 + src];
@@ -699,7 +712,7 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
     }
   }
   cp_async_wait_pending(0);
-  stamp(P.clk, P.clk_blocks, 0, 15);
+  TRACE_STAMP(0, 15);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -741,12 +754,12 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   int* s_grp_e = reinterpret_cast<int*>(s_base + L.grp);
   int* s_grp_off = s_grp_e + max_groups;
   int* s_grp_cnt = s_grp_off + max_groups;
-  stamp(P.clk, P.clk_blocks, 2, 0);
+  TRACE_STAMP(2, 0);
   if (!DENSE)
     for (int i = tid; i < P.K; i += blockDim.x) cp_async16(s_cb + i, P.down.codebook + i);
   cp_async_commit();
   pdl_wait();      // p (and z_d) and the routing lists are complete
-  stamp(P.clk, P.clk_blocks, 2, 1);
+  TRACE_STAMP(2, 1);
   pdl_launch();
   const int n_grp = __ldcg(P.grp_n);
   for (int i = tid; i < n_grp; i += blockDim.x) {
@@ -754,7 +767,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   }
   cp_async_wait_pending(0);
   __syncthreads();
-  stamp(P.clk, P.clk_blocks, 2, 2);
+  TRACE_STAMP(2, 2);
 
   const int team = warp / pl.team_warps, wi = warp - team * pl.team_warps;
   const int team_threads = pl.team_warps * 32;
@@ -770,27 +783,30 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   const int b_first = wi * 32 + (DENSE ? c : 8 * c), rho_first = lr_group * 32 + 8 * c;
   const bool idx_live = DENSE ? (wi * 32 < nb) : (b_first < nb), fac_live = has_lr && rho_first < P.r;
 
-  const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
-  uint4* ring = s_ring + (size_t)warp * D * L.slot_u4 * 32;                        // [slot][chunk][lane]
-  uint4* fring = s_fring + (size_t)(team * pl.n_lr + (has_lr ? lr_group : 0)) * D * 32;
+  const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx) + (size_t)g * nb + b_first;
+  const uint4* dense_d = reinterpret_cast<const uint4*>(P.down.dense + (size_t)g * P.I) + b_first;
+  const bf16* fac_dp = P.down.factor + (size_t)g * P.r + rho_first;
+  uint4* ring = s_ring + (size_t)warp * D * L.slot_u4 * 32 + lane;                 // [slot][chunk][lane]
+  uint4* fring = s_fring + (size_t)(team * pl.n_lr + (has_lr ? lr_group : 0)) * D * 32 + lane;
 
   int pf_grp = n_my > 0 ? u_begin / pl.tiles : 0, pf_jt = n_my > 0 ? u_begin - pf_grp * pl.tiles : 0;
   int cur_grp = pf_grp, cur_jt = pf_jt;
-  auto issue = [&](int i) {
-    const size_t row = (size_t)s_grp_e[pf_grp] * P.H + pf_jt * 8 + g;
-    const int slot = i % D;
+  int pf_slot = 0, cur_slot = 0;
+  auto issue = [&]() {
+    const size_t row0 = (size_t)s_grp_e[pf_grp] * P.H + pf_jt * 8;
     if (ringed && idx_live) {
       if (DENSE) {
-        const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I);
+        const uint4* wd = dense_d + row0 * (P.I / 8);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-          if (b_first + 4 * j < nb) cp_async16(ring + (slot * 8 + j) * 32 + lane, wd + b_first + 4 * j);
+          if (b_first + 4 * j < nb) cp_async16(ring + (pf_slot * 8 + j) * 32, wd + 4 * j);
       } else {
-        cp_async_idx8<IdxT>(ring + slot * 32 + lane, idx_d + row * nb + b_first);
+        cp_async_idx8<IdxT>(ring + pf_slot * 32, idx_d + row0 * nb);
       }
     }
-    if (fac_live) cp_async16(fring + slot * 32 + lane, P.down.factor + row * P.r + rho_first);
+    if (fac_live) cp_async16(fring + pf_slot * 32, fac_dp + row0 * P.r);
     if (++pf_jt == pl.tiles) { pf_jt = 0; ++pf_grp; }
+    if (++pf_slot == D) pf_slot = 0;
   };
 
   uint4 fh[8], fl[8];
@@ -798,21 +814,21 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   int frag_grp = -1, frag_slice = -1, z_grp = -1, z_lg = -1;
   int buf = 0, r_in = 0;
 
-  for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(i); cp_async_commit(); }
-  stamp(P.clk, P.clk_blocks, 2, 3);
+  for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(); cp_async_commit(); }
+  TRACE_STAMP(2, 3);
   for (int i = 0; i < n_my; ++i) {
-    if (i + D - 1 < n_my) issue(i + D - 1);
+    if (i + D - 1 < n_my) issue();
     cp_async_commit();
     cp_async_wait_pending(D - 1);
-    if (i < 5) stamp(P.clk, P.clk_blocks, 2, 4 + 2 * i);
-    const int grp = cur_grp, jt = cur_jt;
+    if (i < 5) TRACE_STAMP(2, 4 + 2 * i);
+    const int grp = cur_grp, jt = cur_jt, slot = cur_slot;
     if (++cur_jt == pl.tiles) { cur_jt = 0; ++cur_grp; }
+    if (++cur_slot == D) cur_slot = 0;
     const int e = s_grp_e[grp], off = s_grp_off[grp], n_tok = s_grp_cnt[grp];
     const size_t row = (size_t)e * P.H + jt * 8 + g;
-    const int slot = i % D;
     uint4 raw = {0, 0, 0, 0}, fac = {0, 0, 0, 0};
-    if (!DENSE && ringed && idx_live) raw = ring_idx8<IdxT>(ring + slot * 32 + lane);
-    if (fac_live) fac = fring[slot * 32 + lane];
+    if (!DENSE && ringed && idx_live) raw = ring_idx8<IdxT>(ring + slot * 32);
+    if (fac_live) fac = fring[slot * 32];
     const int pos = g < n_tok ? off + g : -1;
     float acc[4][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // four independent chains
     for (int sl = wi; sl < pl.n_slices; sl += pl.team_warps) {
@@ -836,12 +852,12 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
         for (int j = 0; j < 8; ++j) {
           const int b = b0 + 4 * j;
           uint4 v = make_uint4(0, 0, 0, 0);
-          if (b < nb) v = ringed ? ring[(slot * 8 + j) * 32 + lane] : __ldg(wd + b);
+          if (b < nb) v = ringed ? ring[(slot * 8 + j) * 32] : __ldg(wd + b);
           mma_block(acc[j & 1], fh[j], v);
           mma_block(acc[2 + (j & 1)], fl[j], v);
         }
       } else {
-        if (!ringed) raw = b0 < nb ? load_idx_raw<IdxT>(idx_d + row * nb + b0) : make_uint4(0, 0, 0, 0);
+        if (!ringed) raw = b0 < nb ? load_idx_raw<IdxT>(static_cast<const IdxT*>(P.down.idx) + row * nb + b0) : make_uint4(0, 0, 0, 0);
         uint32_t id[8];                      // out-of-range groups: index 0, zero fragments
         unpack_idx8<IdxT>(raw, id);
 #pragma unroll
@@ -869,7 +885,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
       mma_block(acc[0], zh, f);
       mma_block(acc[2], zl, f);
     }
-    if (i < 5) stamp(P.clk, P.clk_blocks, 2, 5 + 2 * i);
+    if (i < 5) TRACE_STAMP(2, 5 + 2 * i);
     const int bslot = (buf * pl.n_teams + team) * pl.batch + r_in;
     float2* part = s_part + (size_t)bslot * pl.team_warps * 32;
     part[wi * 32 + lane] = make_float2((acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]), (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]));
@@ -884,6 +900,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
           const float2* pt = s_part + (size_t)(bbase + rt) * pl.team_warps * 32;
           const int src = 4 * m + (n >> 1);
           float sum = 0.f;
+#pragma unroll 4
           for (int w = 0; w < pl.team_warps; ++w) {
             const float2 v = pt[w * 32 + src];
             sum += (n & 1) ? v.y : v.x;
@@ -896,7 +913,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
     }
   }
   cp_async_wait_pending(0);
-  stamp(P.clk, P.clk_blocks, 2, 15);
+  TRACE_STAMP(2, 15);
 }
 
 // z_d[pos][rho] = <basis_down[rho], p[pos]> (link of the chain between gate/up and down).
