@@ -56,7 +56,9 @@ struct Params {
   bf16* p_hi;              // [maxT*(k+S)][I]   p rounded to bf16 ...
   bf16* p_lo;              // [maxT*(k+S)][I]   ... and the bf16 remainder (p = hi + lo to 2^-17)
   float* zd;               // [maxT*(k+S)][r]   basis_down * p per pair position
-  float* y;                // [maxT*(k+S)][H]   expert outputs before the weighted sum, by pair position
+  float* gpart;            // [parts][maxT*(k+S)][I]  partial gate tiles of the tensor-core chain
+  float* upart;            // [parts][maxT*(k+S)][I]  partial up tiles
+  float* ypart;            // [parts][maxT*(k+S)][H]  partial down tiles, by pair position
   int* inv_pos;            // [maxT][k+S]       pair position of (token, slot)
   int* status;             // [1]
   long long* clk;          // optional phase stamps [kernel 4][block][warp 16][stamp 16], or NULL

@@ -13,15 +13,17 @@
 // and its A registers are exactly the matching 16-byte activation block: no unpacking, no
 // shuffles, no FMAs on the CUDA cores.  Token rows 8..15 of the m16 tile are zero; an expert
 // with more than eight tokens is split into work groups of at most eight.
-// The low-rank term (Eq. 1) joins the same accumulator as more k: B = a row of the private
-// factor, A = z split into bf16 hi + lo so that nothing is lost against fp32.
-// The warps of a team (one per slice) add their partial tiles through shared memory in a fixed
-// order; nothing uses floating-point atomics, so results repeat bit for bit.
+// The low-rank term (Eq. 1) is the same product with more k: B = a row of the private factor,
+// A = z split into bf16 hi + lo so that nothing is lost against fp32; each group of 32 ranks is
+// one more "part" next to the slices.
+// Warps never wait for each other: a warp writes the partial tile of its part to global memory
+// and the next kernel of the chain adds the parts in a fixed order (the SwiGLU link for gate/up,
+// the combine for down).  Nothing uses floating-point atomics, so results repeat bit for bit.
 //
 // Kernel chain of a call, linked by programmatic dependent launch (each kernel starts its
 // routing-independent prologue while its predecessor drains):
 //   k_router_z_pdl -> k_gateup_mma (routing redone in every block from the logits)
-//                  -> [k_zdown_pdl] -> k_down_mma -> k_combine
+//                  -> k_act_zdown (sum of parts, SwiGLU, z_d) -> k_down_mma -> k_combine
 #pragma once
 #include "common.cuh"
 
@@ -142,12 +144,25 @@ __device__ __forceinline__ uint4 ring_idx8(const uint4* smem) {
 struct StagePlan {
   int nb;          // blocks per weight row = in_dim / 8
   int n_slices;    // ceil(nb / 32)
-  int team_warps;  // warps that share one row tile
-  int n_teams;     // teams per block
-  int tiles;       // row tiles per expert = out_dim / 8
   int n_lr;        // groups of 32 ranks = ceil(r / 32), 0 without a low-rank term
+  int n_parts;     // n_slices + n_lr: partial tiles that add up to one output tile
+  int tiles;       // row tiles per expert = out_dim / 8
   int depth;       // tiles each warp keeps in flight in its shared-memory ring (2..4)
-  int batch;       // row tiles a team finishes between two of its barriers (1..4)
+};
+
+// Position in the flattened work list of a stage: unit = ((group * n_parts) + part) * tiles + tile.
+struct Cursor {
+  int grp, part, jt;
+  __device__ __forceinline__ void set(int v, const StagePlan& pl) {
+    const int per_grp = pl.n_parts * pl.tiles;
+    grp = v / per_grp;
+    const int rem = v - grp * per_grp;
+    part = rem / pl.tiles;
+    jt = rem - part * pl.tiles;
+  }
+  __device__ __forceinline__ void next(const StagePlan& pl) {
+    if (++jt == pl.tiles) { jt = 0; if (++part == pl.n_parts) { part = 0; ++grp; } }
+  }
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -466,10 +481,11 @@ __device__ __forceinline__ int split_begin(int total, int parts, int idx) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// k_gateup_mma
+// k_gateup_mma: partial gate / up tiles.  A warp owns one part (a 256-value slice of H, or 32
+// ranks of the low-rank term) of one work group and walks a contiguous range of row tiles.
 // ---------------------------------------------------------------------------------------------
 struct GuLayout {         // byte offsets into dynamic shared memory
-  size_t cb_u, x, ring, fring, z, part, meta, route, total;
+  size_t cb_u, x, ring, z, route, total;
 };
 
 __host__ __device__ inline GuLayout gu_layout(int K, int n_books, int T, int H, int r, const StagePlan& pl,
@@ -480,10 +496,7 @@ __host__ __device__ inline GuLayout gu_layout(int K, int n_books, int T, int H, 
   o = (size_t)n_books * K * 16;
   L.x = o;      o += (size_t)T * (H / 8 + 1) * 16;
   L.ring = o;   o += (size_t)warps * pl.depth * 2 * 32 * 16;
-  L.fring = o;  o += (size_t)pl.n_teams * (pl.n_lr > 0 ? pl.n_lr : 0) * pl.depth * 2 * 32 * 16;
   L.z = o;      o += (size_t)2 * T * 2 * ((r + 7) / 8) * 16;            // hi and lo blocks of z
-  L.part = o;   o += (size_t)2 * pl.n_teams * pl.batch * 2 * pl.team_warps * 32 * 8;
-  L.meta = o;   o += (size_t)2 * pl.n_teams * pl.batch * 16;
   L.route = o;  o += route_smem_bytes(T, E, k, S);
   L.total = o;
   return L;
@@ -496,16 +509,14 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   char* s_base = reinterpret_cast<char*>(s_u4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, c = lane & 3;
   const int nb = pl.nb, xs = nb + 1, D = pl.depth, rb = (P.r + 7) / 8;
-  const GuLayout L = gu_layout(P.K, n_books, T, P.H, P.r, pl, blockDim.x >> 5, P.E, P.k, P.S);
+  const int nwarps = blockDim.x >> 5;
+  const GuLayout L = gu_layout(P.K, n_books, T, P.H, P.r, pl, nwarps, P.E, P.k, P.S);
   uint4* s_cb_g = s_u4;
   uint4* s_cb_u = reinterpret_cast<uint4*>(s_base + L.cb_u);
   uint4* s_x = reinterpret_cast<uint4*>(s_base + L.x);
-  uint4* s_ring = reinterpret_cast<uint4*>(s_base + L.ring);
-  uint4* s_fring = reinterpret_cast<uint4*>(s_base + L.fring);
+  uint4* ring = reinterpret_cast<uint4*>(s_base + L.ring) + (size_t)warp * D * 2 * 32 + lane;   // [slot][proj][lane]
   uint4* s_zh = reinterpret_cast<uint4*>(s_base + L.z);          // [T][2][rb]
   uint4* s_zl = s_zh + (size_t)T * 2 * rb;
-  float2* s_part = reinterpret_cast<float2*>(s_base + L.part);
-  int4* s_meta = reinterpret_cast<int4*>(s_base + L.meta);     // [buf][team][tile of the batch] (pair offset, tile, tokens)
   const RouteSmem R = carve_route(s_base + L.route, T, P.E, P.k, P.S);
 
   TRACE_STAMP(0, 0);
@@ -538,52 +549,41 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   __syncthreads();                // ... and so has everybody else's
   TRACE_STAMP(0, 3);
 
-  const int team = warp / pl.team_warps, wi = warp - team * pl.team_warps;
-  const int team_threads = pl.team_warps * 32;
-  const int n_grp = *R.n_grp;
-  const int U = n_grp * pl.tiles;
-  const int G = gridDim.x * pl.n_teams, tau = blockIdx.x * pl.n_teams + team;
-  const int u_begin = team < pl.n_teams ? split_begin(U, G, tau) : 0;
-  const int n_my = team < pl.n_teams ? split_begin(U, G, tau + 1) - u_begin : 0;
-  const bool spw_one = pl.n_slices <= pl.team_warps;         // one slice per warp: fragments stay put
-  const bool ringed = !DENSE && spw_one;
-  // low-rank group handled by this warp (groups are dealt from the last warp of the team down)
-  const int lr_group = pl.team_warps - 1 - wi;
-  const bool has_lr = lr_group < pl.n_lr;                    // n_lr is 0 for a dense projection
-  const int b_first = wi * 32 + 8 * c, rho_first = lr_group * 32 + 8 * c;
-  const bool idx_live = b_first < nb, fac_live = has_lr && rho_first < P.r;
+  const int n_grp = *R.n_grp, n_pos = T * (P.k + P.S);
+  const int V = n_grp * pl.n_parts * pl.tiles;
+  const int W = gridDim.x * nwarps, wid = blockIdx.x * nwarps + warp;
+  const int v_begin = split_begin(V, W, wid);
+  const int n_my = split_begin(V, W, wid + 1) - v_begin;
+  const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
+  const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx);
 
-  // per-lane bases: row g of a tile, this warp's first block group / rank group
-  const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx) + (size_t)g * nb + b_first;
-  const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx) + (size_t)g * nb + b_first;
-  const bf16* fac_gp = P.gate.factor + (size_t)g * P.r + rho_first;
-  const bf16* fac_up = P.up.factor + (size_t)g * P.r + rho_first;
-  uint4* ring = s_ring + (size_t)warp * D * 2 * 32 + lane;                            // [slot][proj][lane]
-  uint4* fring = s_fring + (size_t)(team * pl.n_lr + (has_lr ? lr_group : 0)) * D * 2 * 32 + lane;
-
-  // (group, tile) of the next tile to prefetch and of the tile being computed advance in step
-  int pf_grp = n_my > 0 ? u_begin / pl.tiles : 0, pf_jt = n_my > 0 ? u_begin - pf_grp * pl.tiles : 0;
-  int cur_grp = pf_grp, cur_jt = pf_jt;
+  Cursor pf, cur;
+  pf.set(n_my > 0 ? v_begin : 0, pl);
+  cur = pf;
   int pf_slot = 0, cur_slot = 0;
-  auto issue = [&]() {
-    const size_t row0 = (size_t)R.grp_e[pf_grp] * P.I + pf_jt * 8;     // first row of the tile
-    if (ringed && idx_live) {
-      cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 0) * 32, idx_g + row0 * nb);
-      cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 1) * 32, idx_u + row0 * nb);
+  auto issue = [&]() {          // stream the bytes of the prefetch cursor's tile into the ring
+    if (!DENSE) {
+      const size_t row = (size_t)R.grp_e[pf.grp] * P.I + pf.jt * 8 + g;
+      if (pf.part < pl.n_slices) {
+        const int b = pf.part * 32 + 8 * c;
+        if (b < nb) {
+          cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 0) * 32, idx_g + row * nb + b);
+          cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 1) * 32, idx_u + row * nb + b);
+        }
+      } else {
+        const int rho = (pf.part - pl.n_slices) * 32 + 8 * c;
+        if (rho < P.r) {
+          cp_async16(ring + (pf_slot * 2 + 0) * 32, P.gate.factor + row * P.r + rho);
+          cp_async16(ring + (pf_slot * 2 + 1) * 32, P.up.factor + row * P.r + rho);
+        }
+      }
     }
-    if (fac_live) {
-      cp_async16(fring + (pf_slot * 2 + 0) * 32, fac_gp + row0 * P.r);
-      cp_async16(fring + (pf_slot * 2 + 1) * 32, fac_up + row0 * P.r);
-    }
-    if (++pf_jt == pl.tiles) { pf_jt = 0; ++pf_grp; }
+    pf.next(pl);
     if (++pf_slot == D) pf_slot = 0;
   };
 
-  TRACE_STAMP(1, 6);
-  uint4 fx[8];                       // activation fragments of the current slice
-  int frag_grp = -1, frag_slice = -1;
-  int buf = 0, r_in = 0;
-  const int tid_team = tid - team * team_threads;
+  uint4 fx[8];                       // activation fragments of the current (group, part)
+  int frag_grp = -1, frag_part = -1;
 
   for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(); cp_async_commit(); }
   TRACE_STAMP(1, 7);
@@ -593,35 +593,26 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
     TRACE_STAMP(0, 4 + 3 * i);
     cp_async_wait_pending(D - 1);
     TRACE_STAMP(0, 5 + 3 * i);
-    const int grp = cur_grp, jt = cur_jt, slot = cur_slot;
-    if (++cur_jt == pl.tiles) { cur_jt = 0; ++cur_grp; }
+    const int grp = cur.grp, part = cur.part, jt = cur.jt, slot = cur_slot;
+    cur.next(pl);
     if (++cur_slot == D) cur_slot = 0;
-    const int e = R.grp_e[grp], off = R.grp_off[grp], n_tok = R.grp_cnt[grp];
-    const size_t row = (size_t)e * P.I + jt * 8 + g;       // this lane's weight row
-    uint4 raw_g = {0, 0, 0, 0}, raw_u = {0, 0, 0, 0};
-    uint4 fac_g = {0, 0, 0, 0}, fac_u = {0, 0, 0, 0};
-    if (ringed && idx_live) {
-      raw_g = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32);
-      raw_u = ring_idx8<IdxT>(ring + (slot * 2 + 1) * 32);
-    }
-    if (fac_live) {
-      fac_g = fring[(slot * 2 + 0) * 32];
-      fac_u = fring[(slot * 2 + 1) * 32];
-    }
+    const int off = R.grp_off[grp], n_tok = R.grp_cnt[grp];
     const int tok = g < n_tok ? R.pair_token[off + g] : -1;
+    const bool is_lr = part >= pl.n_slices;
     float acc_g[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     float acc_u[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-    for (int sl = wi; sl < pl.n_slices; sl += pl.team_warps) {
-      const int b0 = sl * 32 + (DENSE ? c : 8 * c);
-      if (frag_grp != grp || frag_slice != sl) {
+    if (!is_lr) {
+      const int b0 = part * 32 + (DENSE ? c : 8 * c);
+      if (frag_grp != grp || frag_part != part) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int b = b0 + (DENSE ? 4 * j : j);
           fx[j] = (tok >= 0 && b < nb) ? s_x[tok * xs + b] : make_uint4(0, 0, 0, 0);
         }
-        frag_grp = grp; frag_slice = sl;
+        frag_grp = grp; frag_part = part;
       }
       if (DENSE) {
+        const size_t row = (size_t)R.grp_e[grp] * P.I + jt * 8 + g;
         const uint4* wg = reinterpret_cast<const uint4*>(P.gate.dense + row * P.H);
         const uint4* wu = reinterpret_cast<const uint4*>(P.up.dense + row * P.H);
         uint4 vg[8], vu[8];
@@ -634,16 +625,13 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
 #pragma unroll
         for (int j = 0; j < 8; ++j) { mma_block(acc_g[j & 1], fx[j], vg[j]); mma_block(acc_u[j & 1], fx[j], vu[j]); }
       } else {
-        if (!ringed) {
-          if (b0 < nb) {
-            raw_g = load_idx_raw<IdxT>(static_cast<const IdxT*>(P.gate.idx) + row * nb + b0);
-            raw_u = load_idx_raw<IdxT>(static_cast<const IdxT*>(P.up.idx) + row * nb + b0);
-          } else {
-            raw_g = raw_u = make_uint4(0, 0, 0, 0);
-          }
+        // mma.sync needs the whole warp: lanes whose block group lies beyond the row run it
+        // with index 0 and zero activation fragments
+        uint4 raw_g = {0, 0, 0, 0}, raw_u = {0, 0, 0, 0};
+        if (b0 < nb) {
+          raw_g = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32);
+          raw_u = ring_idx8<IdxT>(ring + (slot * 2 + 1) * 32);
         }
-        // mma.sync needs the whole warp: lanes whose group lies beyond the row run it with
-        // index 0 and zero activation fragments
         uint32_t ig[8], iu[8];
         unpack_idx8<IdxT>(raw_g, ig);
         unpack_idx8<IdxT>(raw_u, iu);
@@ -653,62 +641,28 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
           mma_block(acc_u[j & 1], fx[j], s_cb_u[iu[j]]);
         }
       }
-    }
-    // joint accumulation of the low-rank term: more k for the same tile
-    for (int lg = lr_group; lg < pl.n_lr; lg += pl.team_warps) {
-      const int rho0 = lg * 32 + 8 * c;
-      uint4 fg = fac_g, fu = fac_u;
-      if (lg != lr_group) {
-        fg = fu = make_uint4(0, 0, 0, 0);
-        if (rho0 < P.r) {
-          fg = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + row * P.r + rho0));
-          fu = __ldg(reinterpret_cast<const uint4*>(P.up.factor + row * P.r + rho0));
-        }
-      }
+    } else {
+      // low-rank part: B = 8 ranks of this lane's factor row, A = the matching z values (hi, lo)
+      const int rho0 = (part - pl.n_slices) * 32 + 8 * c;
+      uint4 fg = {0, 0, 0, 0}, fu = {0, 0, 0, 0};
       uint4 zgh = {0, 0, 0, 0}, zgl = {0, 0, 0, 0}, zuh = {0, 0, 0, 0}, zul = {0, 0, 0, 0};
-      if (tok >= 0 && rho0 < P.r) {
-        const int ig2 = (tok * 2 + P.gate.zslot) * rb + (rho0 >> 3), iu2 = (tok * 2 + P.up.zslot) * rb + (rho0 >> 3);
-        zgh = s_zh[ig2]; zgl = s_zl[ig2]; zuh = s_zh[iu2]; zul = s_zl[iu2];
+      if (rho0 < P.r) {
+        fg = ring[(slot * 2 + 0) * 32];
+        fu = ring[(slot * 2 + 1) * 32];
+        if (tok >= 0) {
+          const int ig2 = (tok * 2 + P.gate.zslot) * rb + (rho0 >> 3), iu2 = (tok * 2 + P.up.zslot) * rb + (rho0 >> 3);
+          zgh = s_zh[ig2]; zgl = s_zl[ig2]; zuh = s_zh[iu2]; zul = s_zl[iu2];
+        }
       }
       mma_block(acc_g[0], zgh, fg); mma_block(acc_g[1], zgl, fg);
       mma_block(acc_u[0], zuh, fu); mma_block(acc_u[1], zul, fu);
     }
-    // ---- add the team's partial tiles and apply SwiGLU -----------------------------------
     TRACE_STAMP(0, 6 + 3 * i);
-    const int bslot = (buf * pl.n_teams + team) * pl.batch + r_in;
-    float2* part = s_part + (size_t)bslot * 2 * pl.team_warps * 32;
-    part[(0 * pl.team_warps + wi) * 32 + lane] = make_float2(acc_g[0][0] + acc_g[1][0], acc_g[0][1] + acc_g[1][1]);
-    part[(1 * pl.team_warps + wi) * 32 + lane] = make_float2(acc_u[0][0] + acc_u[1][0], acc_u[0][1] + acc_u[1][1]);
-    if (wi == 0 && lane == 0) s_meta[bslot] = make_int4(off, jt, n_tok, 0);
-    if (++r_in == pl.batch || i == n_my - 1) {
-      // one barrier per batch of tiles; then the batch's outputs (64 per tile: 8 tokens x 8 rows)
-      // are summed over the team's warps in a fixed order and passed through SwiGLU
-      if (pl.team_warps > 1) team_sync(1 + team, team_threads); else __syncwarp();
-      const int bbase = (buf * pl.n_teams + team) * pl.batch;
-      for (int q = tid_team; q < r_in * 64; q += team_threads) {
-        const int rt = q >> 6, m = (q >> 3) & 7, n = q & 7;   // tile of the batch, token, row
-        const int4 mt = s_meta[bbase + rt];
-        if (m < mt.z) {
-          const float2* pt = s_part + (size_t)(bbase + rt) * 2 * pl.team_warps * 32;
-          const int src = 4 * m + (n >> 1);
-          float gs = 0.f, us = 0.f;
-#pragma unroll 4
-          for (int w = 0; w < pl.team_warps; ++w) {
-            const float2 pg = pt[(0 * pl.team_warps + w) * 32 + src];
-            const float2 pu = pt[(1 * pl.team_warps + w) * 32 + src];
-            gs += (n & 1) ? pg.y : pg.x;
-            us += (n & 1) ? pu.y : pu.x;
-          }
-          const float pv = gs / (1.f + expf(-gs)) * us;       // silu(g) * u
-          const size_t at = (size_t)(mt.x + m) * P.I + mt.y * 8 + n;
-          const bf16 hi = __float2bfloat16_rn(pv);
-          P.p[at] = pv;
-          P.p_hi[at] = hi;                                       // the down kernel's mma fragments
-          P.p_lo[at] = __float2bfloat16_rn(pv - __bfloat162float(hi));
-        }
-      }
-      buf ^= 1;
-      r_in = 0;
+    // partial tile of this part: token g of the group, rows 2c and 2c+1 of the tile
+    if (g < n_tok) {
+      const size_t at = ((size_t)part * n_pos + off + g) * P.I + jt * 8 + 2 * c;
+      *reinterpret_cast<float2*>(P.gpart + at) = make_float2(acc_g[0][0] + acc_g[1][0], acc_g[0][1] + acc_g[1][1]);
+      *reinterpret_cast<float2*>(P.upart + at) = make_float2(acc_u[0][0] + acc_u[1][0], acc_u[0][1] + acc_u[1][1]);
     }
   }
   cp_async_wait_pending(0);
@@ -716,12 +670,93 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
 }
 
 // ---------------------------------------------------------------------------------------------
-// k_down_mma: y[token][slot][h] for every (work group, 8-row tile of H); activations are the
-// fp32 intermediates p split into bf16 hi + lo fragments.
+// k_act_zdown: one block per pair.  p = silu(sum of gate parts) * (sum of up parts), kept as
+// bf16 hi + lo for the down kernel's fragments, then z_d = basis_down * p when the down
+// projection is compressed.  Parts are added in ascending order.
+// ---------------------------------------------------------------------------------------------
+constexpr int kActThreads = 384;
+
+// grid = n_pos * zsplit blocks: block (pos, zs) rebuilds p[pos] (cheap, from L2) and computes the
+// z_d rows rho = zs, zs + zsplit, ...; only zs == 0 writes p_hi / p_lo.
+__global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n_pos, int n_parts, int with_zd, int zsplit) {
+  extern __shared__ float s_p[];                 // [I]
+  pdl_launch();                                  // the down kernel may stage its code book meanwhile
+  pdl_wait();
+  const int pos = blockIdx.x / zsplit, zs = blockIdx.x - pos * zsplit, tid = threadIdx.x;
+  const size_t part_stride = (size_t)n_pos * P.I;
+  for (int i2 = tid; i2 < P.I / 2; i2 += blockDim.x) {
+    float g0 = 0.f, g1 = 0.f, u0 = 0.f, u1 = 0.f;
+    const size_t base = (size_t)pos * P.I + 2 * i2;
+    for (int part0 = 0; part0 < n_parts; part0 += 6) {        // six parts' loads in flight, summed in order
+      float2 gv[6], uv[6];
+#pragma unroll
+      for (int q = 0; q < 6; ++q) {
+        const bool live = part0 + q < n_parts;
+        gv[q] = live ? __ldcg(reinterpret_cast<const float2*>(P.gpart + base + (part0 + q) * part_stride)) : make_float2(0.f, 0.f);
+        uv[q] = live ? __ldcg(reinterpret_cast<const float2*>(P.upart + base + (part0 + q) * part_stride)) : make_float2(0.f, 0.f);
+      }
+#pragma unroll
+      for (int q = 0; q < 6; ++q) { g0 += gv[q].x; g1 += gv[q].y; u0 += uv[q].x; u1 += uv[q].y; }
+    }
+    const float p0 = g0 / (1.f + expf(-g0)) * u0, p1 = g1 / (1.f + expf(-g1)) * u1;   // silu(g) * u
+    s_p[2 * i2] = p0;
+    s_p[2 * i2 + 1] = p1;
+    if (zs == 0) {
+      const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);
+      *reinterpret_cast<__nv_bfloat162*>(P.p_hi + base) = hi;
+      *reinterpret_cast<__nv_bfloat162*>(P.p_lo + base) =
+          __floats2bfloat162_rn(p0 - __low2float(hi), p1 - __high2float(hi));
+    }
+  }
+  if (!with_zd) return;
+  __syncthreads();
+  const int lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
+  const int nchunk = P.I / 8;
+  // two rows of the basis per warp at a time, their loads in flight together
+  for (int rho = zs + warp * zsplit; rho < P.r; rho += 2 * nwarp * zsplit) {
+    const int rho2 = rho + nwarp * zsplit;
+    const bool two = rho2 < P.r;
+    const uint4* brow0 = reinterpret_cast<const uint4*>(P.down.basis + (size_t)rho * P.I);
+    const uint4* brow1 = reinterpret_cast<const uint4*>(P.down.basis + (size_t)(two ? rho2 : rho) * P.I);
+    float acc0 = 0.f, acc1 = 0.f;
+    for (int c0 = 0; c0 < nchunk; c0 += 96) {                // three chunks per lane and row in flight
+      uint4 w0[3], w1[3];
+#pragma unroll
+      for (int q = 0; q < 3; ++q) {
+        const int cidx = c0 + q * 32 + lane;
+        w0[q] = cidx < nchunk ? __ldg(brow0 + cidx) : make_uint4(0, 0, 0, 0);
+        w1[q] = cidx < nchunk ? __ldg(brow1 + cidx) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int q = 0; q < 3; ++q) {
+        const int cidx = c0 + q * 32 + lane;
+        if (cidx < nchunk) {
+          const float4 p0 = *reinterpret_cast<const float4*>(s_p + 8 * cidx), p1 = *reinterpret_cast<const float4*>(s_p + 8 * cidx + 4);
+          const float pf[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+          float wf[8];
+          unpack8(w0[q], wf);
+          acc0 = dot8(wf, pf, acc0);
+          unpack8(w1[q], wf);
+          acc1 = dot8(wf, pf, acc1);
+        }
+      }
+    }
+    acc0 = warp_sum(acc0);
+    acc1 = warp_sum(acc1);
+    if (lane == 0) {
+      P.zd[(size_t)pos * P.r + rho] = acc0;
+      if (two) P.zd[(size_t)pos * P.r + rho2] = acc1;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// k_down_mma: partial y tiles for every (work group, part, 8-row tile of H); activations are the
+// bf16 hi + lo halves of p (or of z_d for a low-rank part).
 // ---------------------------------------------------------------------------------------------
 struct DnLayout {
-  size_t ring, fring, part, yrow, grp, total;
-  int slot_u4;      // uint4 per lane per ring slot: 1 (indices) or 8 (a dense 256-value slice of a row)
+  size_t ring, grp, total;
+  int slot_u4;      // uint4 per lane per ring slot: 1 (indices / factor) or 8 (a dense 256-value slice)
 };
 
 __host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& pl, int warps, int max_groups) {
@@ -729,9 +764,6 @@ __host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& p
   size_t o = vq ? (size_t)K * 16 : 0;
   L.slot_u4 = vq ? 1 : 8;
   L.ring = o;   o += (size_t)warps * pl.depth * L.slot_u4 * 32 * 16;
-  L.fring = o;  o += (size_t)pl.n_teams * (pl.n_lr > 0 ? pl.n_lr : 0) * pl.depth * 32 * 16;
-  L.part = o;   o += (size_t)2 * pl.n_teams * pl.batch * pl.team_warps * 32 * 8;
-  L.yrow = o;   o += (size_t)2 * pl.n_teams * pl.batch * 16;
   L.grp = o;    o += ((size_t)max_groups * 12 + 15) / 16 * 16;
   L.total = o;
   return L;
@@ -743,17 +775,14 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   extern __shared__ uint4 s_u4[];
   char* s_base = reinterpret_cast<char*>(s_u4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, c = lane & 3;
-  const int nb = pl.nb, D = pl.depth;
-  const int max_groups = T * (P.k + P.S);
-  const DnLayout L = dn_layout(P.K, !DENSE, pl, blockDim.x >> 5, max_groups);
+  const int nb = pl.nb, D = pl.depth, nwarps = blockDim.x >> 5;
+  const int n_pos = T * (P.k + P.S);
+  const DnLayout L = dn_layout(P.K, !DENSE, pl, nwarps, n_pos);
   uint4* s_cb = s_u4;
-  uint4* s_ring = reinterpret_cast<uint4*>(s_base + L.ring);
-  uint4* s_fring = reinterpret_cast<uint4*>(s_base + L.fring);
-  float2* s_part = reinterpret_cast<float2*>(s_base + L.part);
-  int4* s_meta = reinterpret_cast<int4*>(s_base + L.yrow);   // [buf][team][tile of the batch] (pair offset, tile, tokens)
+  uint4* ring = reinterpret_cast<uint4*>(s_base + L.ring) + (size_t)warp * D * L.slot_u4 * 32 + lane;   // [slot][chunk][lane]
   int* s_grp_e = reinterpret_cast<int*>(s_base + L.grp);
-  int* s_grp_off = s_grp_e + max_groups;
-  int* s_grp_cnt = s_grp_off + max_groups;
+  int* s_grp_off = s_grp_e + n_pos;
+  int* s_grp_cnt = s_grp_off + n_pos;
   TRACE_STAMP(2, 0);
   if (!DENSE)
     for (int i = tid; i < P.K; i += blockDim.x) cp_async16(s_cb + i, P.down.codebook + i);
@@ -769,50 +798,38 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   __syncthreads();
   TRACE_STAMP(2, 2);
 
-  const int team = warp / pl.team_warps, wi = warp - team * pl.team_warps;
-  const int team_threads = pl.team_warps * 32;
-  const int tid_team = tid - team * team_threads;
-  const int U = n_grp * pl.tiles;
-  const int G = gridDim.x * pl.n_teams, tau = blockIdx.x * pl.n_teams + team;
-  const int u_begin = team < pl.n_teams ? split_begin(U, G, tau) : 0;
-  const int n_my = team < pl.n_teams ? split_begin(U, G, tau + 1) - u_begin : 0;
-  const bool spw_one = pl.n_slices <= pl.team_warps;
-  const bool ringed = spw_one;
-  const int lr_group = pl.team_warps - 1 - wi;
-  const bool has_lr = lr_group < pl.n_lr;
-  const int b_first = wi * 32 + (DENSE ? c : 8 * c), rho_first = lr_group * 32 + 8 * c;
-  const bool idx_live = DENSE ? (wi * 32 < nb) : (b_first < nb), fac_live = has_lr && rho_first < P.r;
+  const int V = n_grp * pl.n_parts * pl.tiles;
+  const int W = gridDim.x * nwarps, wid = blockIdx.x * nwarps + warp;
+  const int v_begin = split_begin(V, W, wid);
+  const int n_my = split_begin(V, W, wid + 1) - v_begin;
+  const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
 
-  const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx) + (size_t)g * nb + b_first;
-  const uint4* dense_d = reinterpret_cast<const uint4*>(P.down.dense + (size_t)g * P.I) + b_first;
-  const bf16* fac_dp = P.down.factor + (size_t)g * P.r + rho_first;
-  uint4* ring = s_ring + (size_t)warp * D * L.slot_u4 * 32 + lane;                 // [slot][chunk][lane]
-  uint4* fring = s_fring + (size_t)(team * pl.n_lr + (has_lr ? lr_group : 0)) * D * 32 + lane;
-
-  int pf_grp = n_my > 0 ? u_begin / pl.tiles : 0, pf_jt = n_my > 0 ? u_begin - pf_grp * pl.tiles : 0;
-  int cur_grp = pf_grp, cur_jt = pf_jt;
+  Cursor pf, cur;
+  pf.set(n_my > 0 ? v_begin : 0, pl);
+  cur = pf;
   int pf_slot = 0, cur_slot = 0;
   auto issue = [&]() {
-    const size_t row0 = (size_t)s_grp_e[pf_grp] * P.H + pf_jt * 8;
-    if (ringed && idx_live) {
+    const size_t row = (size_t)s_grp_e[pf.grp] * P.H + pf.jt * 8 + g;
+    if (pf.part < pl.n_slices) {
       if (DENSE) {
-        const uint4* wd = dense_d + row0 * (P.I / 8);
+        const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I) + pf.part * 32 + c;
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-          if (b_first + 4 * j < nb) cp_async16(ring + (pf_slot * 8 + j) * 32, wd + 4 * j);
+          if (pf.part * 32 + c + 4 * j < nb) cp_async16(ring + (pf_slot * 8 + j) * 32, wd + 4 * j);
       } else {
-        cp_async_idx8<IdxT>(ring + pf_slot * 32, idx_d + row0 * nb);
+        const int b = pf.part * 32 + 8 * c;
+        if (b < nb) cp_async_idx8<IdxT>(ring + pf_slot * 32, idx_d + row * nb + b);
       }
+    } else {
+      const int rho = (pf.part - pl.n_slices) * 32 + 8 * c;
+      if (rho < P.r) cp_async16(ring + pf_slot * L.slot_u4 * 32, P.down.factor + row * P.r + rho);
     }
-    if (fac_live) cp_async16(fring + pf_slot * 32, fac_dp + row0 * P.r);
-    if (++pf_jt == pl.tiles) { pf_jt = 0; ++pf_grp; }
+    pf.next(pl);
     if (++pf_slot == D) pf_slot = 0;
   };
 
   uint4 fh[8], fl[8];
-  uint4 zh = {0, 0, 0, 0}, zl = {0, 0, 0, 0};
-  int frag_grp = -1, frag_slice = -1, z_grp = -1, z_lg = -1;
-  int buf = 0, r_in = 0;
+  int frag_grp = -1, frag_part = -1;
 
   for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(); cp_async_commit(); }
   TRACE_STAMP(2, 3);
@@ -821,19 +838,16 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
     cp_async_commit();
     cp_async_wait_pending(D - 1);
     if (i < 5) TRACE_STAMP(2, 4 + 2 * i);
-    const int grp = cur_grp, jt = cur_jt, slot = cur_slot;
-    if (++cur_jt == pl.tiles) { cur_jt = 0; ++cur_grp; }
+    const int grp = cur.grp, part = cur.part, jt = cur.jt, slot = cur_slot;
+    cur.next(pl);
     if (++cur_slot == D) cur_slot = 0;
-    const int e = s_grp_e[grp], off = s_grp_off[grp], n_tok = s_grp_cnt[grp];
-    const size_t row = (size_t)e * P.H + jt * 8 + g;
-    uint4 raw = {0, 0, 0, 0}, fac = {0, 0, 0, 0};
-    if (!DENSE && ringed && idx_live) raw = ring_idx8<IdxT>(ring + slot * 32);
-    if (fac_live) fac = fring[slot * 32];
+    const int off = s_grp_off[grp], n_tok = s_grp_cnt[grp];
     const int pos = g < n_tok ? off + g : -1;
+    const bool is_lr = part >= pl.n_slices;
     float acc[4][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // four independent chains
-    for (int sl = wi; sl < pl.n_slices; sl += pl.team_warps) {
-      const int b0 = sl * 32 + (DENSE ? c : 8 * c);
-      if (frag_grp != grp || frag_slice != sl) {
+    if (!is_lr) {
+      const int b0 = part * 32 + (DENSE ? c : 8 * c);
+      if (frag_grp != grp || frag_part != part) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int b = b0 + (DENSE ? 4 * j : j);
@@ -844,21 +858,19 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
             fh[j] = fl[j] = make_uint4(0, 0, 0, 0);
           }
         }
-        frag_grp = grp; frag_slice = sl;
+        frag_grp = grp; frag_part = part;
       }
       if (DENSE) {
-        const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          const int b = b0 + 4 * j;
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (b < nb) v = ringed ? ring[(slot * 8 + j) * 32] : __ldg(wd + b);
+          const uint4 v = b0 + 4 * j < nb ? ring[(slot * 8 + j) * 32] : make_uint4(0, 0, 0, 0);
           mma_block(acc[j & 1], fh[j], v);
           mma_block(acc[2 + (j & 1)], fl[j], v);
         }
       } else {
-        if (!ringed) raw = b0 < nb ? load_idx_raw<IdxT>(static_cast<const IdxT*>(P.down.idx) + row * nb + b0) : make_uint4(0, 0, 0, 0);
-        uint32_t id[8];                      // out-of-range groups: index 0, zero fragments
+        uint4 raw = {0, 0, 0, 0};            // out-of-range groups: index 0, zero fragments
+        if (b0 < nb) raw = ring_idx8<IdxT>(ring + slot * 32);
+        uint32_t id[8];
         unpack_idx8<IdxT>(raw, id);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -867,92 +879,70 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
           mma_block(acc[2 + (j & 1)], fl[j], w);
         }
       }
-    }
-    for (int lg = lr_group; lg < pl.n_lr; lg += pl.team_warps) {
-      const int rho0 = lg * 32 + 8 * c;
-      uint4 f = fac;
-      if (lg != lr_group)
-        f = rho0 < P.r ? __ldg(reinterpret_cast<const uint4*>(P.down.factor + row * P.r + rho0)) : make_uint4(0, 0, 0, 0);
-      if (z_grp != grp || z_lg != lg) {
+    } else {
+      const int rho0 = (part - pl.n_slices) * 32 + 8 * c;
+      if (frag_grp != grp || frag_part != part) {        // z_d fragments live in fh[0] / fl[0]
         if (pos >= 0 && rho0 < P.r) {
           const float4* zp = reinterpret_cast<const float4*>(P.zd + (size_t)pos * P.r + rho0);
-          split_hi_lo(__ldcg(zp), __ldcg(zp + 1), zh, zl);
+          split_hi_lo(__ldcg(zp), __ldcg(zp + 1), fh[0], fl[0]);
         } else {
-          zh = zl = make_uint4(0, 0, 0, 0);
+          fh[0] = fl[0] = make_uint4(0, 0, 0, 0);
         }
-        z_grp = grp; z_lg = lg;
+        frag_grp = grp; frag_part = part;
       }
-      mma_block(acc[0], zh, f);
-      mma_block(acc[2], zl, f);
+      const uint4 f = rho0 < P.r ? ring[slot * L.slot_u4 * 32] : make_uint4(0, 0, 0, 0);
+      mma_block(acc[0], fh[0], f);
+      mma_block(acc[2], fl[0], f);
     }
     if (i < 5) TRACE_STAMP(2, 5 + 2 * i);
-    const int bslot = (buf * pl.n_teams + team) * pl.batch + r_in;
-    float2* part = s_part + (size_t)bslot * pl.team_warps * 32;
-    part[wi * 32 + lane] = make_float2((acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]), (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]));
-    if (wi == 0 && lane == 0) s_meta[bslot] = make_int4(off, jt, n_tok, 0);
-    if (++r_in == pl.batch || i == n_my - 1) {
-      if (pl.team_warps > 1) team_sync(1 + team, team_threads); else __syncwarp();
-      const int bbase = (buf * pl.n_teams + team) * pl.batch;
-      for (int q = tid_team; q < r_in * 64; q += team_threads) {
-        const int rt = q >> 6, m = (q >> 3) & 7, n = q & 7;
-        const int4 mt = s_meta[bbase + rt];
-        if (m < mt.z) {
-          const float2* pt = s_part + (size_t)(bbase + rt) * pl.team_warps * 32;
-          const int src = 4 * m + (n >> 1);
-          float sum = 0.f;
-#pragma unroll 4
-          for (int w = 0; w < pl.team_warps; ++w) {
-            const float2 v = pt[w * 32 + src];
-            sum += (n & 1) ? v.y : v.x;
-          }
-          P.y[(size_t)(mt.x + m) * P.H + mt.y * 8 + n] = sum;
-        }
-      }
-      buf ^= 1;
-      r_in = 0;
+    if (pos >= 0) {
+      const size_t at = ((size_t)part * n_pos + pos) * P.H + jt * 8 + 2 * c;
+      *reinterpret_cast<float2*>(P.ypart + at) =
+          make_float2((acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]), (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]));
     }
   }
   cp_async_wait_pending(0);
   TRACE_STAMP(2, 15);
 }
 
-// z_d[pos][rho] = <basis_down[rho], p[pos]> (link of the chain between gate/up and down).
-__global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos) {
-  pdl_wait();
-  pdl_launch();
-  const int lane = threadIdx.x & 31;
-  const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  if (w >= n_pos * P.r) return;
-  const int pos = w / P.r, rho = w - pos * P.r;
-  const uint4* brow = reinterpret_cast<const uint4*>(P.down.basis + (size_t)rho * P.I);
-  const float4* prow = reinterpret_cast<const float4*>(P.p + (size_t)pos * P.I);
-  float acc = 0.f;
-  for (int cidx = lane; cidx < P.I / 8; cidx += 32) {
-    float wf[8];
-    unpack8(__ldg(brow + cidx), wf);
-    const float4 p0 = __ldcg(prow + 2 * cidx), p1 = __ldcg(prow + 2 * cidx + 1);
-    const float pf[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
-    acc = dot8(wf, pf, acc);
-  }
-  acc = warp_sum(acc);
-  if (lane == 0) P.zd[(size_t)pos * P.r + rho] = acc;
-}
+// out[t][h] = sum over slots (in slot order) of affinity * y[t][slot][h], where y is the sum of
+// the down kernel's parts (ascending); shared experts weigh 1.  One block = one token and 64
+// pairs of columns; thread (column pair, slot lane) adds the parts of its slots with all loads
+// in flight, then the slot sums meet in shared memory and are added in slot order.
+constexpr int kCombineCols = 64;    // float2 columns per block
+constexpr int kCombineSlots = 8;    // slot lanes per column
 
-// out[t][h] = sum over slots (in slot order) of affinity * y[t][slot][h]; shared experts weigh 1.
-__global__ void __launch_bounds__(256) k_combine(const Params P, bf16* __restrict__ out, int T) {
+__global__ void __launch_bounds__(kCombineCols * kCombineSlots)
+k_combine(const Params P, bf16* __restrict__ out, int T, int n_parts) {
+  __shared__ float2 s_y[kMaxK + 8][kCombineCols];       // affinity-weighted y per slot (k + S <= 40)
   pdl_wait();
   pdl_launch();
-  const int n_slots = P.k + P.S, H2 = P.H / 2;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < T * H2; i += gridDim.x * blockDim.x) {
-    const int t = i / H2, h2 = i - t * H2;
-    float a0 = 0.f, a1 = 0.f;
-    for (int s = 0; s < n_slots; ++s) {
-      const int pos = __ldcg(P.inv_pos + t * n_slots + s);
-      const float w = __ldcg(P.pair_w + pos);
-      const float2 v = __ldcg(reinterpret_cast<const float2*>(P.y + (size_t)pos * P.H + 2 * h2));
-      a0 = fmaf(w, v.x, a0);
-      a1 = fmaf(w, v.y, a1);
+  const int n_slots = P.k + P.S, H2 = P.H / 2, n_pos = T * n_slots;
+  const int blocks_per_tok = (H2 + kCombineCols - 1) / kCombineCols;
+  const int t = blockIdx.x / blocks_per_tok, h2 = (blockIdx.x - t * blocks_per_tok) * kCombineCols + (threadIdx.x % kCombineCols);
+  const int sl = threadIdx.x / kCombineCols;
+  const size_t part_stride = (size_t)n_pos * P.H;
+  for (int s = sl; s < n_slots; s += kCombineSlots) {
+    const int pos = __ldcg(P.inv_pos + t * n_slots + s);
+    const float w = __ldcg(P.pair_w + pos);
+    float y0 = 0.f, y1 = 0.f;
+    if (h2 < H2) {
+      const float* src = P.ypart + (size_t)pos * P.H + 2 * h2;
+      for (int part0 = 0; part0 < n_parts; part0 += 4) {
+        float2 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          v[q] = part0 + q < n_parts ? __ldcg(reinterpret_cast<const float2*>(src + (part0 + q) * part_stride)) : make_float2(0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { y0 += v[q].x; y1 += v[q].y; }
+      }
     }
+    s_y[s][threadIdx.x % kCombineCols] = make_float2(w * y0, w * y1);
+  }
+  __syncthreads();
+  if (sl == 0 && h2 < H2) {
+    float a0 = 0.f, a1 = 0.f;
+    for (int s = 0; s < n_slots; ++s) { a0 += s_y[s][threadIdx.x].x; a1 += s_y[s][threadIdx.x].y; }
     *reinterpret_cast<__nv_bfloat162*>(out + (size_t)t * P.H + 2 * h2) = __floats2bfloat162_rn(a0, a1);
   }
 }

@@ -3,7 +3,7 @@
 //
 // Two kernel chains (all on the caller's stream):
 //   fast (tensor cores, fast_kernels.cuh), for shapes whose rows split into whole groups of
-//   eight blocks:  k_router_z_pdl -> k_gateup_mma -> [k_zdown_pdl] -> k_down_mma -> k_combine
+//   eight blocks:  k_router_z_pdl -> k_gateup_mma -> k_act_zdown -> k_down_mma -> k_combine
 //   generic (generic_kernels.cuh), for everything else:
 //                  k_router_z -> k_route -> k_gateup -> [k_zdown] -> k_down
 // Stages: router logits and the shared rank-r projections z = basis * x (Section 4.1: the work
@@ -74,17 +74,14 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 
 // Cuts one projection stage into slices and teams for `warps` warps per block.
-StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense, int warps) {
+StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense) {
   StagePlan pl;
   pl.nb = in_dim / kD;
   pl.n_slices = (pl.nb + 31) / 32;
-  pl.team_warps = pl.n_slices < warps ? pl.n_slices : warps;   // one warp per slice when they fit
-  pl.n_teams = warps / pl.team_warps;
-  if (pl.n_teams > 15 && pl.team_warps > 1) pl.n_teams = 15;   // named barriers 1..15
-  pl.tiles = out_dim / 8;
   pl.n_lr = (!dense && r > 0) ? (r + 31) / 32 : 0;
+  pl.n_parts = pl.n_slices + pl.n_lr;
+  pl.tiles = out_dim / 8;
   pl.depth = 2;
-  pl.batch = 1;
   return pl;
 }
 
@@ -165,12 +162,15 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         ran = true;
         break;
       }
-      case 3:
-        if (!h->dn_dense && P.r > 0) {
-          le = launch_pdl(k_zdown_pdl, (n_pos * P.r + 7) / 8, 256, 0, st, P, n_pos);
-          ran = true;
-        }
+      case 3: {
+        const int with_zd = (!h->dn_dense && P.r > 0) ? 1 : 0;
+        int zsplit = 1;                                   // few pairs: spread the z_d rows over more blocks
+        if (with_zd) while (n_pos * zsplit * 2 <= h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
+        le = launch_pdl(k_act_zdown, n_pos * zsplit, kActThreads, (size_t)P.I * sizeof(float), st, P, n_pos,
+                        h->plan_gu.n_parts, with_zd, zsplit);
+        ran = true;
         break;
+      }
       case 4:
         if (h->dn_dense) le = launch_pdl(k_down_mma<uint16_t, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, h->plan_dn);
         else if (h->idx_bytes == 1) le = launch_pdl(k_down_mma<uint8_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, h->plan_dn);
@@ -178,9 +178,8 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         ran = true;
         break;
       case 5: {
-        int grid = (T * P.H / 2 + 255) / 256;
-        if (grid > h->sm_count) grid = h->sm_count;
-        le = launch_pdl(k_combine, grid, 256, 0, st, P, ob, T);
+        const int grid = T * ((P.H / 2 + kCombineCols - 1) / kCombineCols);
+        le = launch_pdl(k_combine, grid, kCombineCols * kCombineSlots, 0, st, P, ob, T, h->plan_dn.n_parts);
         ran = true;
         break;
       }
@@ -325,32 +324,24 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     if (gu_vq && (H % 64 != 0 || (r % 8) != 0)) ok = false;       // whole groups of eight blocks / ranks
     if (!h->dn_dense && (I % 64 != 0 || (r % 8) != 0)) ok = false;
     if (gu_vq && r > 0 && (P.gate.zslot < 0 || P.up.zslot < 0)) ok = false;
+    if (k + S > kMaxK + 8) ok = false;                            // k_combine keeps one partial per slot in shared memory
     h->n_books = gu_vq ? (h->two_books ? 2 : 1) : 0;
-    h->plan_gu = plan_stage(I, H, r, gu_dn, (gu_dn ? kDenseThreads : kFastThreads) / 32);
-    h->plan_dn = plan_stage(H, I, r, h->dn_dense, kDownThreads / 32);
+    h->plan_gu = plan_stage(I, H, r, gu_dn);
+    h->plan_dn = plan_stage(H, I, r, h->dn_dense);
     // deepest rings that still fit the shared memory of one block
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
     const int gu_warps = (gu_dn ? kDenseThreads : kFastThreads) / 32;
-    // deepest rings and largest tile batches that fit: batch first (it removes barriers), then depth
-    {
-      bool found = false;
-      for (int bt = 4; bt >= 1 && !found; --bt)
-        for (int d = kMaxDepth; d >= 2 && !found; --d) {
-          h->plan_gu.batch = bt;
-          h->plan_gu.depth = d;
-          found = gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total <= limit;
-        }
-      found = false;
-      for (int bt = 4; bt >= 1 && !found; --bt)
-        for (int d = kMaxDepth; d >= 2 && !found; --d) {
-          h->plan_dn.batch = bt;
-          h->plan_dn.depth = d;
-          found = dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total <= limit;
-        }
+    for (int d = kMaxDepth; d >= 2; --d) {
+      h->plan_gu.depth = d;
+      if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total <= limit) break;
+    }
+    for (int d = kMaxDepth; d >= 2; --d) {
+      h->plan_dn.depth = d;
+      if (dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total <= limit) break;
     }
     const size_t smem_gu = gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total;
     h->smem_fast_dn = dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total;
-    if (smem_gu > limit || h->smem_fast_dn > limit) ok = false;
+    if (smem_gu > limit || h->smem_fast_dn > limit || (size_t)I * sizeof(float) > limit) ok = false;
     const char* force = getenv("MOE_VQLR_FORCE_GENERIC");
     if (force && force[0] == '1') ok = false;
     h->fast = ok;
@@ -363,7 +354,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       if (h->dn_dense) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
       else if (h->idx_bytes == 1) e2 = cudaFuncSetAttribute(k_down_mma<uint8_t, false>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
       else e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      if (e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); h->fast = false; }
+      cudaError_t e3 = cudaFuncSetAttribute(k_act_zdown, (cudaFuncAttribute)a, (int)((size_t)I * sizeof(float)));
+      if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) { cudaGetLastError(); h->fast = false; }
     }
   }
 
@@ -394,7 +386,9 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     P.p_hi = carve<bf16>(cur, n_pos * I);
     P.p_lo = carve<bf16>(cur, n_pos * I);
     P.zd = carve<float>(cur, n_pos * (r > 0 ? r : 1));
-    P.y = carve<float>(cur, n_pos * H);
+    P.gpart = carve<float>(cur, h->fast ? (size_t)h->plan_gu.n_parts * n_pos * I : 1);
+    P.upart = carve<float>(cur, h->fast ? (size_t)h->plan_gu.n_parts * n_pos * I : 1);
+    P.ypart = carve<float>(cur, h->fast ? (size_t)h->plan_dn.n_parts * n_pos * H : 1);
     P.inv_pos = carve<int>(cur, n_pos);
     P.status = carve<int>(cur, 1);
     if (want_clk) { P.clk = carve<long long>(cur, (size_t)4 * h->sm_count * 16 * 16); P.clk_blocks = h->sm_count; }
