@@ -751,18 +751,19 @@ __global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n
 }
 
 // ---------------------------------------------------------------------------------------------
-// k_down_mma: partial y tiles for every (work group, part, 8-row tile of H); activations are the
-// bf16 hi + lo halves of p (or of z_d for a low-rank part).
+// k_down_mma: partial y tiles for every (work group, slice of I, 8-row tile of H); activations
+// are the bf16 hi + lo halves of p.  The warp of slice s also adds the low-rank groups s,
+// s + n_slices, ... (32 ranks each; A = z_d as hi + lo), so the parts are the slices alone.
 // ---------------------------------------------------------------------------------------------
 struct DnLayout {
   size_t ring, grp, total;
-  int slot_u4;      // uint4 per lane per ring slot: 1 (indices / factor) or 8 (a dense 256-value slice)
+  int slot_u4;      // uint4 per lane per ring slot: 2 (indices, factor) or 8 (a dense 256-value slice)
 };
 
 __host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& pl, int warps, int max_groups) {
   DnLayout L;
   size_t o = vq ? (size_t)K * 16 : 0;
-  L.slot_u4 = vq ? 1 : 8;
+  L.slot_u4 = vq ? 2 : 8;
   L.ring = o;   o += (size_t)warps * pl.depth * L.slot_u4 * 32 * 16;
   L.grp = o;    o += ((size_t)max_groups * 12 + 15) / 16 * 16;
   L.total = o;
@@ -810,25 +811,22 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   int pf_slot = 0, cur_slot = 0;
   auto issue = [&]() {
     const size_t row = (size_t)s_grp_e[pf.grp] * P.H + pf.jt * 8 + g;
-    if (pf.part < pl.n_slices) {
-      if (DENSE) {
-        const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I) + pf.part * 32 + c;
+    if (DENSE) {
+      const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I) + pf.part * 32 + c;
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (pf.part * 32 + c + 4 * j < nb) cp_async16(ring + (pf_slot * 8 + j) * 32, wd + 4 * j);
-      } else {
-        const int b = pf.part * 32 + 8 * c;
-        if (b < nb) cp_async_idx8<IdxT>(ring + pf_slot * 32, idx_d + row * nb + b);
-      }
+      for (int j = 0; j < 8; ++j)
+        if (pf.part * 32 + c + 4 * j < nb) cp_async16(ring + (pf_slot * 8 + j) * 32, wd + 4 * j);
     } else {
-      const int rho = (pf.part - pl.n_slices) * 32 + 8 * c;
-      if (rho < P.r) cp_async16(ring + pf_slot * L.slot_u4 * 32, P.down.factor + row * P.r + rho);
+      const int b = pf.part * 32 + 8 * c, rho = pf.part * 32 + 8 * c;
+      if (b < nb) cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 0) * 32, idx_d + row * nb + b);
+      if (pf.part < pl.n_lr && rho < P.r) cp_async16(ring + (pf_slot * 2 + 1) * 32, P.down.factor + row * P.r + rho);
     }
     pf.next(pl);
     if (++pf_slot == D) pf_slot = 0;
   };
 
   uint4 fh[8], fl[8];
+  uint4 zh = {0, 0, 0, 0}, zl = {0, 0, 0, 0};     // z_d fragments of the low-rank group this part carries
   int frag_grp = -1, frag_part = -1;
 
   for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(); cp_async_commit(); }
@@ -843,56 +841,65 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
     if (++cur_slot == D) cur_slot = 0;
     const int off = s_grp_off[grp], n_tok = s_grp_cnt[grp];
     const int pos = g < n_tok ? off + g : -1;
-    const bool is_lr = part >= pl.n_slices;
+    const int b0 = part * 32 + (DENSE ? c : 8 * c);
+    const int rho0 = part * 32 + 8 * c;
     float acc[4][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // four independent chains
-    if (!is_lr) {
-      const int b0 = part * 32 + (DENSE ? c : 8 * c);
-      if (frag_grp != grp || frag_part != part) {
+    if (frag_grp != grp || frag_part != part) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int b = b0 + (DENSE ? 4 * j : j);
-          if (pos >= 0 && b < nb) {
-            fh[j] = __ldcg(reinterpret_cast<const uint4*>(P.p_hi + (size_t)pos * P.I) + b);
-            fl[j] = __ldcg(reinterpret_cast<const uint4*>(P.p_lo + (size_t)pos * P.I) + b);
-          } else {
-            fh[j] = fl[j] = make_uint4(0, 0, 0, 0);
-          }
+      for (int j = 0; j < 8; ++j) {
+        const int b = b0 + (DENSE ? 4 * j : j);
+        if (pos >= 0 && b < nb) {
+          fh[j] = __ldcg(reinterpret_cast<const uint4*>(P.p_hi + (size_t)pos * P.I) + b);
+          fl[j] = __ldcg(reinterpret_cast<const uint4*>(P.p_lo + (size_t)pos * P.I) + b);
+        } else {
+          fh[j] = fl[j] = make_uint4(0, 0, 0, 0);
         }
-        frag_grp = grp; frag_part = part;
       }
-      if (DENSE) {
+      zh = zl = make_uint4(0, 0, 0, 0);
+      if (!DENSE && part < pl.n_lr && pos >= 0 && rho0 < P.r) {
+        const float4* zp = reinterpret_cast<const float4*>(P.zd + (size_t)pos * P.r + rho0);
+        split_hi_lo(__ldcg(zp), __ldcg(zp + 1), zh, zl);
+      }
+      frag_grp = grp; frag_part = part;
+    }
+    if (DENSE) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint4 v = b0 + 4 * j < nb ? ring[(slot * 8 + j) * 32] : make_uint4(0, 0, 0, 0);
-          mma_block(acc[j & 1], fh[j], v);
-          mma_block(acc[2 + (j & 1)], fl[j], v);
-        }
-      } else {
-        uint4 raw = {0, 0, 0, 0};            // out-of-range groups: index 0, zero fragments
-        if (b0 < nb) raw = ring_idx8<IdxT>(ring + slot * 32);
-        uint32_t id[8];
-        unpack_idx8<IdxT>(raw, id);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint4 w = s_cb[id[j]];
-          mma_block(acc[j & 1], fh[j], w);
-          mma_block(acc[2 + (j & 1)], fl[j], w);
-        }
+      for (int j = 0; j < 8; ++j) {
+        const uint4 v = b0 + 4 * j < nb ? ring[(slot * 8 + j) * 32] : make_uint4(0, 0, 0, 0);
+        mma_block(acc[j & 1], fh[j], v);
+        mma_block(acc[2 + (j & 1)], fl[j], v);
       }
     } else {
-      const int rho0 = (part - pl.n_slices) * 32 + 8 * c;
-      if (frag_grp != grp || frag_part != part) {        // z_d fragments live in fh[0] / fl[0]
-        if (pos >= 0 && rho0 < P.r) {
-          const float4* zp = reinterpret_cast<const float4*>(P.zd + (size_t)pos * P.r + rho0);
-          split_hi_lo(__ldcg(zp), __ldcg(zp + 1), fh[0], fl[0]);
-        } else {
-          fh[0] = fl[0] = make_uint4(0, 0, 0, 0);
-        }
-        frag_grp = grp; frag_part = part;
+      // mma.sync needs the whole warp: out-of-range block groups use index 0 and zero fragments
+      uint4 raw = {0, 0, 0, 0};
+      if (b0 < nb) raw = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32);
+      uint32_t id[8];
+      unpack_idx8<IdxT>(raw, id);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint4 w = s_cb[id[j]];
+        mma_block(acc[j & 1], fh[j], w);
+        mma_block(acc[2 + (j & 1)], fl[j], w);
       }
-      const uint4 f = rho0 < P.r ? ring[slot * L.slot_u4 * 32] : make_uint4(0, 0, 0, 0);
-      mma_block(acc[0], fh[0], f);
-      mma_block(acc[2], fl[0], f);
+      if (part < pl.n_lr) {                   // warp-uniform: the low-rank group carried by this part
+        const uint4 f = rho0 < P.r ? ring[(slot * 2 + 1) * 32] : make_uint4(0, 0, 0, 0);
+        mma_block(acc[0], zh, f);
+        mma_block(acc[2], zl, f);
+        const size_t row = (size_t)s_grp_e[grp] * P.H + jt * 8 + g;
+        for (int lg = part + pl.n_slices; lg < pl.n_lr; lg += pl.n_slices) {   // more rank groups than slices
+          const int rho = lg * 32 + 8 * c;
+          uint4 f2 = {0, 0, 0, 0}, zh2 = {0, 0, 0, 0}, zl2 = {0, 0, 0, 0};
+          if (rho < P.r) {
+            f2 = __ldg(reinterpret_cast<const uint4*>(P.down.factor + row * P.r + rho));
+            if (pos >= 0) {
+              const float4* zp = reinterpret_cast<const float4*>(P.zd + (size_t)pos * P.r + rho);
+              split_hi_lo(__ldcg(zp), __ldcg(zp + 1), zh2, zl2);
+            }
+          }
+          mma_block(acc[1], zh2, f2);
+          mma_block(acc[3], zl2, f2);
+        }
+      }
     }
     if (i < 5) TRACE_STAMP(2, 5 + 2 * i);
     if (pos >= 0) {

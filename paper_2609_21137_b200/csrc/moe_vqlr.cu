@@ -328,6 +328,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->n_books = gu_vq ? (h->two_books ? 2 : 1) : 0;
     h->plan_gu = plan_stage(I, H, r, gu_dn);
     h->plan_dn = plan_stage(H, I, r, h->dn_dense);
+    h->plan_dn.n_parts = h->plan_dn.n_slices;          // the down kernel folds the low-rank groups into the slices
     // deepest rings that still fit the shared memory of one block
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
     const int gu_warps = (gu_dn ? kDenseThreads : kFastThreads) / 32;
