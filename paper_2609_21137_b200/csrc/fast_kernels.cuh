@@ -148,20 +148,39 @@ struct StagePlan {
   int n_parts;     // n_slices + n_lr: partial tiles that add up to one output tile
   int tiles;       // row tiles per expert = out_dim / 8
   int depth;       // tiles each warp keeps in flight in its shared-memory ring (2..4)
+  int chunk;       // consecutive row tiles of one part in the work order (see Cursor)
 };
 
-// Position in the flattened work list of a stage: unit = ((group * n_parts) + part) * tiles + tile.
+// Position in the flattened work list of a stage.  Units are ordered (group, chunk of `chunk`
+// row tiles, part, tile inside the chunk): a warp's contiguous range then mixes cheap low-rank
+// parts with lookup-heavy slice parts instead of drawing only one kind, while consecutive tiles
+// of one part still share its activation fragments.  chunk = tiles gives (group, part, tile).
 struct Cursor {
-  int grp, part, jt;
+  int grp, part, jt, chunk_end;       // jt = absolute tile, chunk_end = first tile after its chunk
   __device__ __forceinline__ void set(int v, const StagePlan& pl) {
     const int per_grp = pl.n_parts * pl.tiles;
     grp = v / per_grp;
-    const int rem = v - grp * per_grp;
-    part = rem / pl.tiles;
-    jt = rem - part * pl.tiles;
+    int rem = v - grp * per_grp;
+    const int per_chunk = pl.n_parts * pl.chunk;
+    const int ch = rem / per_chunk;                 // the last chunk may be shorter
+    rem -= ch * per_chunk;
+    const int c0 = ch * pl.chunk;
+    const int clen = min(pl.chunk, pl.tiles - c0);
+    part = rem / clen;
+    jt = c0 + (rem - part * clen);
+    chunk_end = c0 + clen;
   }
   __device__ __forceinline__ void next(const StagePlan& pl) {
-    if (++jt == pl.tiles) { jt = 0; if (++part == pl.n_parts) { part = 0; ++grp; } }
+    if (++jt == chunk_end) {
+      const int c0 = chunk_end - min(pl.chunk, chunk_end - ((chunk_end - 1) / pl.chunk) * pl.chunk);
+      if (++part == pl.n_parts) {
+        part = 0;
+        if (chunk_end == pl.tiles) { ++grp; jt = 0; chunk_end = min(pl.chunk, pl.tiles); }
+        else { jt = chunk_end; chunk_end = min(chunk_end + pl.chunk, pl.tiles); }
+      } else {
+        jt = c0;
+      }
+    }
   }
 };
 

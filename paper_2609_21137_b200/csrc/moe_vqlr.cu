@@ -82,6 +82,7 @@ StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense) {
   pl.n_parts = pl.n_slices + pl.n_lr;
   pl.tiles = out_dim / 8;
   pl.depth = 2;
+  pl.chunk = pl.tiles;
   return pl;
 }
 
@@ -328,6 +329,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->n_books = gu_vq ? (h->two_books ? 2 : 1) : 0;
     h->plan_gu = plan_stage(I, H, r, gu_dn);
     h->plan_dn = plan_stage(H, I, r, h->dn_dense);
+    if (h->plan_gu.n_lr > 0) h->plan_gu.chunk = h->plan_gu.tiles < 4 ? h->plan_gu.tiles : 4;   // mix slice and low-rank parts
     h->plan_dn.n_parts = h->plan_dn.n_slices;          // the down kernel folds the low-rank groups into the slices
     // deepest rings that still fit the shared memory of one block
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
