@@ -149,6 +149,9 @@ struct StagePlan {
   int tiles;       // row tiles per expert = out_dim / 8
   int depth;       // tiles each warp keeps in flight in its shared-memory ring (2..4)
   int chunk;       // consecutive row tiles of one part in the work order (see Cursor)
+  int x_smem;      // gate/up: tokens are staged in shared memory (else fragments come from global)
+  int repl;        // code book stored eight times, entry i of copy c at slot 8 i + c: lane l reads
+                   // copy l % 8, so the eight lanes of a quarter warp never share a bank group
 };
 
 // Position in the flattened work list of a stage.  Units are ordered (group, chunk of `chunk`
@@ -504,19 +507,21 @@ __device__ __forceinline__ int split_begin(int total, int parts, int idx) {
 // ranks of the low-rank term) of one work group and walks a contiguous range of row tiles.
 // ---------------------------------------------------------------------------------------------
 struct GuLayout {         // byte offsets into dynamic shared memory
-  size_t cb_u, x, ring, z, route, total;
+  size_t cb_u, x, ring, z, route, cb_tmp, total;
 };
 
 __host__ __device__ inline GuLayout gu_layout(int K, int n_books, int T, int H, int r, const StagePlan& pl,
                                               int warps, int E, int k, int S) {
   GuLayout L;
   size_t o = 0;
-  L.cb_u = n_books == 2 ? (size_t)K * 16 : 0;
-  o = (size_t)n_books * K * 16;
-  L.x = o;      o += (size_t)T * (H / 8 + 1) * 16;
+  const size_t cb_bytes = (size_t)K * 16 * (pl.repl ? 8 : 1);
+  L.cb_u = n_books == 2 ? cb_bytes : 0;
+  o = (size_t)n_books * cb_bytes;
+  L.x = o;      o += pl.x_smem ? (size_t)T * (H / 8 + 1) * 16 : 0;
   L.ring = o;   o += (size_t)warps * pl.depth * 2 * 32 * 16;
   L.z = o;      o += (size_t)2 * T * 2 * ((r + 7) / 8) * 16;            // hi and lo blocks of z
   L.route = o;  o += route_smem_bytes(T, E, k, S);
+  L.cb_tmp = o; o += pl.repl ? (size_t)n_books * K * 16 : 0;      // compact copy the replicas are made from
   L.total = o;
   return L;
 }
@@ -540,18 +545,20 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
 
   TRACE_STAMP(0, 0);
   // ---- routing-independent prologue: code books and tokens start streaming into shared memory
-  if (!DENSE) {
-    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(s_cb_g + i, P.gate.codebook + i);
+  const uint4* x4 = reinterpret_cast<const uint4*>(x);
+  uint4* s_tmp = reinterpret_cast<uint4*>(s_base + L.cb_tmp);
+  if (!DENSE) {       // a replicated book is fetched once and copied eight times inside shared memory
+    uint4* dst_g = pl.repl ? s_tmp : s_cb_g;
+    uint4* dst_u = pl.repl ? s_tmp + P.K : s_cb_u;
+    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_g + i, P.gate.codebook + i);
     if (n_books == 2)
-      for (int i = tid; i < P.K; i += blockDim.x) cp_async16(s_cb_u + i, P.up.codebook + i);
+      for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_u + i, P.up.codebook + i);
   }
-  {
-    const uint4* x4 = reinterpret_cast<const uint4*>(x);
+  if (pl.x_smem)
     for (int i = tid; i < T * nb; i += blockDim.x) {
       const int t = i / nb, b = i - t * nb;
       cp_async16(s_x + t * xs + b, x4 + i);
     }
-  }
   cp_async_commit();
   TRACE_STAMP(0, 1);
   pdl_wait();      // logits and z of this call are complete
@@ -566,6 +573,13 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   pdl_launch();
   cp_async_wait_pending(0);       // this thread's share of code book and tokens has landed ...
   __syncthreads();                // ... and so has everybody else's
+  if (!DENSE && pl.repl) {
+    for (int i = tid; i < P.K * 8; i += blockDim.x) {
+      s_cb_g[i] = s_tmp[i >> 3];
+      if (n_books == 2) s_cb_u[i] = s_tmp[P.K + (i >> 3)];
+    }
+    __syncthreads();
+  }
   TRACE_STAMP(0, 3);
 
   const int n_grp = *R.n_grp, n_pos = T * (P.k + P.S);
@@ -626,7 +640,7 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int b = b0 + (DENSE ? 4 * j : j);
-          fx[j] = (tok >= 0 && b < nb) ? s_x[tok * xs + b] : make_uint4(0, 0, 0, 0);
+          fx[j] = (tok >= 0 && b < nb) ? (pl.x_smem ? s_x[tok * xs + b] : __ldg(x4 + (size_t)tok * nb + b)) : make_uint4(0, 0, 0, 0);
         }
         frag_grp = grp; frag_part = part;
       }
@@ -654,10 +668,18 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
         uint32_t ig[8], iu[8];
         unpack_idx8<IdxT>(raw_g, ig);
         unpack_idx8<IdxT>(raw_u, iu);
+        if (pl.repl) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          mma_block(acc_g[j & 1], fx[j], s_cb_g[ig[j]]);
-          mma_block(acc_u[j & 1], fx[j], s_cb_u[iu[j]]);
+          for (int j = 0; j < 8; ++j) {
+            mma_block(acc_g[j & 1], fx[j], s_cb_g[(ig[j] << 3) | (lane & 7)]);
+            mma_block(acc_u[j & 1], fx[j], s_cb_u[(iu[j] << 3) | (lane & 7)]);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            mma_block(acc_g[j & 1], fx[j], s_cb_g[ig[j]]);
+            mma_block(acc_u[j & 1], fx[j], s_cb_u[iu[j]]);
+          }
         }
       }
     } else {
@@ -769,22 +791,87 @@ __global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n
   }
 }
 
+// The same link as two fully parallel kernels, for layers with few pairs or a long intermediate:
+// k_act (one thread per pair of p values) and k_zdown_pdl (one warp per z_d value).
+__global__ void __launch_bounds__(256) k_act(const Params P, int n_pos, int n_parts) {
+  pdl_launch();
+  pdl_wait();
+  const int I2 = P.I / 2;
+  const size_t part_stride = (size_t)n_pos * P.I;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_pos * I2; i += gridDim.x * blockDim.x) {
+    const size_t base = 2 * (size_t)i;                      // = pos * I + 2 * i2
+    float g0 = 0.f, g1 = 0.f, u0 = 0.f, u1 = 0.f;
+    for (int part0 = 0; part0 < n_parts; part0 += 6) {
+      float2 gv[6], uv[6];
+#pragma unroll
+      for (int q = 0; q < 6; ++q) {
+        const bool live = part0 + q < n_parts;
+        gv[q] = live ? __ldcg(reinterpret_cast<const float2*>(P.gpart + base + (part0 + q) * part_stride)) : make_float2(0.f, 0.f);
+        uv[q] = live ? __ldcg(reinterpret_cast<const float2*>(P.upart + base + (part0 + q) * part_stride)) : make_float2(0.f, 0.f);
+      }
+#pragma unroll
+      for (int q = 0; q < 6; ++q) { g0 += gv[q].x; g1 += gv[q].y; u0 += uv[q].x; u1 += uv[q].y; }
+    }
+    const float p0 = g0 / (1.f + expf(-g0)) * u0, p1 = g1 / (1.f + expf(-g1)) * u1;
+    *reinterpret_cast<float2*>(P.p + base) = make_float2(p0, p1);
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);
+    *reinterpret_cast<__nv_bfloat162*>(P.p_hi + base) = hi;
+    *reinterpret_cast<__nv_bfloat162*>(P.p_lo + base) =
+        __floats2bfloat162_rn(p0 - __low2float(hi), p1 - __high2float(hi));
+  }
+}
+
+__global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos) {
+  pdl_launch();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (w >= n_pos * P.r) return;
+  const int pos = w / P.r, rho = w - pos * P.r;
+  const uint4* brow = reinterpret_cast<const uint4*>(P.down.basis + (size_t)rho * P.I);
+  const float4* prow = reinterpret_cast<const float4*>(P.p + (size_t)pos * P.I);
+  const int nchunk = P.I / 8;
+  float acc = 0.f;
+  for (int c0 = 0; c0 < nchunk; c0 += 128) {
+    uint4 wv[4];
+    float4 pa[4], pb[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int cidx = c0 + q * 32 + lane;
+      const bool live = cidx < nchunk;
+      wv[q] = live ? __ldg(brow + cidx) : make_uint4(0, 0, 0, 0);
+      pa[q] = live ? __ldcg(prow + 2 * cidx) : make_float4(0.f, 0.f, 0.f, 0.f);
+      pb[q] = live ? __ldcg(prow + 2 * cidx + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float wf[8];
+      unpack8(wv[q], wf);
+      const float pf[8] = {pa[q].x, pa[q].y, pa[q].z, pa[q].w, pb[q].x, pb[q].y, pb[q].z, pb[q].w};
+      acc = dot8(wf, pf, acc);
+    }
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) P.zd[(size_t)pos * P.r + rho] = acc;
+}
+
 // ---------------------------------------------------------------------------------------------
 // k_down_mma: partial y tiles for every (work group, slice of I, 8-row tile of H); activations
 // are the bf16 hi + lo halves of p.  The warp of slice s also adds the low-rank groups s,
 // s + n_slices, ... (32 ranks each; A = z_d as hi + lo), so the parts are the slices alone.
 // ---------------------------------------------------------------------------------------------
 struct DnLayout {
-  size_t ring, grp, total;
+  size_t ring, grp, cb_tmp, total;
   int slot_u4;      // uint4 per lane per ring slot: 2 (indices, factor) or 8 (a dense 256-value slice)
 };
 
 __host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& pl, int warps, int max_groups) {
   DnLayout L;
-  size_t o = vq ? (size_t)K * 16 : 0;
+  size_t o = vq ? (size_t)K * 16 * (pl.repl ? 8 : 1) : 0;
   L.slot_u4 = vq ? 2 : 8;
   L.ring = o;   o += (size_t)warps * pl.depth * L.slot_u4 * 32 * 16;
   L.grp = o;    o += ((size_t)max_groups * 12 + 15) / 16 * 16;
+  L.cb_tmp = o; o += (vq && pl.repl) ? (size_t)K * 16 : 0;
   L.total = o;
   return L;
 }
@@ -804,8 +891,11 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   int* s_grp_off = s_grp_e + n_pos;
   int* s_grp_cnt = s_grp_off + n_pos;
   TRACE_STAMP(2, 0);
-  if (!DENSE)
-    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(s_cb + i, P.down.codebook + i);
+  uint4* s_tmp = reinterpret_cast<uint4*>(s_base + L.cb_tmp);
+  if (!DENSE) {
+    uint4* dst = pl.repl ? s_tmp : s_cb;
+    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst + i, P.down.codebook + i);
+  }
   cp_async_commit();
   pdl_wait();      // p (and z_d) and the routing lists are complete
   TRACE_STAMP(2, 1);
@@ -816,6 +906,10 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   }
   cp_async_wait_pending(0);
   __syncthreads();
+  if (!DENSE && pl.repl) {
+    for (int i = tid; i < P.K * 8; i += blockDim.x) s_cb[i] = s_tmp[i >> 3];
+    __syncthreads();
+  }
   TRACE_STAMP(2, 2);
 
   const int V = n_grp * pl.n_parts * pl.tiles;
@@ -896,7 +990,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
       unpack_idx8<IdxT>(raw, id);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const uint4 w = s_cb[id[j]];
+        const uint4 w = s_cb[pl.repl ? ((id[j] << 3) | (lane & 7)) : id[j]];
         mma_block(acc[j & 1], fh[j], w);
         mma_block(acc[2 + (j & 1)], fl[j], w);
       }

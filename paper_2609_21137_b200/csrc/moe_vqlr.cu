@@ -83,6 +83,8 @@ StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense) {
   pl.tiles = out_dim / 8;
   pl.depth = 2;
   pl.chunk = pl.tiles;
+  pl.x_smem = 1;
+  pl.repl = 0;
   return pl;
 }
 
@@ -165,10 +167,20 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
       }
       case 3: {
         const int with_zd = (!h->dn_dense && P.r > 0) ? 1 : 0;
-        int zsplit = 1;                                   // few pairs: spread the z_d rows over more blocks
-        if (with_zd) while (n_pos * zsplit * 2 <= h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
-        le = launch_pdl(k_act_zdown, n_pos * zsplit, kActThreads, (size_t)P.I * sizeof(float), st, P, n_pos,
-                        h->plan_gu.n_parts, with_zd, zsplit);
+        if (n_pos >= 32 && P.I <= 4096) {                 // one fused block per pair
+          int zsplit = 1;
+          if (with_zd) while (n_pos * zsplit * 2 <= h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
+          le = launch_pdl(k_act_zdown, n_pos * zsplit, kActThreads, (size_t)P.I * sizeof(float), st, P, n_pos,
+                          h->plan_gu.n_parts, with_zd, zsplit);
+        } else {                                          // few pairs or a long intermediate: two wide kernels
+          int grid = (n_pos * (P.I / 2) + 255) / 256;
+          if (grid > 4 * h->sm_count) grid = 4 * h->sm_count;
+          le = launch_pdl(k_act, grid, 256, 0, st, P, n_pos, h->plan_gu.n_parts);
+          if (le == cudaSuccess && with_zd) {
+            le = launch_pdl(k_zdown_pdl, (n_pos * P.r + 7) / 8, 256, 0, st, P, n_pos);
+            h->launches += 1;
+          }
+        }
         ran = true;
         break;
       }
@@ -331,9 +343,15 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->plan_dn = plan_stage(H, I, r, h->dn_dense);
     if (h->plan_gu.n_lr > 0) h->plan_gu.chunk = h->plan_gu.tiles < 4 ? h->plan_gu.tiles : 4;   // mix slice and low-rank parts
     h->plan_dn.n_parts = h->plan_dn.n_slices;          // the down kernel folds the low-rank groups into the slices
-    // deepest rings that still fit the shared memory of one block
+    // shared-memory plan: replicate a small code book eight times (conflict-free lookups), stage the
+    // tokens when they fit, then take the deepest rings that still fit
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
     const int gu_warps = (gu_dn ? kDenseThreads : kFastThreads) / 32;
+    h->plan_gu.repl = (gu_vq && (size_t)K * 128 * h->n_books <= 72 * 1024) ? 1 : 0;
+    h->plan_dn.repl = (!h->dn_dense && (size_t)K * 128 <= 72 * 1024) ? 1 : 0;
+    h->plan_gu.x_smem = 1;
+    h->plan_gu.depth = 2;
+    if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total > limit) h->plan_gu.x_smem = 0;
     for (int d = kMaxDepth; d >= 2; --d) {
       h->plan_gu.depth = d;
       if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total <= limit) break;
