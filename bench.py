@@ -26,6 +26,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) per launch of the dominant kernel, from the ncu captures summarised
+# in profiles/k_gateup_mma_k_down_mma_qwen3_*.md (small case; per-launch traffic is that of the
+# full benchmark because every launch reads one layer's activated experts).
+NCU_TRAFFIC = {("qwen3", "full", "gateup"): 8.01e6, ("qwen3", "full", "down"): 5.36e6,
+               ("qwen3_b16", "full", "gateup"): 42.5e6 + 0.37e6, ("qwen3_b16", "full", "down"): 28.7e6 + 0.05e6}
+
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
@@ -373,12 +379,29 @@ def main():
     achieved = stage_bytes[dominant] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": f"k_{dominant}", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                "traffic": None, "algorithmic_bytes_per_launch": stage_bytes[dominant],
+                "traffic": NCU_TRAFFIC.get((args.workload, args.mode, dominant)), "algorithmic_bytes_per_launch": stage_bytes[dominant],
                 "us_per_launch": dom_ms * 1e3,
                 "how": "each stage's kernel replayed back to back over the rotating layers in a captured graph, CUDA events",
                 "stage_us": {k_: v * 1e3 for k_, v in stage_ms.items()},
                 "layer": {"algorithmic_bytes": wl.mean_bytes, "gbs": layer_gbs, "frac_of_measured": layer_gbs / peak,
                           "frac_of_nominal_8TBs": layer_gbs / NOMINAL_HBM_GBS}}
+
+    # ---- second bound: shared-memory lookup rate (measured live by a probe kernel) ----------
+    lookup_bound = None
+    mean_lookups = sum(b.lookups for b in wl.bytes) / len(wl.bytes)
+    if mean_lookups > 0:
+        from paper_2609_21137_b200 import binding
+        n_books = 1
+        repl = shp.K * 128 * n_books <= 72 * 1024
+        rate = binding.probe_lookup_rate(shp.K, replicated=repl)
+        sm_mhz = (clocks.summary().get("sm_mhz") or 1965.0)
+        sms = torch.cuda.get_device_properties(device).multi_processor_count
+        t_us = mean_lookups / (rate * sms * sm_mhz)          # lookups / (lookups per us)
+        lookup_bound = {"what": "random 16-byte shared-memory code-word reads; the compressed projections cannot run faster than this",
+                        "lookups_per_layer": mean_lookups, "measured_lookups_per_clk_per_sm": rate,
+                        "replicated_codebook": bool(repl), "sms": sms, "sm_mhz": sm_mhz,
+                        "us_per_layer_at_that_rate": t_us, "frac_of_lookup_bound": t_us / (ms_per_step * 1e3),
+                        "hbm_us_per_layer_at_measured_peak": wl.mean_bytes / peak / 1e3}
 
     # ---- end to end through host buffers --------------------------------------------------
     e2e_steps = min(args.steps, 400)
@@ -427,7 +450,7 @@ def main():
                 "hbm_frac_of_nominal_8TBs": layer_gbs / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_layer": wl.mean_bytes, "distinct_experts_per_layer": wl.mean_active,
                 "gpu_launches": launches, "clocks": clocks.summary(), "roofline": roofline, "e2e": e2e,
-                "cpu_baseline": cpu, "extras": extras}
+                "lookup_bound": lookup_bound, "cpu_baseline": cpu, "extras": extras}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -172,6 +172,14 @@ int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h);
 /* Device workspace the handle owns, in bytes. */
 int64_t moe_vqlr_workspace_bytes(const moe_vqlr_handle* h);
 
+/* Measurement aid (no counterpart in the paper): runs a short probe kernel on the current device
+ * and returns how many random 16-byte shared-memory reads per clock one SM sustains from a
+ * code book of codebook_size entries (replicated != 0: the eightfold bank-replicated layout used
+ * for small code books).  This is the rate that bounds the compressed projections.  Synchronous;
+ * allocates and frees a few KB.  Returns OK, INVALID_ARG, UNSUPPORTED (book too large for shared
+ * memory), OOM or CUDA. */
+int moe_vqlr_probe_lookup_rate(int32_t codebook_size, int32_t replicated, double* lookups_per_clk_per_sm);
+
 /* Routing step only, for callers that must not allocate device memory (no counterpart in the
  * paper: it exists for processes where a memory pool or the host application owns every
  * allocation, so moe_vqlr_create(), which allocates a workspace, is off limits).  Computes

@@ -20,6 +20,8 @@ class LayerBytes:
     per_expert_down: int
     tokens_io: int
     n_active: int          # distinct activated experts, shared experts included
+    lookups_per_expert_gateup: int = 0   # code-word selections (one per length-d block), gate + up
+    lookups_per_expert_down: int = 0
 
     @property
     def per_expert(self) -> int:
@@ -37,6 +39,11 @@ class LayerBytes:
     @property
     def down_kernel(self) -> int:
         return self.n_active * self.per_expert_down
+
+    @property
+    def lookups(self) -> int:
+        """Code-word selections of the whole layer (the paper's `H I / d` per projection and expert)."""
+        return self.n_active * (self.lookups_per_expert_gateup + self.lookups_per_expert_down)
 
 
 def index_bits(K: int) -> int:
@@ -65,7 +72,9 @@ def layer_bytes(*, H: int, I: int, E: int, d: int, K: int, r: int, T: int, mode:
     return LayerBytes(router=2 * E * H, shared=shared,
                       per_expert_gateup=2 * projection_private_bytes(vq_gu, I, H, d, K, r),
                       per_expert_down=projection_private_bytes(vq_d, H, I, d, K, r),
-                      tokens_io=2 * 2 * T * H, n_active=n_active)
+                      tokens_io=2 * 2 * T * H, n_active=n_active,
+                      lookups_per_expert_gateup=2 * I * (H // d) if vq_gu else 0,
+                      lookups_per_expert_down=H * (I // d) if vq_d else 0)
 
 
 def dense_equivalent_bytes(H: int, I: int, n_active: int) -> int:

@@ -23,7 +23,7 @@ EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_ho
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",
            "moe_vqlr_workspace_bytes", "moe_vqlr_set_profiling", "moe_vqlr_last_stage_times",
            "moe_vqlr_stage_count", "moe_vqlr_stage_name", "moe_vqlr_route_noalloc",
-           "moe_vqlr_run_stage", "moe_vqlr_phase_clocks"]
+           "moe_vqlr_run_stage", "moe_vqlr_phase_clocks", "moe_vqlr_probe_lookup_rate"]
 
 
 class MoeVqlrError(RuntimeError):
@@ -87,6 +87,8 @@ def _load():
     lib.moe_vqlr_run_stage.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     lib.moe_vqlr_phase_clocks.restype = C.c_int64
     lib.moe_vqlr_phase_clocks.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
+    lib.moe_vqlr_probe_lookup_rate.restype = C.c_int
+    lib.moe_vqlr_probe_lookup_rate.argtypes = [C.c_int32, C.c_int32, C.POINTER(C.c_double)]
     lib.moe_vqlr_route_noalloc.restype = C.c_int
     lib.moe_vqlr_route_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int32] * 5 + \
                                           [C.c_void_p, C.c_void_p, C.c_void_p]
@@ -113,6 +115,15 @@ def bits_to_device(a: Optional[np.ndarray], device) -> Optional[torch.Tensor]:
 
 def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def probe_lookup_rate(codebook_size: int, replicated: bool = False) -> float:
+    """Random 16-byte shared-memory lookups per clock per SM on the current device (measured)."""
+    out = C.c_double()
+    rc = _lib.moe_vqlr_probe_lookup_rate(codebook_size, 1 if replicated else 0, C.byref(out))
+    if rc != OK:
+        raise MoeVqlrError(rc, "lookup-rate probe failed")
+    return float(out.value)
 
 
 def route_noalloc(x: torch.Tensor, router_w: torch.Tensor, router_bias: Optional[torch.Tensor],
