@@ -497,9 +497,11 @@ __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params
   }
 }
 
-// Splits `total` tiles evenly over `parts` teams: first tile of team `idx`.
+// Splits `total` units evenly over `parts` warps: first unit of warp `idx` = floor(total * idx / parts),
+// in 32-bit arithmetic (parts < 65536).
 __device__ __forceinline__ int split_begin(int total, int parts, int idx) {
-  return (int)(((long long)total * idx) / parts);
+  const unsigned int q = (unsigned int)total / (unsigned int)parts, rem = (unsigned int)total - q * (unsigned int)parts;
+  return (int)(q * (unsigned int)idx + (rem * (unsigned int)idx) / (unsigned int)parts);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -901,7 +903,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   TRACE_STAMP(2, 1);
   pdl_launch();
   const int n_grp = __ldcg(P.grp_n);
-  for (int i = tid; i < n_grp; i += blockDim.x) {
+  for (int i = tid; i < n_pos; i += blockDim.x) {      // all n_pos slots (>= n_grp): no dependent second trip
     s_grp_e[i] = __ldcg(P.grp_e + i); s_grp_off[i] = __ldcg(P.grp_off + i); s_grp_cnt[i] = __ldcg(P.grp_cnt + i);
   }
   cp_async_wait_pending(0);
