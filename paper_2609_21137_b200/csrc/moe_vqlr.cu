@@ -167,7 +167,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
       }
       case 3: {
         const int with_zd = (!h->dn_dense && P.r > 0) ? 1 : 0;
-        if (n_pos >= 32 && P.I <= 4096) {                 // one fused block per pair
+        if (P.I <= 4096) {                                // one fused block per pair (times zsplit)
           int zsplit = 1;
           if (with_zd) while (n_pos * zsplit * 2 <= h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
           le = launch_pdl(k_act_zdown, n_pos * zsplit, kActThreads, (size_t)P.I * sizeof(float), st, P, n_pos,
