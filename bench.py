@@ -415,7 +415,7 @@ def main():
     extras = []
     if rank == 0 and world == 1 and not args.no_extras:
         todo = [("qwen3", "paper"), ("qwen3", "dense"), ("qwen3_b16", "full"), ("qwen3_b16", "paper"),
-                ("qwen3_b16", "dense")]
+                ("qwen3_b16", "dense"), ("qwen3_deployed", "paper"), ("qwen3_deployed_b16", "paper")]
         todo = [t_ for t_ in todo if t_ != (args.workload, args.mode)]
         for name, mode in todo:
             try:

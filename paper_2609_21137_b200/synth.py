@@ -62,6 +62,16 @@ SHAPES: Dict[str, LayerShape] = {
     "mixtral_b4": LayerShape("mixtral_b4", H=4096, I=14336, E=8, k=2, d=8, K=4096, r=128, T=4),
     "mixtral_b16": LayerShape("mixtral_b16", H=4096, I=14336, E=8, k=2, d=8, K=4096, r=128,
                               T=16),
+    # the paper's own deployed operating points (evaluation-setup table): K = 256, uint8 indices,
+    # gate/up compressed, down kept in bf16 ("paper" mode), one code book per projection
+    "qwen3_deployed": LayerShape("qwen3_deployed", H=2048, I=768, E=128, k=8, d=8, K=256, r=384, T=1,
+                                 mode="paper", per_projection_codebook=True),
+    "qwen3_deployed_b16": LayerShape("qwen3_deployed_b16", H=2048, I=768, E=128, k=8, d=8, K=256, r=384,
+                                     T=16, router_bias=True, mode="paper", per_projection_codebook=True),
+    "dsv2lite_deployed": LayerShape("dsv2lite_deployed", H=2048, I=1408, E=64, k=6, d=8, K=256, r=384, T=1,
+                                    mode="paper", per_projection_codebook=True),
+    "gemma4_deployed": LayerShape("gemma4_deployed", H=2816, I=704, E=128, k=8, d=8, K=256, r=384, T=1,
+                                  mode="paper", per_projection_codebook=True),
 }
 
 

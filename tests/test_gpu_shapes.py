@@ -47,6 +47,26 @@ def test_more_slices_than_warps_b16():
     _sampled_check(shp, rows)
 
 
+@pytest.mark.parametrize("name", ["qwen3_deployed", "qwen3_deployed_b16", "gemma4_deployed"])
+def test_papers_deployed_operating_points(name):
+    # K = 256 / uint8, r = 384 (twelve low-rank parts), separate gate and up code books, bf16 down;
+    # fewer experts than the real models to keep the oracle quick (routing width is unchanged)
+    shp = synth.shape(name, E=24)
+    layer, res = None, None
+    for s in range(10):
+        layer = synth.make_layer(shp, seed=s)
+        res = oracle.OracleLayer.from_synth(layer).decode_layer(layer.x)
+        if logit_gaps(res, shp.k) > MIN_LOGIT_GAP:
+            break
+    from paper_2609_21137_b200 import binding
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    out, dbg = mod.decode(binding.bits_to_device(layer.x, "cuda"), debug=True)
+    torch.cuda.synchronize()
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out, what=name)
+    mod.close()
+
+
 def test_host_buffer_entry_point_matches_device_path():
     from paper_2609_21137_b200 import binding
     shp = synth.shape("qwen3_b16", E=32)
