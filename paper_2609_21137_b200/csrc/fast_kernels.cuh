@@ -435,14 +435,13 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
 // ---------------------------------------------------------------------------------------------
 constexpr int kRouterWarps = 2;
 
-__global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
-  pdl_wait();      // the previous call's kernels may still read logits / z
-  pdl_launch();
-  const int lane = threadIdx.x & 31;
-  const int unit = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
-  const int n_rows = P.E + P.n_zrows;
+// One unit = one (row, group of four tokens); executed by one warp.
+__device__ __forceinline__ int router_z_units(const Params& P, int T) {
+  return (P.E + P.n_zrows) * ((T + kTokGroup - 1) / kTokGroup);
+}
+
+__device__ __forceinline__ void router_z_unit(const Params& P, const bf16* __restrict__ x, int T, int unit, int lane) {
   const int n_groups = (T + kTokGroup - 1) / kTokGroup;
-  if (unit >= n_rows * n_groups) return;
   const int row = unit / n_groups, t0 = (unit - row * n_groups) * kTokGroup;
   const bf16* wrow;
   float* dst;
@@ -497,6 +496,13 @@ __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params
   }
 }
 
+__global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
+  pdl_wait();      // the previous call's kernels may still read logits / z
+  pdl_launch();
+  const int unit = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
+  if (unit < router_z_units(P, T)) router_z_unit(P, x, T, unit, threadIdx.x & 31);
+}
+
 // Splits `total` units evenly over `parts` warps: first unit of warp `idx` = floor(total * idx / parts),
 // in 32-bit arithmetic (parts < 65536).
 __device__ __forceinline__ int split_begin(int total, int parts, int idx) {
@@ -528,30 +534,36 @@ __host__ __device__ inline GuLayout gu_layout(int K, int n_books, int T, int H, 
   return L;
 }
 
-template <typename IdxT, bool DENSE>
-__global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
-k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {
-  extern __shared__ uint4 s_u4[];
-  char* s_base = reinterpret_cast<char*>(s_u4);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, c = lane & 3;
-  const int nb = pl.nb, xs = nb + 1, D = pl.depth, rb = (P.r + 7) / 8;
-  const int nwarps = blockDim.x >> 5;
-  const GuLayout L = gu_layout(P.K, n_books, T, P.H, P.r, pl, nwarps, P.E, P.k, P.S);
-  uint4* s_cb_g = s_u4;
-  uint4* s_cb_u = reinterpret_cast<uint4*>(s_base + L.cb_u);
-  uint4* s_x = reinterpret_cast<uint4*>(s_base + L.x);
-  uint4* ring = reinterpret_cast<uint4*>(s_base + L.ring) + (size_t)warp * D * 2 * 32 + lane;   // [slot][proj][lane]
-  uint4* s_zh = reinterpret_cast<uint4*>(s_base + L.z);          // [T][2][rb]
-  uint4* s_zl = s_zh + (size_t)T * 2 * rb;
-  const RouteSmem R = carve_route(s_base + L.route, T, P.E, P.k, P.S);
+// Shared-memory views of the gate/up stage.
+struct GuSmem {
+  uint4 *cb_g, *cb_u, *x, *ring, *zh, *zl, *tmp;
+  RouteSmem R;
+};
 
-  TRACE_STAMP(0, 0);
-  // ---- routing-independent prologue: code books and tokens start streaming into shared memory
+__device__ __forceinline__ GuSmem gu_carve(char* s_base, const GuLayout& L, const Params& P, int T, int warp, int lane, int depth) {
+  GuSmem m;
+  const int rb = (P.r + 7) / 8;
+  m.cb_g = reinterpret_cast<uint4*>(s_base);
+  m.cb_u = reinterpret_cast<uint4*>(s_base + L.cb_u);
+  m.x = reinterpret_cast<uint4*>(s_base + L.x);
+  m.ring = reinterpret_cast<uint4*>(s_base + L.ring) + (size_t)warp * depth * 2 * 32 + lane;   // [slot][proj][lane]
+  m.zh = reinterpret_cast<uint4*>(s_base + L.z);          // [T][2][rb]
+  m.zl = m.zh + (size_t)T * 2 * rb;
+  m.tmp = reinterpret_cast<uint4*>(s_base + L.cb_tmp);
+  m.R = carve_route(s_base + L.route, T, P.E, P.k, P.S);
+  return m;
+}
+
+// Routing-independent prologue: code books and tokens start streaming into shared memory
+// (one cp.async group per thread, not yet waited for).
+template <bool DENSE>
+__device__ __forceinline__ void gu_stage_async(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
+                                               int n_books, const GuSmem& m) {
+  const int tid = threadIdx.x, nb = pl.nb, xs = nb + 1;
   const uint4* x4 = reinterpret_cast<const uint4*>(x);
-  uint4* s_tmp = reinterpret_cast<uint4*>(s_base + L.cb_tmp);
   if (!DENSE) {       // a replicated book is fetched once and copied eight times inside shared memory
-    uint4* dst_g = pl.repl ? s_tmp : s_cb_g;
-    uint4* dst_u = pl.repl ? s_tmp + P.K : s_cb_u;
+    uint4* dst_g = pl.repl ? m.tmp : m.cb_g;
+    uint4* dst_u = pl.repl ? m.tmp + P.K : m.cb_u;
     for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_g + i, P.gate.codebook + i);
     if (n_books == 2)
       for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_u + i, P.up.codebook + i);
@@ -559,34 +571,49 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   if (pl.x_smem)
     for (int i = tid; i < T * nb; i += blockDim.x) {
       const int t = i / nb, b = i - t * nb;
-      cp_async16(s_x + t * xs + b, x4 + i);
+      cp_async16(m.x + t * xs + b, x4 + i);
     }
   cp_async_commit();
-  TRACE_STAMP(0, 1);
-  pdl_wait();      // logits and z of this call are complete
-  TRACE_STAMP(0, 2);
+}
+
+// After logits and z are complete: z as bf16 hi / lo blocks, routing, and the staged bytes landed.
+template <bool DENSE>
+__device__ __forceinline__ void gu_route_and_finish_stage(const Params& P, int T, const StagePlan& pl, int n_books,
+                                                          const GuSmem& m, bool write_global, bool want_dbg) {
+  const int tid = threadIdx.x, rb = (P.r + 7) / 8;
   if (pl.n_lr > 0)
-    for (int i = tid; i < T * 2 * rb; i += blockDim.x) {      // z as bf16 hi / lo blocks
-      const float* zp = P.z + (size_t)i * 8;                   // z is [T][2][r], r a multiple of 8
-      split_hi_lo(__ldcg(reinterpret_cast<const float4*>(zp)), __ldcg(reinterpret_cast<const float4*>(zp + 4)), s_zh[i], s_zl[i]);
+    for (int i = tid; i < T * 2 * rb; i += blockDim.x) {      // z is [T][2][r], r a multiple of 8
+      const float* zp = P.z + (size_t)i * 8;
+      split_hi_lo(__ldcg(reinterpret_cast<const float4*>(zp)), __ldcg(reinterpret_cast<const float4*>(zp + 4)), m.zh[i], m.zl[i]);
     }
-  route_in_block(P, T, R, blockIdx.x == 0, want_dbg != 0);
-  TRACE_STAMP(1, 5);
-  pdl_launch();
+  route_in_block(P, T, m.R, write_global, want_dbg);
   cp_async_wait_pending(0);       // this thread's share of code book and tokens has landed ...
   __syncthreads();                // ... and so has everybody else's
   if (!DENSE && pl.repl) {
     for (int i = tid; i < P.K * 8; i += blockDim.x) {
-      s_cb_g[i] = s_tmp[i >> 3];
-      if (n_books == 2) s_cb_u[i] = s_tmp[P.K + (i >> 3)];
+      m.cb_g[i] = m.tmp[i >> 3];
+      if (n_books == 2) m.cb_u[i] = m.tmp[P.K + (i >> 3)];
     }
     __syncthreads();
   }
-  TRACE_STAMP(0, 3);
+}
 
+// The tile loop of warp `wid` out of `W` warps.
+template <typename IdxT, bool DENSE>
+__device__ __forceinline__ void gu_tiles(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
+                                         const GuSmem& m, int wid, int W) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+  const int nb = pl.nb, xs = nb + 1, D = pl.depth, rb = (P.r + 7) / 8;
+  const uint4* x4 = reinterpret_cast<const uint4*>(x);
+  uint4* s_cb_g = m.cb_g;
+  uint4* s_cb_u = m.cb_u;
+  uint4* s_x = m.x;
+  uint4* ring = m.ring;
+  uint4* s_zh = m.zh;
+  uint4* s_zl = m.zl;
+  const RouteSmem& R = m.R;
   const int n_grp = *R.n_grp, n_pos = T * (P.k + P.S);
   const int V = n_grp * pl.n_parts * pl.tiles;
-  const int W = gridDim.x * nwarps, wid = blockIdx.x * nwarps + warp;
   const int v_begin = split_begin(V, W, wid);
   const int n_my = split_begin(V, W, wid + 1) - v_begin;
   const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
@@ -712,6 +739,24 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   TRACE_STAMP(0, 15);
 }
 
+template <typename IdxT, bool DENSE>
+__global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
+k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {
+  extern __shared__ uint4 s_u4[];
+  const int nwarps = blockDim.x >> 5, warp = threadIdx.x >> 5;
+  const GuLayout L = gu_layout(P.K, n_books, T, P.H, P.r, pl, nwarps, P.E, P.k, P.S);
+  const GuSmem m = gu_carve(reinterpret_cast<char*>(s_u4), L, P, T, warp, threadIdx.x & 31, pl.depth);
+  TRACE_STAMP(0, 0);
+  gu_stage_async<DENSE>(P, x, T, pl, n_books, m);
+  TRACE_STAMP(0, 1);
+  pdl_wait();      // logits and z of this call are complete
+  TRACE_STAMP(0, 2);
+  gu_route_and_finish_stage<DENSE>(P, T, pl, n_books, m, blockIdx.x == 0, want_dbg != 0);
+  pdl_launch();
+  TRACE_STAMP(0, 3);
+  gu_tiles<IdxT, DENSE>(P, x, T, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps);
+}
+
 // ---------------------------------------------------------------------------------------------
 // k_act_zdown: one block per pair.  p = silu(sum of gate parts) * (sum of up parts), kept as
 // bf16 hi + lo for the down kernel's fragments, then z_d = basis_down * p when the down
@@ -721,11 +766,10 @@ constexpr int kActThreads = 384;
 
 // grid = n_pos * zsplit blocks: block (pos, zs) rebuilds p[pos] (cheap, from L2) and computes the
 // z_d rows rho = zs, zs + zsplit, ...; only zs == 0 writes p_hi / p_lo.
-__global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n_pos, int n_parts, int with_zd, int zsplit) {
-  extern __shared__ float s_p[];                 // [I]
-  pdl_launch();                                  // the down kernel may stage its code book meanwhile
-  pdl_wait();
-  const int pos = blockIdx.x / zsplit, zs = blockIdx.x - pos * zsplit, tid = threadIdx.x;
+// One unit = one (pair, z_d row class): the whole block works on it.  s_p: [I] floats.
+__device__ __forceinline__ void act_zdown_unit(const Params& P, int n_pos, int n_parts, int with_zd, int zsplit,
+                                               int unit, float* s_p) {
+  const int pos = unit / zsplit, zs = unit - pos * zsplit, tid = threadIdx.x;
   const size_t part_stride = (size_t)n_pos * P.I;
   for (int i2 = tid; i2 < P.I / 2; i2 += blockDim.x) {
     float g0 = 0.f, g1 = 0.f, u0 = 0.f, u1 = 0.f;
@@ -751,8 +795,8 @@ __global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n
           __floats2bfloat162_rn(p0 - __low2float(hi), p1 - __high2float(hi));
     }
   }
-  if (!with_zd) return;
   __syncthreads();
+  if (!with_zd) return;
   const int lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
   const int nchunk = P.I / 8;
   // two rows of the basis per warp at a time, their loads in flight together
@@ -791,6 +835,13 @@ __global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n
       if (two) P.zd[(size_t)pos * P.r + rho2] = acc1;
     }
   }
+}
+
+__global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n_pos, int n_parts, int with_zd, int zsplit) {
+  extern __shared__ float s_p[];                 // [I]
+  pdl_launch();                                  // the down kernel may stage its code book meanwhile
+  pdl_wait();
+  act_zdown_unit(P, n_pos, n_parts, with_zd, zsplit, blockIdx.x, s_p);
 }
 
 // The same link as two fully parallel kernels, for layers with few pairs or a long intermediate:
@@ -878,44 +929,16 @@ __host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& p
   return L;
 }
 
+// The tile loop of warp `wid` out of `W` warps.  ring: this lane's slot base; s_grp_*: work groups.
 template <typename IdxT, bool DENSE>
-__global__ void __launch_bounds__(kDownThreads, 1)
-k_down_mma(const Params P, int T, const StagePlan pl) {
-  extern __shared__ uint4 s_u4[];
-  char* s_base = reinterpret_cast<char*>(s_u4);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, c = lane & 3;
-  const int nb = pl.nb, D = pl.depth, nwarps = blockDim.x >> 5;
+__device__ __forceinline__ void dn_tiles(const Params& P, int T, const StagePlan& pl, const uint4* s_cb, uint4* ring,
+                                         int slot_u4, const int* s_grp_e, const int* s_grp_off, const int* s_grp_cnt,
+                                         int n_grp, int wid, int W) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+  const int nb = pl.nb, D = pl.depth;
   const int n_pos = T * (P.k + P.S);
-  const DnLayout L = dn_layout(P.K, !DENSE, pl, nwarps, n_pos);
-  uint4* s_cb = s_u4;
-  uint4* ring = reinterpret_cast<uint4*>(s_base + L.ring) + (size_t)warp * D * L.slot_u4 * 32 + lane;   // [slot][chunk][lane]
-  int* s_grp_e = reinterpret_cast<int*>(s_base + L.grp);
-  int* s_grp_off = s_grp_e + n_pos;
-  int* s_grp_cnt = s_grp_off + n_pos;
-  TRACE_STAMP(2, 0);
-  uint4* s_tmp = reinterpret_cast<uint4*>(s_base + L.cb_tmp);
-  if (!DENSE) {
-    uint4* dst = pl.repl ? s_tmp : s_cb;
-    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst + i, P.down.codebook + i);
-  }
-  cp_async_commit();
-  pdl_wait();      // p (and z_d) and the routing lists are complete
-  TRACE_STAMP(2, 1);
-  pdl_launch();
-  const int n_grp = __ldcg(P.grp_n);
-  for (int i = tid; i < n_pos; i += blockDim.x) {      // all n_pos slots (>= n_grp): no dependent second trip
-    s_grp_e[i] = __ldcg(P.grp_e + i); s_grp_off[i] = __ldcg(P.grp_off + i); s_grp_cnt[i] = __ldcg(P.grp_cnt + i);
-  }
-  cp_async_wait_pending(0);
-  __syncthreads();
-  if (!DENSE && pl.repl) {
-    for (int i = tid; i < P.K * 8; i += blockDim.x) s_cb[i] = s_tmp[i >> 3];
-    __syncthreads();
-  }
-  TRACE_STAMP(2, 2);
-
+  struct { int slot_u4; } L = {slot_u4};
   const int V = n_grp * pl.n_parts * pl.tiles;
-  const int W = gridDim.x * nwarps, wid = blockIdx.x * nwarps + warp;
   const int v_begin = split_begin(V, W, wid);
   const int n_my = split_begin(V, W, wid + 1) - v_begin;
   const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
@@ -1027,24 +1050,66 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   TRACE_STAMP(2, 15);
 }
 
+template <typename IdxT, bool DENSE>
+__global__ void __launch_bounds__(kDownThreads, 1)
+k_down_mma(const Params P, int T, const StagePlan pl) {
+  extern __shared__ uint4 s_u4[];
+  char* s_base = reinterpret_cast<char*>(s_u4);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int D = pl.depth, nwarps = blockDim.x >> 5;
+  const int n_pos = T * (P.k + P.S);
+  const DnLayout L = dn_layout(P.K, !DENSE, pl, nwarps, n_pos);
+  uint4* s_cb = s_u4;
+  uint4* ring = reinterpret_cast<uint4*>(s_base + L.ring) + (size_t)warp * D * L.slot_u4 * 32 + lane;   // [slot][chunk][lane]
+  int* s_grp_e = reinterpret_cast<int*>(s_base + L.grp);
+  int* s_grp_off = s_grp_e + n_pos;
+  int* s_grp_cnt = s_grp_off + n_pos;
+  TRACE_STAMP(2, 0);
+  uint4* s_tmp = reinterpret_cast<uint4*>(s_base + L.cb_tmp);
+  if (!DENSE) {
+    uint4* dst = pl.repl ? s_tmp : s_cb;
+    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst + i, P.down.codebook + i);
+  }
+  cp_async_commit();
+  pdl_wait();      // p (and z_d) and the routing lists are complete
+  TRACE_STAMP(2, 1);
+  pdl_launch();
+  const int n_grp = __ldcg(P.grp_n);
+  for (int i = tid; i < n_pos; i += blockDim.x) {      // all n_pos slots (>= n_grp): no dependent second trip
+    s_grp_e[i] = __ldcg(P.grp_e + i); s_grp_off[i] = __ldcg(P.grp_off + i); s_grp_cnt[i] = __ldcg(P.grp_cnt + i);
+  }
+  cp_async_wait_pending(0);
+  __syncthreads();
+  if (!DENSE && pl.repl) {
+    for (int i = tid; i < P.K * 8; i += blockDim.x) s_cb[i] = s_tmp[i >> 3];
+    __syncthreads();
+  }
+  TRACE_STAMP(2, 2);
+  dn_tiles<IdxT, DENSE>(P, T, pl, s_cb, ring, L.slot_u4, s_grp_e, s_grp_off, s_grp_cnt, n_grp,
+                        blockIdx.x * nwarps + warp, gridDim.x * nwarps);
+}
+
 // out[t][h] = sum over slots (in slot order) of affinity * y[t][slot][h], where y is the sum of
 // the down kernel's parts (ascending); shared experts weigh 1.  One block = one token and 64
 // pairs of columns; thread (column pair, slot lane) adds the parts of its slots with all loads
 // in flight, then the slot sums meet in shared memory and are added in slot order.
-constexpr int kCombineCols = 64;    // float2 columns per block
-constexpr int kCombineSlots = 8;    // slot lanes per column
+constexpr int kCombineCols = 64;    // float2 columns per unit
+constexpr int kCombineSlots = 8;    // slot lanes per column in the stand-alone kernel
 
-__global__ void __launch_bounds__(kCombineCols * kCombineSlots)
-k_combine(const Params P, bf16* __restrict__ out, int T, int n_parts) {
-  __shared__ float2 s_y[kMaxK + 8][kCombineCols];       // affinity-weighted y per slot (k + S <= 40)
-  pdl_wait();
-  pdl_launch();
+__device__ __forceinline__ int combine_units(const Params& P, int T) {
+  return T * ((P.H / 2 + kCombineCols - 1) / kCombineCols);
+}
+
+// One unit = one token and 64 pairs of columns; the whole block works on it (blockDim a multiple
+// of 64).  s_y: [k + S][64] float2.
+__device__ __forceinline__ void combine_unit(const Params& P, bf16* __restrict__ out, int T, int n_parts, int unit,
+                                             float2 (*s_y)[kCombineCols]) {
   const int n_slots = P.k + P.S, H2 = P.H / 2, n_pos = T * n_slots;
   const int blocks_per_tok = (H2 + kCombineCols - 1) / kCombineCols;
-  const int t = blockIdx.x / blocks_per_tok, h2 = (blockIdx.x - t * blocks_per_tok) * kCombineCols + (threadIdx.x % kCombineCols);
-  const int sl = threadIdx.x / kCombineCols;
+  const int col = threadIdx.x % kCombineCols, sl = threadIdx.x / kCombineCols, n_sl = blockDim.x / kCombineCols;
+  const int t = unit / blocks_per_tok, h2 = (unit - t * blocks_per_tok) * kCombineCols + col;
   const size_t part_stride = (size_t)n_pos * P.H;
-  for (int s = sl; s < n_slots; s += kCombineSlots) {
+  for (int s = sl; s < n_slots; s += n_sl) {
     const int pos = __ldcg(P.inv_pos + t * n_slots + s);
     const float w = __ldcg(P.pair_w + pos);
     float y0 = 0.f, y1 = 0.f;
@@ -1059,14 +1124,22 @@ k_combine(const Params P, bf16* __restrict__ out, int T, int n_parts) {
         for (int q = 0; q < 4; ++q) { y0 += v[q].x; y1 += v[q].y; }
       }
     }
-    s_y[s][threadIdx.x % kCombineCols] = make_float2(w * y0, w * y1);
+    s_y[s][col] = make_float2(w * y0, w * y1);
   }
   __syncthreads();
   if (sl == 0 && h2 < H2) {
     float a0 = 0.f, a1 = 0.f;
-    for (int s = 0; s < n_slots; ++s) { a0 += s_y[s][threadIdx.x].x; a1 += s_y[s][threadIdx.x].y; }
+    for (int s = 0; s < n_slots; ++s) { a0 += s_y[s][col].x; a1 += s_y[s][col].y; }
     *reinterpret_cast<__nv_bfloat162*>(out + (size_t)t * P.H + 2 * h2) = __floats2bfloat162_rn(a0, a1);
   }
+}
+
+__global__ void __launch_bounds__(kCombineCols * kCombineSlots)
+k_combine(const Params P, bf16* __restrict__ out, int T, int n_parts) {
+  __shared__ float2 s_y[kMaxK + 8][kCombineCols];       // affinity-weighted y per slot (k + S <= 40)
+  pdl_wait();
+  pdl_launch();
+  combine_unit(P, out, T, n_parts, blockIdx.x, s_y);
 }
 
 }  // namespace
