@@ -69,9 +69,18 @@ typedef struct {
 } moe_vqlr_proj;
 
 enum {
-  MOE_VQLR_FLAG_VALIDATE_INDICES = 1u /* create() scans every index map once and fails with
+  MOE_VQLR_FLAG_VALIDATE_INDICES = 1u, /* create() scans every index map once and fails with
                                          BAD_INDEX if a value >= K is found (costs one pass
                                          over the index maps; never done on the decode path) */
+  MOE_VQLR_FLAG_PERSISTENT = 2u       /* decode calls run the whole layer as ONE persistent
+                                         cooperative kernel whose phases are separated by
+                                         grid-wide barriers (every wait bounded: a barrier
+                                         that gives up reports MOE_VQLR_ERR_TIMEOUT through
+                                         the status word) instead of the chain of five
+                                         kernels.  Same results; measured slower than the
+                                         chain on B200, so off by default.  Ignored where the
+                                         configuration cannot use it.  The environment
+                                         variable MOE_VQLR_COOP=1 at create() sets it too. */
 };
 
 typedef struct {
@@ -155,7 +164,9 @@ const char* moe_vqlr_stage_name(int32_t i);
  * on cuda_stream, with the same arguments as moe_vqlr_decode_layer, reading whatever the
  * previous stages of an earlier full call on this handle (same x, same T) left in the
  * workspace.  Lets a benchmark time a single kernel back to back, e.g. inside a captured graph.
- * A stage the configuration does not have enqueues nothing and returns MOE_VQLR_OK. */
+ * A stage the configuration does not have enqueues nothing and returns MOE_VQLR_OK.  Stages
+ * always run as the separate kernels of the chain, also on a handle created with
+ * MOE_VQLR_FLAG_PERSISTENT. */
 int moe_vqlr_run_stage(moe_vqlr_handle* h, int32_t stage, const void* x, int32_t T, void* out,
                        void* cuda_stream);
 

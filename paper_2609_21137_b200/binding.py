@@ -18,6 +18,7 @@ from . import build as _build
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_OOM, ERR_TIMEOUT, ERR_BAD_INDEX = range(7)
 PROJ_VQLR, PROJ_DENSE_BF16 = 0, 1
 FLAG_VALIDATE_INDICES = 1
+FLAG_PERSISTENT = 2
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",

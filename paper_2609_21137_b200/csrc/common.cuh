@@ -61,6 +61,7 @@ struct Params {
   float* ypart;            // [parts][maxT*(k+S)][H]  partial down tiles, by pair position
   int* inv_pos;            // [maxT][k+S]       pair position of (token, slot)
   int* status;             // [1]
+  unsigned int* grid_bar;  // [2] arrivals and generation of the cooperative kernel's grid barrier
   long long* clk;          // optional phase stamps [kernel 4][block][warp 16][stamp 16], or NULL
   int clk_blocks;
 };

@@ -14,6 +14,7 @@
 #include "common.cuh"
 #include "generic_kernels.cuh"
 #include "fast_kernels.cuh"
+#include "coop_kernel.cuh"
 
 #include <cstdlib>
 
@@ -38,10 +39,14 @@ struct moe_vqlr_handle {
   int two_books;
   size_t smem_gateup_per_token, smem_gateup_fixed, smem_down;
   bool fast;                 // tensor-core chain eligible for this configuration
+  bool coop;                 // ... and run as one persistent cooperative kernel
+  int dn_restage;            // the down projection has a code book (or layout) of its own
+  size_t smem_coop;
   int want_dbg;              // the running call asked for counts / offsets
   bool gu_dense, dn_dense;
   int n_books;               // distinct gate/up code books staged by k_gateup_mma
   StagePlan plan_gu, plan_dn;
+  StagePlan plan_gu_coop, plan_dn_coop;   // the same cuts with ring depths chosen for the cooperative kernel
   size_t smem_fast_dn;
   void* workspace;
   size_t workspace_bytes;
@@ -72,6 +77,21 @@ int fail(moe_vqlr_handle* h, int code, const char* fmt, ...) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_coop(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeCooperative;
+  at[0].val.cooperative = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
 
 // Cuts one projection stage into slices and teams for `warps` warps per block.
 StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense) {
@@ -145,12 +165,24 @@ T* carve(char*& cur, size_t n) {
 }
 
 // Enqueues the kernel of one stage (nothing for a stage this configuration does not have).
-cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, bf16* ob, cudaStream_t st) {
+cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, bf16* ob, cudaStream_t st, bool allow_coop) {
   const Params& P = h->P;
   cudaError_t le = cudaSuccess;
   bool ran = false;
   const int n_pos = T * (P.k + P.S);
-  if (h->fast) {
+  if (h->coop && allow_coop) {
+    if (stage == 0) {
+      int zsplit = 1;
+      if (!h->dn_dense && P.r > 0) while (n_pos * zsplit * 2 <= h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
+      const size_t smem = coop_layout(P.K, h->n_books, T, P.H, P.I, P.r, h->plan_gu_coop, h->plan_dn_coop, !h->dn_dense, kCoopThreads / 32, P.E, P.k, P.S).total;
+      // the index type is the gate/up projections' (a dense down projection has no indices)
+      if (h->dn_dense && h->idx_bytes == 1) le = launch_coop(k_layer_coop<uint8_t, true>, h->sm_count, kCoopThreads, smem, st, P, xb, ob, T, h->plan_gu_coop, h->plan_dn_coop, h->n_books, h->want_dbg, h->dn_restage, zsplit);
+      else if (h->dn_dense) le = launch_coop(k_layer_coop<uint16_t, true>, h->sm_count, kCoopThreads, smem, st, P, xb, ob, T, h->plan_gu_coop, h->plan_dn_coop, h->n_books, h->want_dbg, h->dn_restage, zsplit);
+      else if (h->idx_bytes == 1) le = launch_coop(k_layer_coop<uint8_t, false>, h->sm_count, kCoopThreads, smem, st, P, xb, ob, T, h->plan_gu_coop, h->plan_dn_coop, h->n_books, h->want_dbg, h->dn_restage, zsplit);
+      else le = launch_coop(k_layer_coop<uint16_t, false>, h->sm_count, kCoopThreads, smem, st, P, xb, ob, T, h->plan_gu_coop, h->plan_dn_coop, h->n_books, h->want_dbg, h->dn_restage, zsplit);
+      ran = true;
+    }
+  } else if (h->fast) {
     switch (stage) {
       case 0:
         le = launch_pdl(k_router_z_pdl, ((P.E + P.n_zrows) * ((T + kTokGroup - 1) / kTokGroup) + kRouterWarps - 1) / kRouterWarps,
@@ -380,6 +412,41 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     }
   }
 
+  // ---- the same chain as one persistent cooperative kernel --------------------------------------
+  h->coop = false;
+  h->dn_restage = 0;
+  h->smem_coop = 0;
+  {
+    const char* coop_env = getenv("MOE_VQLR_COOP");
+    int coop_attr = 0;
+    cudaDeviceGetAttribute(&coop_attr, cudaDevAttrCooperativeLaunch, h->device);
+    const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) || (coop_env && coop_env[0] == '1');
+    if (h->fast && !h->gu_dense && coop_attr && want_coop) {
+      const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
+      const int warps = kCoopThreads / 32;
+      h->plan_gu_coop = h->plan_gu;
+      h->plan_dn_coop = h->plan_dn;
+      bool fits = false;
+      for (int xs = 1; xs >= 0 && !fits; --xs)
+        for (int d = kMaxDepth; d >= 2 && !fits; --d) {
+          h->plan_gu_coop.x_smem = xs;
+          h->plan_gu_coop.depth = d;
+          h->plan_dn_coop.depth = h->dn_dense ? (d > 3 ? 3 : d) : d;
+          h->smem_coop = coop_layout(K, h->n_books, maxT, H, I, r, h->plan_gu_coop, h->plan_dn_coop, !h->dn_dense, warps, E, k, S).total;
+          fits = h->smem_coop <= limit;
+        }
+      if (fits) {
+        h->dn_restage = (!h->dn_dense && (P.down.codebook != P.gate.codebook || h->plan_dn_coop.repl != h->plan_gu_coop.repl)) ? 1 : 0;
+        const void* fn = h->dn_dense ? (h->idx_bytes == 1 ? (const void*)k_layer_coop<uint8_t, true> : (const void*)k_layer_coop<uint16_t, true>)
+                         : h->idx_bytes == 1 ? (const void*)k_layer_coop<uint8_t, false> : (const void*)k_layer_coop<uint16_t, false>;
+        int per_sm = 0;
+        cudaError_t e1 = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_coop);
+        if (e1 == cudaSuccess) e1 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kCoopThreads, h->smem_coop);
+        if (e1 == cudaSuccess && per_sm >= 1) h->coop = true; else cudaGetLastError();
+      }
+    }
+  }
+
   // workspace
   const char* clk_env = getenv("MOE_VQLR_PHASE_CLOCKS");
   const bool want_clk = clk_env && clk_env[0] == '1';
@@ -412,6 +479,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     P.ypart = carve<float>(cur, h->fast ? (size_t)h->plan_dn.n_parts * n_pos * H : 1);
     P.inv_pos = carve<int>(cur, n_pos);
     P.status = carve<int>(cur, 1);
+    P.grid_bar = carve<unsigned int>(cur, 2);
     if (want_clk) { P.clk = carve<long long>(cur, (size_t)4 * h->sm_count * 16 * 16); P.clk_blocks = h->sm_count; }
     h->x_stage = carve<bf16>(cur, (size_t)maxT * H);
     h->out_stage = carve<bf16>(cur, (size_t)maxT * H);
@@ -475,7 +543,7 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
   for (int i = 0; i < kStages; ++i) h->stage_ran[i] = false;
   for (int stage = 0; stage < kStages; ++stage) {
     if (prof) cudaEventRecord(h->ev[stage], st);
-    const cudaError_t le = launch_stage(h, stage, xb, T, ob, st);
+    const cudaError_t le = launch_stage(h, stage, xb, T, ob, st, true);
     if (le != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "launch of stage %s: %s", kStageNames[stage], cudaGetErrorString(le));
   }
   if (prof) cudaEventRecord(h->ev[kStages], st);
@@ -566,7 +634,7 @@ int moe_vqlr_run_stage(moe_vqlr_handle* h, int32_t stage, const void* x, int32_t
   if (stage < 0 || stage >= kStages || !x || !out || T < 1 || T > h->cfg.max_tokens)
     return fail(h, MOE_VQLR_ERR_INVALID_ARG, "run_stage: bad stage, pointer or T");
   const cudaError_t le = launch_stage(h, stage, static_cast<const bf16*>(x), T, static_cast<bf16*>(out),
-                                      static_cast<cudaStream_t>(cuda_stream));
+                                      static_cast<cudaStream_t>(cuda_stream), false);
   if (le != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "launch of stage %s: %s", kStageNames[stage], cudaGetErrorString(le));
   return MOE_VQLR_OK;
 }

@@ -81,3 +81,24 @@ def test_generic_kernels_forced(shp):
     assert_routing(dbg, res)
     assert_output(bf16_tensor_to_f64(out), res.out)
     mod.close()
+
+
+@pytest.mark.parametrize("shp", [synth.shape("tiny", T=5), synth.shape("tiny", T=2, mode="paper"),
+                                 synth.shape("qwen3", E=16, T=3), synth.shape("qwen3", E=16, T=9, mode="paper"),
+                                 synth.shape("dsv2lite", E=16, T=1)],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
+def test_persistent_kernel(shp):
+    """MOE_VQLR_FLAG_PERSISTENT: the whole layer as one cooperative kernel gives the chain's results,
+    in one launch per call, twice in a row (the grid barrier's state carries over between calls)."""
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_PERSISTENT)
+    x = binding.bits_to_device(layer.x, "cuda")
+    for _ in range(2):
+        before = mod.launch_count
+        out, dbg = mod.decode(x, debug=True)
+        torch.cuda.synchronize()
+        assert mod.launch_count - before == 1
+        assert_routing(dbg, res)
+        assert_output(bf16_tensor_to_f64(out), res.out)
+    mod.close()
