@@ -13,10 +13,10 @@
 namespace {
 
 constexpr int kCoopThreads = 384;
-constexpr long long kGridSyncSpinLimit = 1LL << 21;     // x ~100 ns per poll: gives up after ~0.2 s
+constexpr long long kGridSyncSpinLimit = 1LL << 19;     // x ~0.4 us per poll (an L2 round trip): gives up after ~0.2 s
 
 struct CoopLayout {
-  size_t cb_u, x, ring, z, route, tmp, total;
+  size_t cb_u, x, ring, scratch, z, route, tmp, total;
   int dn_slot_u4;
 };
 
@@ -30,12 +30,12 @@ __host__ __device__ inline CoopLayout coop_layout(int K, int n_books, int T, int
   size_t o = coop_max((size_t)n_books * gu_book, dn_book);
   L.x = o;      o += pg.x_smem ? (size_t)T * (H / 8 + 1) * 16 : 0;
   L.dn_slot_u4 = dn_vq ? 2 : 8;
-  // one region serves, in turn: gate/up ring, p of one pair, down ring, the combine's slot sums
+  // the ring serves the gate/up walk, then the down walk (whose first units are requested while
+  // the activation phase still runs, hence a scratch region of its own for that phase and the combine)
   size_t region = (size_t)warps * pg.depth * 2 * 32 * 16;
   region = coop_max(region, (size_t)warps * pd.depth * L.dn_slot_u4 * 32 * 16);
-  region = coop_max(region, (size_t)I * 4);
-  region = coop_max(region, (size_t)(kMaxK + 8) * kCombineCols * 8);
   L.ring = o;   o += region;
+  L.scratch = o; o += coop_max((size_t)I * 4, (size_t)(kMaxK + 8) * kCombineCols * 8);
   L.z = o;      o += (size_t)2 * T * 2 * ((r + 7) / 8) * 16;
   L.route = o;  o += route_smem_bytes(T, E, k, S);
   L.tmp = o;    o += (pg.repl || pd.repl) ? (size_t)2 * K * 16 : 0;
@@ -49,27 +49,25 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
   return v;
 }
 
-// bar[0] = arrivals of the current barrier, bar[1] = generation.  Returns false after a timeout.
-__device__ __forceinline__ bool grid_sync(unsigned int* bar, int* status) {
+// bar[0] counts arrivals and is never reset: every launch adds kCoopBarriers * gridDim.x to it.
+// bar[1] is the number of completed launches (mod 2^32); a block reads it once at its start and
+// derives the counter value that completes each barrier, so that a barrier is one fire-and-forget
+// reduction plus polling loads -- no read-modify-write on the critical path and no reset.
+// Block 0 advances bar[1] after the last barrier.  Returns false after a timeout; the counters
+// are then out of step and the handle must not be used for further persistent launches.
+constexpr unsigned int kCoopBarriers = 4;
+
+__device__ __forceinline__ bool grid_sync(unsigned int* bar, unsigned int target, int* status) {
   __shared__ int s_ok;
   __syncthreads();
   if (threadIdx.x == 0) {
     bool ok = true;
-    const unsigned int gen0 = ld_acquire_u32(bar + 1);
     __threadfence();
-    const unsigned int old = atomicAdd(bar, 1u);
-    if (old == gridDim.x - 1) {
-      atomicExch(bar, 0u);
-      __threadfence();
-      atomicAdd(bar + 1, 1u);
-    } else {
-      long long spins = 0;
-      while (ld_acquire_u32(bar + 1) == gen0) {
-        if (++spins > kGridSyncSpinLimit) { ok = false; atomicExch(status, MOE_VQLR_ERR_TIMEOUT); break; }
-        __nanosleep(64);
-      }
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
+    long long spins = 0;
+    while ((int)(ld_acquire_u32(bar) - target) < 0) {
+      if (++spins > kGridSyncSpinLimit) { ok = false; atomicExch(status, MOE_VQLR_ERR_TIMEOUT); break; }
     }
-    __threadfence();
     s_ok = ok ? 1 : 0;
   }
   __syncthreads();
@@ -98,41 +96,72 @@ k_layer_coop(const Params P, const bf16* __restrict__ x, bf16* __restrict__ out,
     m.R = carve_route(s_base + L.route, T, P.E, P.k, P.S);
   }
   unsigned int* bar = P.grid_bar;
+  // every thread derives the barrier targets from the launch count (read before this block's first arrival)
+  const unsigned int bar_epoch = __ldcg(bar + 1);
+  const unsigned int bar_base = bar_epoch * kCoopBarriers * gridDim.x;
   const int n_pos = T * (P.k + P.S);
 
   // ---- phase A: router logits and shared projections; code books and tokens stream in meanwhile
   TRACE_STAMP(3, 0);
-  gu_stage_async<false>(P, x, T, pg, n_books, m);
-  for (int unit = wid; unit < router_z_units(P, T); unit += W) router_z_unit(P, x, T, unit, lane);
+  {
+    // rows are dealt round-robin over the blocks first, so that every SM streams a few of them
+    const int n_units = router_z_units(P, T), unit0 = warp * gridDim.x + blockIdx.x;
+    gu_stage_tokens_async(x, T, pg, m);
+    RouterRow u;
+    uint4 wv[8];
+    const bool staged = pg.x_smem && unit0 < n_units;
+    if (staged) {                                    // weight row and tokens travel together
+      u = router_z_row(P, T, unit0);
+      router_z_load8(u, 0, P.H / 8, lane, wv);
+    }
+    gu_stage_books_async<false>(P, pg, n_books, m);  // lands while the block waits at the barrier
+    cp_async_wait_pending(1);
+    __syncthreads();                                 // tokens are in shared memory
+    if (staged) router_z_finish(P, u, m.x, pg.nb + 1, lane, wv);
+    for (int unit = staged ? unit0 + W : unit0; unit < n_units; unit += W) router_z_unit(P, x, T, unit, lane);
+  }
   TRACE_STAMP(3, 1);
-  if (!grid_sync(bar, P.status)) return;
+  if (!grid_sync(bar, bar_base + 1u * gridDim.x, P.status)) return;
   TRACE_STAMP(3, 2);
 
   // ---- phase B: routing (every block), gate/up partial tiles
-  gu_route_and_finish_stage<false>(P, T, pg, n_books, m, blockIdx.x == 0, want_dbg != 0);
-  TRACE_STAMP(3, 3);
-  gu_tiles<IdxT, false>(P, x, T, pg, m, wid, W);
+  {
+    gu_route(P, T, pg, m, blockIdx.x == 0, want_dbg != 0);
+    Walk w;
+    gu_tiles_begin<IdxT, false>(P, pg, m, wid, W, w);
+    gu_finish_stage<false>(P, pg, n_books, m, pg.depth - 1);      // the code books landed long ago
+    TRACE_STAMP(3, 3);
+    gu_tiles_run<IdxT, false>(P, x, T, pg, m, w);
+  }
   TRACE_STAMP(3, 4);
-  if (!grid_sync(bar, P.status)) return;
+  if (!grid_sync(bar, bar_base + 2u * gridDim.x, P.status)) return;
   TRACE_STAMP(3, 5);
 
-  // ---- phase C: sum of parts, SwiGLU, z_d; a down code book of its own streams in meanwhile
+  // ---- phase C: sum of parts, SwiGLU, z_d; meanwhile a down code book of its own streams in
+  // and so do the first index / weight bytes of this warp's down units
   if (!DN_DENSE && dn_restage) {
     uint4* dst = pd.repl ? m.tmp : m.cb_g;
     for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst + i, P.down.codebook + i);
   }
   cp_async_commit();
+  DnSmem dm;
+  dm.cb = m.cb_g;
+  dm.ring = reinterpret_cast<uint4*>(s_base + L.ring) + (size_t)warp * pd.depth * L.dn_slot_u4 * 32 + lane;
+  dm.slot_u4 = L.dn_slot_u4;
+  dm.grp_e = m.R.grp_e; dm.grp_off = m.R.grp_off; dm.grp_cnt = m.R.grp_cnt; dm.n_grp = *m.R.n_grp;
+  Walk dw;
+  dn_tiles_begin<IdxT, DN_DENSE>(P, pd, dm, wid, W, dw);
   {
-    float* s_p = reinterpret_cast<float*>(s_base + L.ring);
+    float* s_p = reinterpret_cast<float*>(s_base + L.scratch);
     const int with_zd = (!DN_DENSE && P.r > 0) ? 1 : 0;
     for (int unit = blockIdx.x; unit < n_pos * zsplit; unit += gridDim.x) {
       act_zdown_unit(P, n_pos, pg.n_parts, with_zd, zsplit, unit, s_p);
       __syncthreads();
     }
   }
-  cp_async_wait_pending(0);
+  cp_async_wait_pending(pd.depth - 1);      // the code book (the walk's groups may still travel)
   TRACE_STAMP(3, 6);
-  if (!grid_sync(bar, P.status)) return;
+  if (!grid_sync(bar, bar_base + 3u * gridDim.x, P.status)) return;
   TRACE_STAMP(3, 7);
   if (!DN_DENSE && dn_restage && pd.repl) {
     for (int i = tid; i < P.K * 8; i += blockDim.x) m.cb_g[i] = m.tmp[i >> 3];
@@ -140,17 +169,15 @@ k_layer_coop(const Params P, const bf16* __restrict__ x, bf16* __restrict__ out,
   }
 
   // ---- phase D: down partial tiles (work groups are still in shared memory)
-  {
-    uint4* ring = reinterpret_cast<uint4*>(s_base + L.ring) + (size_t)warp * pd.depth * L.dn_slot_u4 * 32 + lane;
-    dn_tiles<IdxT, DN_DENSE>(P, T, pd, m.cb_g, ring, L.dn_slot_u4, m.R.grp_e, m.R.grp_off, m.R.grp_cnt, *m.R.n_grp, wid, W);
-  }
+  dn_tiles_run<IdxT, DN_DENSE>(P, T, pd, dm, dw);
   TRACE_STAMP(3, 8);
-  if (!grid_sync(bar, P.status)) return;
+  if (!grid_sync(bar, bar_base + 4u * gridDim.x, P.status)) return;
   TRACE_STAMP(3, 9);
+  if (blockIdx.x == 0 && tid == 0) bar[1] = bar_epoch + 1u;   // this launch is past its last barrier
 
   // ---- phase E: weighted sum
   {
-    float2 (*s_y)[kCombineCols] = reinterpret_cast<float2 (*)[kCombineCols]>(s_base + L.ring);
+    float2 (*s_y)[kCombineCols] = reinterpret_cast<float2 (*)[kCombineCols]>(s_base + L.scratch);
     for (int unit = blockIdx.x; unit < combine_units(P, T); unit += gridDim.x) {
       combine_unit(P, out, T, pd.n_parts, unit, s_y);
       __syncthreads();

@@ -140,7 +140,28 @@ __device__ __forceinline__ uint4 ring_idx8(const uint4* smem) {
   return make_uint4(v.x, v.y, 0u, 0u);
 }
 
-// How one projection stage is cut up (computed on the host, see plan_stage()).
+// Division by a run-time constant as multiply-high and shift (the magic numbers come from the
+// host): exact for 0 <= n < 2^31.  A hardware-emulated 32-bit division costs about a hundred
+// clocks of dependent instructions, and the work-list arithmetic below sits on the critical path
+// of a warp that has nothing else to overlap it with.
+struct FastDiv {
+  unsigned int mul, shr;      // mul == 0: divisor 1
+};
+__host__ inline FastDiv make_fastdiv(unsigned int d) {
+  FastDiv f = {0u, 0u};
+  if (d <= 1u) return f;
+  unsigned int L = 0;
+  while ((1ull << L) < d) ++L;
+  const unsigned int p = 31u + L;
+  f.mul = (unsigned int)(((1ull << p) + d - 1ull) / d);
+  f.shr = p - 32u;
+  return f;
+}
+__device__ __forceinline__ int fdiv(int n, const FastDiv& f) {
+  return f.mul ? (int)(__umulhi((unsigned int)n, f.mul) >> f.shr) : n;
+}
+
+// How one projection stage is cut up (computed on the host, see plan_stage() / finish_plan()).
 struct StagePlan {
   int nb;          // blocks per weight row = in_dim / 8
   int n_slices;    // ceil(nb / 32)
@@ -152,6 +173,9 @@ struct StagePlan {
   int x_smem;      // gate/up: tokens are staged in shared memory (else fragments come from global)
   int repl;        // code book stored eight times, entry i of copy c at slot 8 i + c: lane l reads
                    // copy l % 8, so the eight lanes of a quarter warp never share a bank group
+  int W;           // warps of the launch that walks this plan (grid * warps per block)
+  int tail;        // tiles % chunk: length of a shorter last chunk (0: none)
+  FastDiv d_per_grp, d_per_chunk, d_chunk, d_tail, d_W;   // n_parts*tiles, n_parts*chunk, chunk, tail, W
 };
 
 // Position in the flattened work list of a stage.  Units are ordered (group, chunk of `chunk`
@@ -162,20 +186,20 @@ struct Cursor {
   int grp, part, jt, chunk_end;       // jt = absolute tile, chunk_end = first tile after its chunk
   __device__ __forceinline__ void set(int v, const StagePlan& pl) {
     const int per_grp = pl.n_parts * pl.tiles;
-    grp = v / per_grp;
+    grp = fdiv(v, pl.d_per_grp);
     int rem = v - grp * per_grp;
     const int per_chunk = pl.n_parts * pl.chunk;
-    const int ch = rem / per_chunk;                 // the last chunk may be shorter
+    const int ch = fdiv(rem, pl.d_per_chunk);       // the last chunk may be shorter
     rem -= ch * per_chunk;
     const int c0 = ch * pl.chunk;
     const int clen = min(pl.chunk, pl.tiles - c0);
-    part = rem / clen;
+    part = clen == pl.chunk ? fdiv(rem, pl.d_chunk) : fdiv(rem, pl.d_tail);
     jt = c0 + (rem - part * clen);
     chunk_end = c0 + clen;
   }
   __device__ __forceinline__ void next(const StagePlan& pl) {
     if (++jt == chunk_end) {
-      const int c0 = chunk_end - min(pl.chunk, chunk_end - ((chunk_end - 1) / pl.chunk) * pl.chunk);
+      const int c0 = chunk_end - min(pl.chunk, chunk_end - fdiv(chunk_end - 1, pl.d_chunk) * pl.chunk);
       if (++part == pl.n_parts) {
         part = 0;
         if (chunk_end == pl.tiles) { ++grp; jt = 0; chunk_end = min(pl.chunk, pl.tiles); }
@@ -496,6 +520,77 @@ __device__ __forceinline__ void router_z_unit(const Params& P, const bf16* __res
   }
 }
 
+// The same unit in two steps for a persistent kernel: the weight row (first 8 chunks per lane)
+// is requested into registers BEFORE the block waits for the tokens to land in shared memory,
+// so that both round trips overlap; summation order as in router_z_unit.
+struct RouterRow {
+  const uint4* w4;
+  float* dst;
+  int dst_stride, t0, nt;
+  float bias;
+};
+
+__device__ __forceinline__ RouterRow router_z_row(const Params& P, int T, int unit) {
+  const int n_groups = (T + kTokGroup - 1) / kTokGroup;
+  const int row = unit / n_groups;
+  RouterRow u;
+  u.t0 = (unit - row * n_groups) * kTokGroup;
+  u.nt = min(kTokGroup, T - u.t0);
+  u.bias = 0.f;
+  if (row < P.E) {
+    u.w4 = reinterpret_cast<const uint4*>(P.router_w + (size_t)row * P.H);
+    u.dst = P.logits + row;
+    u.dst_stride = P.E;
+    if (P.router_bias) u.bias = P.router_bias[row];
+  } else {
+    const int q = row - P.E;
+    const int slot = q / P.r, rho = q - slot * P.r;
+    const bf16* basis = (slot == P.gate.zslot && P.gate.basis) ? P.gate.basis : P.up.basis;
+    u.w4 = reinterpret_cast<const uint4*>(basis + (size_t)rho * P.H);
+    u.dst = P.z + slot * P.r + rho;
+    u.dst_stride = 2 * P.r;
+  }
+  return u;
+}
+
+__device__ __forceinline__ void router_z_load8(const RouterRow& u, int c0, int nchunk, int lane, uint4 (&wv)[8]) {
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const int c = c0 + q * 32 + lane;
+    wv[q] = c < nchunk ? __ldg(u.w4 + c) : make_uint4(0, 0, 0, 0);
+  }
+}
+
+// s_x: tokens in shared memory, row stride xs blocks.  wv: chunks 0..255 of the row, already requested.
+__device__ __forceinline__ void router_z_finish(const Params& P, const RouterRow& u, const uint4* s_x, int xs, int lane, uint4 (&wv)[8]) {
+  const int nchunk = P.H / 8;
+  float acc[kTokGroup] = {0.f, 0.f, 0.f, 0.f};
+  for (int c0 = 0; c0 < nchunk; c0 += 32 * 8) {
+    if (c0 > 0) router_z_load8(u, c0, nchunk, lane, wv);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int c = c0 + q * 32 + lane;
+      if (c < nchunk) {
+        float wf[8];
+        unpack8(wv[q], wf);
+#pragma unroll
+        for (int tt = 0; tt < kTokGroup; ++tt) {
+          if (tt < u.nt) {
+            float xf[8];
+            unpack8(s_x[(u.t0 + tt) * xs + c], xf);
+            acc[tt] = dot8(wf, xf, acc[tt]);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int tt = 0; tt < kTokGroup; ++tt) {
+    const float sum = warp_sum(acc[tt]);
+    if (lane == 0 && tt < u.nt) u.dst[(size_t)(u.t0 + tt) * u.dst_stride] = sum + u.bias;
+  }
+}
+
 __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
   pdl_wait();      // the previous call's kernels may still read logits / z
   pdl_launch();
@@ -508,6 +603,12 @@ __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params
 __device__ __forceinline__ int split_begin(int total, int parts, int idx) {
   const unsigned int q = (unsigned int)total / (unsigned int)parts, rem = (unsigned int)total - q * (unsigned int)parts;
   return (int)(q * (unsigned int)idx + (rem * (unsigned int)idx) / (unsigned int)parts);
+}
+
+// The same with the plan's warp count and its magic number (total, idx < 2^15 or so: rem * idx < 2^31).
+__device__ __forceinline__ int split_begin(int total, const StagePlan& pl, int idx) {
+  const int q = fdiv(total, pl.d_W), rem = total - q * pl.W;
+  return q * idx + fdiv(rem * idx, pl.d_W);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -556,18 +657,10 @@ __device__ __forceinline__ GuSmem gu_carve(char* s_base, const GuLayout& L, cons
 
 // Routing-independent prologue: code books and tokens start streaming into shared memory
 // (one cp.async group per thread, not yet waited for).
-template <bool DENSE>
-__device__ __forceinline__ void gu_stage_async(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
-                                               int n_books, const GuSmem& m) {
+// Requests the tokens (one cp.async group) ...
+__device__ __forceinline__ void gu_stage_tokens_async(const bf16* __restrict__ x, int T, const StagePlan& pl, const GuSmem& m) {
   const int tid = threadIdx.x, nb = pl.nb, xs = nb + 1;
   const uint4* x4 = reinterpret_cast<const uint4*>(x);
-  if (!DENSE) {       // a replicated book is fetched once and copied eight times inside shared memory
-    uint4* dst_g = pl.repl ? m.tmp : m.cb_g;
-    uint4* dst_u = pl.repl ? m.tmp + P.K : m.cb_u;
-    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_g + i, P.gate.codebook + i);
-    if (n_books == 2)
-      for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_u + i, P.up.codebook + i);
-  }
   if (pl.x_smem)
     for (int i = tid; i < T * nb; i += blockDim.x) {
       const int t = i / nb, b = i - t * nb;
@@ -576,19 +669,63 @@ __device__ __forceinline__ void gu_stage_async(const Params& P, const bf16* __re
   cp_async_commit();
 }
 
-// After logits and z are complete: z as bf16 hi / lo blocks, routing, and the staged bytes landed.
+// ... and the code books (a second group).  A replicated book is fetched once and copied eight
+// times inside shared memory later.
 template <bool DENSE>
-__device__ __forceinline__ void gu_route_and_finish_stage(const Params& P, int T, const StagePlan& pl, int n_books,
-                                                          const GuSmem& m, bool write_global, bool want_dbg) {
+__device__ __forceinline__ void gu_stage_books_async(const Params& P, const StagePlan& pl, int n_books, const GuSmem& m) {
+  const int tid = threadIdx.x;
+  if (!DENSE) {
+    uint4* dst_g = pl.repl ? m.tmp : m.cb_g;
+    uint4* dst_u = pl.repl ? m.tmp + P.K : m.cb_u;
+    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_g + i, P.gate.codebook + i);
+    if (n_books == 2)
+      for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_u + i, P.up.codebook + i);
+  }
+  cp_async_commit();
+}
+
+template <bool DENSE>
+__device__ __forceinline__ void gu_stage_async(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
+                                               int n_books, const GuSmem& m) {
+  gu_stage_tokens_async(x, T, pl, m);
+  gu_stage_books_async<DENSE>(P, pl, n_books, m);
+}
+
+// After logits and z are complete: z as bf16 hi / lo blocks, routing, and the staged bytes landed.
+__device__ __forceinline__ void gu_route(const Params& P, int T, const StagePlan& pl, const GuSmem& m,
+                                         bool write_global, bool want_dbg) {
   const int tid = threadIdx.x, rb = (P.r + 7) / 8;
-  if (pl.n_lr > 0)
-    for (int i = tid; i < T * 2 * rb; i += blockDim.x) {      // z is [T][2][r], r a multiple of 8
+  float4 zv[2][2];                 // this thread's z values travel while the routing runs (up to two blocks of 8 each)
+  const int nz = pl.n_lr > 0 ? T * 2 * rb : 0;
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int i = tid + q * blockDim.x;
+    if (i < nz) {
       const float* zp = P.z + (size_t)i * 8;
-      split_hi_lo(__ldcg(reinterpret_cast<const float4*>(zp)), __ldcg(reinterpret_cast<const float4*>(zp + 4)), m.zh[i], m.zl[i]);
+      zv[q][0] = __ldcg(reinterpret_cast<const float4*>(zp));
+      zv[q][1] = __ldcg(reinterpret_cast<const float4*>(zp + 4));
     }
+  }
   route_in_block(P, T, m.R, write_global, want_dbg);
-  cp_async_wait_pending(0);       // this thread's share of code book and tokens has landed ...
-  __syncthreads();                // ... and so has everybody else's
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int i = tid + q * blockDim.x;
+    if (i < nz) split_hi_lo(zv[q][0], zv[q][1], m.zh[i], m.zl[i]);
+  }
+  for (int i = tid + 2 * blockDim.x; i < nz; i += blockDim.x) {      // z is [T][2][r], r a multiple of 8
+    const float* zp = P.z + (size_t)i * 8;
+    split_hi_lo(__ldcg(reinterpret_cast<const float4*>(zp)), __ldcg(reinterpret_cast<const float4*>(zp + 4)), m.zh[i], m.zl[i]);
+  }
+  TRACE_STAMP(1, 5);
+}
+
+// The staged bytes have landed (the `newer` most recent cp.async groups may still be in flight).
+template <bool DENSE>
+__device__ __forceinline__ void gu_finish_stage(const Params& P, const StagePlan& pl, int n_books, const GuSmem& m, int newer) {
+  const int tid = threadIdx.x;
+  cp_async_wait_pending(newer);   // this thread's share of code book and tokens has landed ...
+  __syncthreads();                // ... and so has everybody else's (and z, and the routing lists)
+  TRACE_STAMP(1, 6);
   if (!DENSE && pl.repl) {
     for (int i = tid; i < P.K * 8; i += blockDim.x) {
       m.cb_g[i] = m.tmp[i >> 3];
@@ -598,10 +735,58 @@ __device__ __forceinline__ void gu_route_and_finish_stage(const Params& P, int T
   }
 }
 
-// The tile loop of warp `wid` out of `W` warps.
+// A warp's walk over its contiguous range of the work list: the prefetch cursor runs depth - 1
+// units ahead of the compute cursor through the warp's ring.
+struct Walk {
+  Cursor pf, cur;
+  int pf_slot, cur_slot, n_my;
+};
+
+// Streams the bytes of the prefetch cursor's unit into the ring and advances that cursor.
 template <typename IdxT, bool DENSE>
-__device__ __forceinline__ void gu_tiles(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
-                                         const GuSmem& m, int wid, int W) {
+__device__ __forceinline__ void gu_issue(const Params& P, const StagePlan& pl, const GuSmem& m, Walk& w) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3, nb = pl.nb;
+  uint4* ring = m.ring;
+  if (!DENSE) {
+    const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
+    const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx);
+    const size_t row = (size_t)m.R.grp_e[w.pf.grp] * P.I + w.pf.jt * 8 + g;
+    if (w.pf.part < pl.n_slices) {
+      const int b = w.pf.part * 32 + 8 * c;
+      if (b < nb) {
+        cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_g + row * nb + b);
+        cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 1) * 32, idx_u + row * nb + b);
+      }
+    } else {
+      const int rho = (w.pf.part - pl.n_slices) * 32 + 8 * c;
+      if (rho < P.r) {
+        cp_async16(ring + (w.pf_slot * 2 + 0) * 32, P.gate.factor + row * P.r + rho);
+        cp_async16(ring + (w.pf_slot * 2 + 1) * 32, P.up.factor + row * P.r + rho);
+      }
+    }
+  }
+  w.pf.next(pl);
+  if (++w.pf_slot == pl.depth) w.pf_slot = 0;
+}
+
+// Start of the walk of warp `wid` out of `W` warps (needs the work groups): depth - 1 units are
+// requested, each as one cp.async group.
+template <typename IdxT, bool DENSE>
+__device__ __forceinline__ void gu_tiles_begin(const Params& P, const StagePlan& pl, const GuSmem& m, int wid, int W, Walk& w) {
+  const int V = *m.R.n_grp * pl.n_parts * pl.tiles;
+  const int v_begin = split_begin(V, pl, wid);         // W == pl.W by construction of the launch
+  w.n_my = split_begin(V, pl, wid + 1) - v_begin;
+  w.pf.set(w.n_my > 0 ? v_begin : 0, pl);
+  w.cur = w.pf;
+  w.pf_slot = 0; w.cur_slot = 0;
+  for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) gu_issue<IdxT, DENSE>(P, pl, m, w); cp_async_commit(); }
+  TRACE_STAMP(1, 7);
+}
+
+// The tile loop proper (needs code books, tokens and z in shared memory).
+template <typename IdxT, bool DENSE>
+__device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
+                                             const GuSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
   const int nb = pl.nb, xs = nb + 1, D = pl.depth, rb = (P.r + 7) / 8;
   const uint4* x4 = reinterpret_cast<const uint4*>(x);
@@ -612,43 +797,14 @@ __device__ __forceinline__ void gu_tiles(const Params& P, const bf16* __restrict
   uint4* s_zh = m.zh;
   uint4* s_zl = m.zl;
   const RouteSmem& R = m.R;
-  const int n_grp = *R.n_grp, n_pos = T * (P.k + P.S);
-  const int V = n_grp * pl.n_parts * pl.tiles;
-  const int v_begin = split_begin(V, W, wid);
-  const int n_my = split_begin(V, W, wid + 1) - v_begin;
-  const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
-  const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx);
-
-  Cursor pf, cur;
-  pf.set(n_my > 0 ? v_begin : 0, pl);
-  cur = pf;
-  int pf_slot = 0, cur_slot = 0;
-  auto issue = [&]() {          // stream the bytes of the prefetch cursor's tile into the ring
-    if (!DENSE) {
-      const size_t row = (size_t)R.grp_e[pf.grp] * P.I + pf.jt * 8 + g;
-      if (pf.part < pl.n_slices) {
-        const int b = pf.part * 32 + 8 * c;
-        if (b < nb) {
-          cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 0) * 32, idx_g + row * nb + b);
-          cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 1) * 32, idx_u + row * nb + b);
-        }
-      } else {
-        const int rho = (pf.part - pl.n_slices) * 32 + 8 * c;
-        if (rho < P.r) {
-          cp_async16(ring + (pf_slot * 2 + 0) * 32, P.gate.factor + row * P.r + rho);
-          cp_async16(ring + (pf_slot * 2 + 1) * 32, P.up.factor + row * P.r + rho);
-        }
-      }
-    }
-    pf.next(pl);
-    if (++pf_slot == D) pf_slot = 0;
-  };
+  const int n_pos = T * (P.k + P.S), n_my = w.n_my;
+  Cursor& cur = w.cur;
+  int& cur_slot = w.cur_slot;
+  auto issue = [&]() { gu_issue<IdxT, DENSE>(P, pl, m, w); };
 
   uint4 fx[8];                       // activation fragments of the current (group, part)
   int frag_grp = -1, frag_part = -1;
 
-  for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(); cp_async_commit(); }
-  TRACE_STAMP(1, 7);
   for (int i = 0; i < n_my; ++i) {
     if (i + D - 1 < n_my) issue();
     cp_async_commit();
@@ -751,10 +907,13 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   TRACE_STAMP(0, 1);
   pdl_wait();      // logits and z of this call are complete
   TRACE_STAMP(0, 2);
-  gu_route_and_finish_stage<DENSE>(P, T, pl, n_books, m, blockIdx.x == 0, want_dbg != 0);
+  gu_route(P, T, pl, m, blockIdx.x == 0, want_dbg != 0);
+  Walk w;
+  gu_tiles_begin<IdxT, DENSE>(P, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps, w);   // index bytes travel ...
+  gu_finish_stage<DENSE>(P, pl, n_books, m, pl.depth - 1);                                     // ... while the stage settles
   pdl_launch();
   TRACE_STAMP(0, 3);
-  gu_tiles<IdxT, DENSE>(P, x, T, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps);
+  gu_tiles_run<IdxT, DENSE>(P, x, T, pl, m, w);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -929,46 +1088,68 @@ __host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& p
   return L;
 }
 
-// The tile loop of warp `wid` out of `W` warps.  ring: this lane's slot base; s_grp_*: work groups.
+// Shared-memory views of the down stage.  ring: this lane's slot base; grp_*: work groups.
+struct DnSmem {
+  const uint4* cb;
+  uint4* ring;
+  int slot_u4;
+  const int *grp_e, *grp_off, *grp_cnt;
+  int n_grp;
+};
+
+// Streams the bytes of the prefetch cursor's unit into the ring and advances that cursor.
 template <typename IdxT, bool DENSE>
-__device__ __forceinline__ void dn_tiles(const Params& P, int T, const StagePlan& pl, const uint4* s_cb, uint4* ring,
-                                         int slot_u4, const int* s_grp_e, const int* s_grp_off, const int* s_grp_cnt,
-                                         int n_grp, int wid, int W) {
+__device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, const DnSmem& m, Walk& w) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3, nb = pl.nb;
+  uint4* ring = m.ring;
+  const Cursor& pf = w.pf;
+  const size_t row = (size_t)m.grp_e[pf.grp] * P.H + pf.jt * 8 + g;
+  if (DENSE) {
+    const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I) + pf.part * 32 + c;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (pf.part * 32 + c + 4 * j < nb) cp_async16(ring + (w.pf_slot * 8 + j) * 32, wd + 4 * j);
+  } else {
+    const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
+    const int b = pf.part * 32 + 8 * c, rho = pf.part * 32 + 8 * c;
+    if (b < nb) cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_d + row * nb + b);
+    if (pf.part < pl.n_lr && rho < P.r) cp_async16(ring + (w.pf_slot * 2 + 1) * 32, P.down.factor + row * P.r + rho);
+  }
+  w.pf.next(pl);
+  if (++w.pf_slot == pl.depth) w.pf_slot = 0;
+}
+
+// Start of the walk of warp `wid` out of `W` warps (needs only the work groups, not p).
+template <typename IdxT, bool DENSE>
+__device__ __forceinline__ void dn_tiles_begin(const Params& P, const StagePlan& pl, const DnSmem& m, int wid, int W, Walk& w) {
+  const int V = m.n_grp * pl.n_parts * pl.tiles;
+  const int v_begin = split_begin(V, pl, wid);         // W == pl.W by construction of the launch
+  w.n_my = split_begin(V, pl, wid + 1) - v_begin;
+  w.pf.set(w.n_my > 0 ? v_begin : 0, pl);
+  w.cur = w.pf;
+  w.pf_slot = 0; w.cur_slot = 0;
+  for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) dn_issue<IdxT, DENSE>(P, pl, m, w); cp_async_commit(); }
+  TRACE_STAMP(2, 3);
+}
+
+// The tile loop proper (needs p, z_d and the code book).
+template <typename IdxT, bool DENSE>
+__device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const StagePlan& pl, const DnSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
   const int nb = pl.nb, D = pl.depth;
-  const int n_pos = T * (P.k + P.S);
-  struct { int slot_u4; } L = {slot_u4};
-  const int V = n_grp * pl.n_parts * pl.tiles;
-  const int v_begin = split_begin(V, W, wid);
-  const int n_my = split_begin(V, W, wid + 1) - v_begin;
-  const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
-
-  Cursor pf, cur;
-  pf.set(n_my > 0 ? v_begin : 0, pl);
-  cur = pf;
-  int pf_slot = 0, cur_slot = 0;
-  auto issue = [&]() {
-    const size_t row = (size_t)s_grp_e[pf.grp] * P.H + pf.jt * 8 + g;
-    if (DENSE) {
-      const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I) + pf.part * 32 + c;
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (pf.part * 32 + c + 4 * j < nb) cp_async16(ring + (pf_slot * 8 + j) * 32, wd + 4 * j);
-    } else {
-      const int b = pf.part * 32 + 8 * c, rho = pf.part * 32 + 8 * c;
-      if (b < nb) cp_async_idx8<IdxT>(ring + (pf_slot * 2 + 0) * 32, idx_d + row * nb + b);
-      if (pf.part < pl.n_lr && rho < P.r) cp_async16(ring + (pf_slot * 2 + 1) * 32, P.down.factor + row * P.r + rho);
-    }
-    pf.next(pl);
-    if (++pf_slot == D) pf_slot = 0;
-  };
+  const int n_pos = T * (P.k + P.S), n_my = w.n_my;
+  struct { int slot_u4; } L = {m.slot_u4};
+  const uint4* s_cb = m.cb;
+  uint4* ring = m.ring;
+  const int *s_grp_e = m.grp_e, *s_grp_off = m.grp_off, *s_grp_cnt = m.grp_cnt;
+  Cursor& cur = w.cur;
+  int& cur_slot = w.cur_slot;
+  auto issue = [&]() { dn_issue<IdxT, DENSE>(P, pl, m, w); };
 
   uint4 fh[8], fl[8];
   uint4 zh = {0, 0, 0, 0}, zl = {0, 0, 0, 0};     // z_d fragments of the low-rank group this part carries
   int frag_grp = -1, frag_part = -1;
 
-  for (int i = 0; i < D - 1; ++i) { if (i < n_my) issue(); cp_async_commit(); }
-  TRACE_STAMP(2, 3);
   for (int i = 0; i < n_my; ++i) {
     if (i + D - 1 < n_my) issue();
     cp_async_commit();
@@ -1078,15 +1259,20 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   for (int i = tid; i < n_pos; i += blockDim.x) {      // all n_pos slots (>= n_grp): no dependent second trip
     s_grp_e[i] = __ldcg(P.grp_e + i); s_grp_off[i] = __ldcg(P.grp_off + i); s_grp_cnt[i] = __ldcg(P.grp_cnt + i);
   }
-  cp_async_wait_pending(0);
+  __syncthreads();                 // work groups are in shared memory
+  DnSmem m;
+  m.cb = s_cb; m.ring = ring; m.slot_u4 = L.slot_u4;
+  m.grp_e = s_grp_e; m.grp_off = s_grp_off; m.grp_cnt = s_grp_cnt; m.n_grp = n_grp;
+  Walk w;
+  dn_tiles_begin<IdxT, DENSE>(P, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps, w);   // index bytes travel ...
+  cp_async_wait_pending(D - 1);                                                                // ... the code book has landed
   __syncthreads();
   if (!DENSE && pl.repl) {
     for (int i = tid; i < P.K * 8; i += blockDim.x) s_cb[i] = s_tmp[i >> 3];
     __syncthreads();
   }
   TRACE_STAMP(2, 2);
-  dn_tiles<IdxT, DENSE>(P, T, pl, s_cb, ring, L.slot_u4, s_grp_e, s_grp_off, s_grp_cnt, n_grp,
-                        blockIdx.x * nwarps + warp, gridDim.x * nwarps);
+  dn_tiles_run<IdxT, DENSE>(P, T, pl, m, w);
 }
 
 // out[t][h] = sum over slots (in slot order) of affinity * y[t][slot][h], where y is the sum of

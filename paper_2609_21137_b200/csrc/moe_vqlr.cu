@@ -108,6 +108,17 @@ StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense) {
   return pl;
 }
 
+// After the last change to a plan: the derived constants of the work-list arithmetic.
+void finish_plan(StagePlan& pl, int W) {
+  pl.W = W;
+  pl.tail = pl.tiles % pl.chunk;
+  pl.d_per_grp = make_fastdiv((unsigned int)(pl.n_parts * pl.tiles));
+  pl.d_per_chunk = make_fastdiv((unsigned int)(pl.n_parts * pl.chunk));
+  pl.d_chunk = make_fastdiv((unsigned int)pl.chunk);
+  pl.d_tail = make_fastdiv((unsigned int)(pl.tail > 0 ? pl.tail : 1));
+  pl.d_W = make_fastdiv((unsigned int)W);
+}
+
 // Launch as a link of a programmatic-dependent-launch chain.  On the legacy default stream
 // (NULL) and the per-thread default stream the attribute is left out and the kernels run in
 // plain stream order (their griddepcontrol instructions are then no-ops).
@@ -392,6 +403,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       h->plan_dn.depth = d;
       if (dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total <= limit) break;
     }
+    finish_plan(h->plan_gu, h->sm_count * gu_warps);
+    finish_plan(h->plan_dn, h->sm_count * (kDownThreads / 32));
     const size_t smem_gu = gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total;
     h->smem_fast_dn = dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total;
     if (smem_gu > limit || h->smem_fast_dn > limit || (size_t)I * sizeof(float) > limit) ok = false;
@@ -435,6 +448,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
           h->smem_coop = coop_layout(K, h->n_books, maxT, H, I, r, h->plan_gu_coop, h->plan_dn_coop, !h->dn_dense, warps, E, k, S).total;
           fits = h->smem_coop <= limit;
         }
+      finish_plan(h->plan_gu_coop, h->sm_count * warps);
+      finish_plan(h->plan_dn_coop, h->sm_count * warps);
       if (fits) {
         h->dn_restage = (!h->dn_dense && (P.down.codebook != P.gate.codebook || h->plan_dn_coop.repl != h->plan_gu_coop.repl)) ? 1 : 0;
         const void* fn = h->dn_dense ? (h->idx_bytes == 1 ? (const void*)k_layer_coop<uint8_t, true> : (const void*)k_layer_coop<uint16_t, true>)
