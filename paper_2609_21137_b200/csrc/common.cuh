@@ -59,6 +59,7 @@ struct Params {
   float* gpart;            // [parts][maxT*(k+S)][I]  partial gate tiles of the tensor-core chain
   float* upart;            // [parts][maxT*(k+S)][I]  partial up tiles
   float* ypart;            // [parts][maxT*(k+S)][H]  partial down tiles, by pair position
+  float* zd_part;          // [maxT*(k+S)][slices][r] partial z_d of the fused kernel's slices
   int* inv_pos;            // [maxT][k+S]       pair position of (token, slot)
   int* status;             // [1]
   unsigned int* grid_bar;  // [2] arrivals and generation of the cooperative kernel's grid barrier

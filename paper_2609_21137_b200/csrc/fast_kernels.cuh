@@ -66,6 +66,21 @@ __device__ __forceinline__ void mma_block(float (&d)[4], const uint4& a, const u
   mma_tok8(d, a.z, a.w, w.z, w.w);
 }
 
+// The same block against an activation block given as bf16 hi + lo halves: hi fills token rows
+// 0..7 of the m16 tile, lo rows 8..15, so ONE pair of mma's forms both products (the tensor pipe
+// issues 0.4 m16n8k16 per clock per SM, which is as scarce here as the shared-memory lookups).
+// d[0], d[1]: hi product of token g, rows 2c and 2c+1; d[2], d[3]: the lo product.
+__device__ __forceinline__ void mma_block_hilo(float (&d)[4], const uint4& hi, const uint4& lo, const uint4& w) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(hi.x), "r"(lo.x), "r"(hi.y), "r"(lo.y), "r"(w.x), "r"(w.y));
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(hi.z), "r"(lo.z), "r"(hi.w), "r"(lo.w), "r"(w.z), "r"(w.w));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -126,7 +141,11 @@ __device__ __forceinline__ void cp_async_wait_pending(int pending) {
     case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
     case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
     case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-    default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+    case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+    case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+    case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+    case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
   }
 }
 template <typename IdxT>

@@ -15,6 +15,7 @@
 #include "generic_kernels.cuh"
 #include "fast_kernels.cuh"
 #include "coop_kernel.cuh"
+#include "fused_kernel.cuh"
 
 #include <cstdlib>
 
@@ -48,6 +49,14 @@ struct moe_vqlr_handle {
   StagePlan plan_gu, plan_dn;
   StagePlan plan_gu_coop, plan_dn_coop;   // the same cuts with ring depths chosen for the cooperative kernel
   size_t smem_fast_dn;
+  bool fused;                // router -> one kernel per (work group, slice of I) -> weighted sum
+  bool fused_forced;         // ... also for calls whose items exceed one wave (tests)
+  int fused_max_T;           // ... for calls of up to this many tokens (shared memory)
+  FusedPlan fplan;
+  signed char fused_dg[kMaxT + 1], fused_dd[kMaxT + 1];   // ring depths that fit for T tokens (0: the chain runs)
+  signed char fused_xs[kMaxT + 1];                        // ... with the tokens staged in shared memory (else read from L2)
+  StagePlan plan_gu_fused;
+  void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
   size_t workspace_bytes;
   bf16* x_stage;     // [maxT][H] device staging for the host-buffer entry point
@@ -192,6 +201,49 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
       else if (h->idx_bytes == 1) le = launch_coop(k_layer_coop<uint8_t, false>, h->sm_count, kCoopThreads, smem, st, P, xb, ob, T, h->plan_gu_coop, h->plan_dn_coop, h->n_books, h->want_dbg, h->dn_restage, zsplit);
       else le = launch_coop(k_layer_coop<uint16_t, false>, h->sm_count, kCoopThreads, smem, st, P, xb, ob, T, h->plan_gu_coop, h->plan_dn_coop, h->n_books, h->want_dbg, h->dn_restage, zsplit);
       ran = true;
+    }
+  } else if (h->fused && T <= h->fused_max_T && (h->fused_forced || T * (P.k + P.S) * h->fplan.n_sl <= h->sm_count)) {
+    // one wave of (work group, slice) items at most: with more, the chain's finer parts balance better
+    switch (stage) {
+      case 0:
+        le = launch_pdl(k_router_z_pdl, ((P.E + P.n_zrows) * ((T + kTokGroup - 1) / kTokGroup) + kRouterWarps - 1) / kRouterWarps,
+                        32 * kRouterWarps, 0, st, P, xb, T);
+        ran = true;
+        break;
+      case 2: {
+        FusedPlan fpl = h->fplan;
+        fpl.depth_g = h->fused_dg[T];
+        fpl.depth_d = h->fused_dd[T];
+        StagePlan pgl = h->plan_gu_fused;
+        pgl.x_smem = h->fused_xs[T];
+        const size_t smem2 = fused_layout(P.K, h->n_books, T, P.H, P.r, pgl, fpl, h->dn_dense, h->idx_bytes, P.E, P.k, P.S).total;
+#define MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, JDV)                                                                       \
+  le = launch_pdl(k_expert_fused<IDXT, DENSE, JDV>, h->sm_count, kFusedThreads, smem2, st, P, xb, T, pgl, fpl, h->n_books, \
+                  h->want_dbg, static_cast<const IDXT*>(DENSE ? nullptr : h->idx_dp))
+#define MOE_VQLR_FUSED_JD(IDXT, DENSE)                                  \
+  switch (fpl.jd) {                                                     \
+    case 1: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 1); break;               \
+    case 2: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 2); break;               \
+    case 3: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 3); break;               \
+    default: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 4); break;              \
+  }
+        if (h->dn_dense && h->idx_bytes == 1) { MOE_VQLR_FUSED_JD(uint8_t, true) }
+        else if (h->dn_dense) { MOE_VQLR_FUSED_JD(uint16_t, true) }
+        else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_JD(uint8_t, false) }
+        else { MOE_VQLR_FUSED_JD(uint16_t, false) }
+#undef MOE_VQLR_FUSED_JD
+#undef MOE_VQLR_FUSED_LAUNCH
+        ran = true;
+        break;
+      }
+      case 5: {
+        const int lr = (!h->dn_dense && P.r > 0) ? 1 : 0;
+        const size_t smem = ((lr ? (size_t)(P.k + P.S) * P.r : 0) + (size_t)(P.k + P.S) * kCfCols * 2) * sizeof(float);
+        le = launch_pdl(k_combine_fused, T * (P.H / 2 / kCfCols), kCfThreads, smem, st, P, ob, T, h->fplan.n_sl, lr);
+        ran = true;
+        break;
+      }
+      default: break;
     }
   } else if (h->fast) {
     switch (stage) {
@@ -462,6 +514,103 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     }
   }
 
+  // ---- one kernel per (work group, slice of I) between router and weighted sum ------------------
+  h->fused = false;
+  h->fused_forced = false;
+  h->fused_max_T = 0;
+  h->idx_dp = nullptr;
+  size_t idx_dp_bytes = 0;
+  {
+    const char* fenv = getenv("MOE_VQLR_FUSED");
+    const bool book_ok = h->dn_dense || P.down.codebook == P.gate.codebook || (h->n_books == 2 && P.down.codebook == P.up.codebook);
+    if (h->fast && !h->gu_dense && book_ok && H % 16 == 0 && !(fenv && fenv[0] == '0')) {
+      const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
+      const int tiles = I / 8;
+      int target = h->sm_count / (k + S);            // slices per expert that fill the GPU at one token
+      if (target < 1) target = 1;
+      FusedPlan fp;
+      memset(&fp, 0, sizeof fp);
+      StagePlan pg = h->plan_gu;
+      pg.x_smem = 1;
+      bool found = false;
+      for (int tps = (tiles + target - 1) / target; tps >= 1 && !found; --tps) {
+        if (tps > 4 * kFusedMaxJd) tps = 4 * kFusedMaxJd;
+        fp.tps = tps;
+        fp.n_sl = (tiles + tps - 1) / tps;
+        fp.t_last = tiles - (fp.n_sl - 1) * tps;
+        fp.jd = (tps + 3) / 4;
+        fp.rp_log2 = 3;
+        while ((1 << fp.rp_log2) < 8 * tps) ++fp.rp_log2;
+        // compressed down projection: every index byte of a warp's down tiles is resident (one slot per
+        // tile); dense: a ring as deep as fits, its bytes in flight are what hides the DRAM latency
+        const int dn_tiles_per_warp = (H / 8 + kFusedWarps - 1) / kFusedWarps;
+        for (int dd = h->dn_dense ? 8 : dn_tiles_per_warp; dd >= (h->dn_dense ? 2 : dn_tiles_per_warp) && !found; --dd)
+          for (int dg = 3; dg >= 2 && !found; --dg) {
+            fp.depth_g = dg;
+            fp.depth_d = dd;
+            found = fused_layout(K, h->n_books, 1, H, r, pg, fp, h->dn_dense, h->idx_bytes, E, k, S).total <= limit;
+          }
+      }
+      // many thin slices would turn the partial y into the dominant traffic: leave those shapes to the chain
+      const bool forced = fenv && fenv[0] == '1';
+      h->fused_forced = forced;      // tests: also where the items would not fill the GPU
+      if (found && fp.n_sl <= 32 && (forced || (k + S) * fp.n_sl * 2 >= h->sm_count)) {
+        fp.d_nsl = make_fastdiv((unsigned int)fp.n_sl);
+        fp.d_tps = make_fastdiv((unsigned int)fp.tps);
+        fp.d_tlast = make_fastdiv((unsigned int)fp.t_last);
+        int maxT_fit = 0;
+        size_t smem_max = 0;
+        const int dn_tiles_per_warp = (H / 8 + kFusedWarps - 1) / kFusedWarps;
+        memset(h->fused_dg, 0, sizeof h->fused_dg);
+        memset(h->fused_dd, 0, sizeof h->fused_dd);
+        memset(h->fused_xs, 0, sizeof h->fused_xs);
+        for (int t = 1; t <= maxT; ++t) {          // staged tokens and the deepest rings that fit beside them
+          bool fit = false;
+          for (int xsm = 1; xsm >= 0 && !fit; --xsm)
+            for (int dd = h->dn_dense ? 8 : dn_tiles_per_warp; dd >= (h->dn_dense ? 3 : dn_tiles_per_warp) && !fit; --dd)
+              for (int dg = 3; dg >= 2 && !fit; --dg) {
+                StagePlan pgt = pg;
+                pgt.x_smem = xsm;
+                fp.depth_g = dg;
+                fp.depth_d = dd;
+                const size_t need = fused_layout(K, h->n_books, t, H, r, pgt, fp, h->dn_dense, h->idx_bytes, E, k, S).total;
+                if (need <= limit) {
+                  fit = true;
+                  h->fused_dg[t] = (signed char)dg;
+                  h->fused_dd[t] = (signed char)dd;
+                  h->fused_xs[t] = (signed char)xsm;
+                  if (need > smem_max) smem_max = need;
+                }
+              }
+          if (!fit) break;                         // more tokens need more room
+          maxT_fit = t;
+        }
+        const void* fn = nullptr;
+#define MOE_VQLR_FUSED_FN(IDXT, DENSE)                                                             \
+  fn = fp.jd == 1 ? (const void*)k_expert_fused<IDXT, DENSE, 1> : fp.jd == 2 ? (const void*)k_expert_fused<IDXT, DENSE, 2> \
+     : fp.jd == 3 ? (const void*)k_expert_fused<IDXT, DENSE, 3> : (const void*)k_expert_fused<IDXT, DENSE, 4>
+        if (h->dn_dense && h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, true); }
+        else if (h->dn_dense) { MOE_VQLR_FUSED_FN(uint16_t, true); }
+        else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, false); }
+        else { MOE_VQLR_FUSED_FN(uint16_t, false); }
+#undef MOE_VQLR_FUSED_FN
+        cudaError_t e1 = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+        const size_t cf_smem = ((size_t)(k + S) * (r > 0 ? r : 0) + (size_t)(k + S) * kCfCols * 2) * sizeof(float);
+        if (e1 == cudaSuccess && cf_smem > 48 * 1024)
+          e1 = cf_smem <= limit ? cudaFuncSetAttribute(k_combine_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cf_smem) : cudaErrorInvalidValue;
+        if (e1 == cudaSuccess && maxT_fit >= 1) {
+          h->fused = true;
+          h->fused_max_T = maxT_fit;
+          h->fplan = fp;
+          h->plan_gu_fused = pg;
+          if (!h->dn_dense) idx_dp_bytes = (size_t)(E + S) * fp.n_sl * (H / 8) * 32 * fp.jd * h->idx_bytes;
+        } else {
+          cudaGetLastError();
+        }
+      }
+    }
+  }
+
   // workspace
   const char* clk_env = getenv("MOE_VQLR_PHASE_CLOCKS");
   const bool want_clk = clk_env && clk_env[0] == '1';
@@ -491,7 +640,13 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     P.zd = carve<float>(cur, n_pos * (r > 0 ? r : 1));
     P.gpart = carve<float>(cur, h->fast ? (size_t)h->plan_gu.n_parts * n_pos * I : 1);
     P.upart = carve<float>(cur, h->fast ? (size_t)h->plan_gu.n_parts * n_pos * I : 1);
-    P.ypart = carve<float>(cur, h->fast ? (size_t)h->plan_dn.n_parts * n_pos * H : 1);
+    {
+      int y_parts = h->fast ? h->plan_dn.n_parts : 0;
+      if (h->fused && h->fplan.n_sl > y_parts) y_parts = h->fplan.n_sl;
+      P.ypart = carve<float>(cur, y_parts > 0 ? (size_t)y_parts * n_pos * H : 1);
+    }
+    P.zd_part = carve<float>(cur, (h->fused && !h->dn_dense && r > 0) ? n_pos * h->fplan.n_sl * r : 1);
+    h->idx_dp = carve<char>(cur, idx_dp_bytes > 0 ? idx_dp_bytes : 1);
     P.inv_pos = carve<int>(cur, n_pos);
     P.status = carve<int>(cur, 1);
     P.grid_bar = carve<unsigned int>(cur, 2);
@@ -510,6 +665,20 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   }
   plan(static_cast<char*>(h->workspace));
   cudaMemset(h->workspace, 0, h->workspace_bytes);
+  if (h->fused && !h->dn_dense) {      // one-off: the down index map per slice
+    const FusedPlan& fp = h->fplan;
+    if (h->idx_bytes == 1)
+      k_relay_down_idx<uint8_t><<<h->sm_count * 8, 256>>>(static_cast<const uint8_t*>(P.down.idx), static_cast<uint8_t*>(h->idx_dp), E + S, H, I / kD, fp.tps, fp.n_sl, fp.jd);
+    else
+      k_relay_down_idx<uint16_t><<<h->sm_count * 8, 256>>>(static_cast<const uint16_t*>(P.down.idx), static_cast<uint16_t*>(h->idx_dp), E + S, H, I / kD, fp.tps, fp.n_sl, fp.jd);
+    ce = cudaDeviceSynchronize();
+    if (ce != cudaSuccess) {
+      rc = fail(nullptr, MOE_VQLR_ERR_CUDA, "re-laying the down index map: %s", cudaGetErrorString(ce));
+      cudaFree(h->workspace);
+      delete h;
+      return rc;
+    }
+  }
 
   if (cfg->flags & MOE_VQLR_FLAG_VALIDATE_INDICES) {
     unsigned int* d_max = reinterpret_cast<unsigned int*>(P.status);

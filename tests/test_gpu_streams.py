@@ -102,3 +102,29 @@ def test_persistent_kernel(shp):
         assert_routing(dbg, res)
         assert_output(bf16_tensor_to_f64(out), res.out)
     mod.close()
+
+
+@pytest.mark.parametrize("shp", [synth.shape("tiny", T=5), synth.shape("tiny", T=2, mode="paper"),
+                                 synth.shape("qwen3", E=16, T=3), synth.shape("qwen3", E=16, T=9, mode="paper"),
+                                 synth.shape("qwen3", E=16, T=16, I=832), synth.shape("dsv2lite", E=16, T=1),
+                                 synth.shape("dsv2lite", E=16, T=2, mode="paper")],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}-I{s.I}")
+def test_fused_expert_kernel_forced(shp):
+    """Router -> one kernel per (work group, slice of I) -> weighted sum, forced also where the
+    items would not fill the GPU: three launches per call, the chain's results."""
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    os.environ["MOE_VQLR_FUSED"] = "1"
+    try:
+        mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    finally:
+        del os.environ["MOE_VQLR_FUSED"]
+    x = binding.bits_to_device(layer.x, "cuda")
+    for _ in range(2):
+        before = mod.launch_count
+        out, dbg = mod.decode(x, debug=True)
+        torch.cuda.synchronize()
+        assert mod.launch_count - before == 3
+        assert_routing(dbg, res)
+        assert_output(bf16_tensor_to_f64(out), res.out)
+    mod.close()
