@@ -29,8 +29,8 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) per launch of the dominant kernel, from the ncu captures summarised
 # in profiles/k_gateup_mma_k_down_mma_qwen3_*.md (small case; per-launch traffic is that of the
 # full benchmark because every launch reads one layer's activated experts).
-NCU_TRAFFIC = {("qwen3", "full", "gateup"): 8.01e6, ("qwen3", "full", "down"): 5.36e6,
-               ("qwen3_b16", "full", "gateup"): 42.5e6 + 0.37e6, ("qwen3_b16", "full", "down"): 28.7e6 + 0.05e6}
+NCU_TRAFFIC = {("qwen3", "full", "k_gateup_mma"): 8.01e6, ("qwen3", "full", "k_down_mma"): 5.36e6,
+               ("qwen3_b16", "full", "k_gateup_mma"): 42.5e6 + 0.37e6, ("qwen3_b16", "full", "k_down_mma"): 28.7e6 + 0.05e6}
 
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
@@ -374,12 +374,20 @@ def main():
     gu_bytes = sum(b.gateup_kernel for b in wl.bytes) / len(wl.bytes)
     dn_bytes = sum(b.down_kernel for b in wl.bytes) / len(wl.bytes)
     stage_bytes = {"gateup": gu_bytes, "down": dn_bytes}
+    kernel_names = {"gateup": "k_gateup_mma", "down": "k_down_mma"}
+    if stage_ms.get("down", 0.0) == 0.0 and stage_ms.get("zdown", 0.0) == 0.0:
+        # the fused expert kernel ran as the "gateup" stage: it streams gate/up and the down indices (or the
+        # dense down matrix); the low-rank factor of a compressed down projection is read by the weighted sum
+        lr_down = 2 * shp.H * shp.r if args.mode == "full" else 0
+        n_act = sum(b.n_active for b in wl.bytes) / len(wl.bytes)
+        stage_bytes = {"gateup": gu_bytes + dn_bytes - n_act * lr_down}
+        kernel_names = {"gateup": "k_expert_fused"}
     dominant = max(stage_bytes, key=lambda s: stage_ms.get(s, 0.0))
     dom_ms = stage_ms[dominant]
     achieved = stage_bytes[dominant] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": f"k_{dominant}", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": kernel_names[dominant], "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                "traffic": NCU_TRAFFIC.get((args.workload, args.mode, dominant)), "algorithmic_bytes_per_launch": stage_bytes[dominant],
+                "traffic": NCU_TRAFFIC.get((args.workload, args.mode, kernel_names[dominant])), "algorithmic_bytes_per_launch": stage_bytes[dominant],
                 "us_per_launch": dom_ms * 1e3,
                 "how": "each stage's kernel replayed back to back over the rotating layers in a captured graph, CUDA events",
                 "stage_us": {k_: v * 1e3 for k_, v in stage_ms.items()},

@@ -899,8 +899,10 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
           zgh = s_zh[ig2]; zgl = s_zl[ig2]; zuh = s_zh[iu2]; zul = s_zl[iu2];
         }
       }
-      mma_block(acc_g[0], zgh, fg); mma_block(acc_g[1], zgl, fg);
-      mma_block(acc_u[0], zuh, fu); mma_block(acc_u[1], zul, fu);
+      mma_block_hilo(acc_g[0], zgh, zgl, fg);      // rows 8..15 of the tile carry the lo product
+      mma_block_hilo(acc_u[0], zuh, zul, fu);
+      acc_g[0][0] += acc_g[0][2]; acc_g[0][1] += acc_g[0][3];
+      acc_u[0][0] += acc_u[0][2]; acc_u[0][1] += acc_u[0][3];
     }
     TRACE_STAMP(0, 6 + 3 * i);
     // partial tile of this part: token g of the group, rows 2c and 2c+1 of the tile
@@ -1204,8 +1206,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const uint4 v = b0 + 4 * j < nb ? ring[(slot * 8 + j) * 32] : make_uint4(0, 0, 0, 0);
-        mma_block(acc[j & 1], fh[j], v);
-        mma_block(acc[2 + (j & 1)], fl[j], v);
+        mma_block_hilo(acc[j & 1], fh[j], fl[j], v);
       }
     } else {
       // mma.sync needs the whole warp: out-of-range block groups use index 0 and zero fragments
@@ -1216,13 +1217,11 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const uint4 w = s_cb[pl.repl ? ((id[j] << 3) | (lane & 7)) : id[j]];
-        mma_block(acc[j & 1], fh[j], w);
-        mma_block(acc[2 + (j & 1)], fl[j], w);
+        mma_block_hilo(acc[j & 1], fh[j], fl[j], w);      // hi product in rows 0..7 of the tile, lo in rows 8..15
       }
       if (part < pl.n_lr) {                   // warp-uniform: the low-rank group carried by this part
         const uint4 f = rho0 < P.r ? ring[(slot * 2 + 1) * 32] : make_uint4(0, 0, 0, 0);
-        mma_block(acc[0], zh, f);
-        mma_block(acc[2], zl, f);
+        mma_block_hilo(acc[2], zh, zl, f);
         const size_t row = (size_t)s_grp_e[grp] * P.H + jt * 8 + g;
         for (int lg = part + pl.n_slices; lg < pl.n_lr; lg += pl.n_slices) {   // more rank groups than slices
           const int rho = lg * 32 + 8 * c;
@@ -1234,8 +1233,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
               split_hi_lo(__ldcg(zp), __ldcg(zp + 1), zh2, zl2);
             }
           }
-          mma_block(acc[1], zh2, f2);
-          mma_block(acc[3], zl2, f2);
+          mma_block_hilo(acc[3], zh2, zl2, f2);
         }
       }
     }
@@ -1243,7 +1241,8 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
     if (pos >= 0) {
       const size_t at = ((size_t)part * n_pos + pos) * P.H + jt * 8 + 2 * c;
       *reinterpret_cast<float2*>(P.ypart + at) =
-          make_float2((acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]), (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]));
+          make_float2(((acc[0][0] + acc[0][2]) + (acc[1][0] + acc[1][2])) + ((acc[2][0] + acc[2][2]) + (acc[3][0] + acc[3][2])),
+                      ((acc[0][1] + acc[0][3]) + (acc[1][1] + acc[1][3])) + ((acc[2][1] + acc[2][3]) + (acc[3][1] + acc[3][3])));
     }
   }
   cp_async_wait_pending(0);

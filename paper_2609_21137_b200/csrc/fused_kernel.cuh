@@ -127,8 +127,11 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
   // (part-major: consecutive units share their activation fragments) followed by an even share of
   // the cheap low-rank units.
   struct Item {
-    int e, off, cnt, si, tiles, row0, s0, ns, l0, n_my;
-    FastDiv d_tiles;
+    int e, off, cnt, si, tiles, row0, ns, n_my;
+    int sp, st, lp, lt;       // (part, tile) of the first slice unit and of the first low-rank unit of this warp
+  };
+  struct UnitCur {            // walks the warp's units in order: slice units, then low-rank units
+    int i, part, tile;
   };
   auto load_item = [&](int v) {
     Item it;
@@ -137,25 +140,32 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     it.e = R.grp_e[gi]; it.off = R.grp_off[gi]; it.cnt = R.grp_cnt[gi];
     const bool last_sl = it.si == fp.n_sl - 1;
     it.tiles = last_sl ? fp.t_last : fp.tps;
-    it.d_tiles = last_sl ? fp.d_tlast : fp.d_tps;
+    const FastDiv d_tiles = last_sl ? fp.d_tlast : fp.d_tps;
     it.row0 = it.si * fp.tps * 8;
     const int Us = pg.n_slices * it.tiles, Ul = pg.n_lr * it.tiles;
-    it.s0 = Us * warp / kFusedWarps;
-    it.ns = Us * (warp + 1) / kFusedWarps - it.s0;
-    it.l0 = Ul * warp / kFusedWarps;
-    it.n_my = it.ns + Ul * (warp + 1) / kFusedWarps - it.l0;
+    const int s0 = Us * warp / kFusedWarps, l0 = Ul * warp / kFusedWarps;
+    it.ns = Us * (warp + 1) / kFusedWarps - s0;
+    it.n_my = it.ns + Ul * (warp + 1) / kFusedWarps - l0;
+    it.sp = fdiv(s0, d_tiles); it.st = s0 - it.sp * it.tiles;
+    const int lq = fdiv(l0, d_tiles);
+    it.lp = pg.n_slices + lq; it.lt = l0 - lq * it.tiles;
     return it;
   };
-  auto unit_of = [&](const Item& it, int i, int& part, int& tile) {       // i-th gate/up unit of this warp
-    const int u = i < it.ns ? it.s0 + i : it.l0 + (i - it.ns);
-    const int q = fdiv(u, it.d_tiles);
-    tile = u - q * it.tiles;
-    part = i < it.ns ? q : pg.n_slices + q;
+  auto cur_begin = [&](const Item& it) {
+    UnitCur u;
+    u.i = 0;
+    if (it.ns > 0) { u.part = it.sp; u.tile = it.st; } else { u.part = it.lp; u.tile = it.lt; }
+    return u;
+  };
+  auto cur_next = [&](const Item& it, UnitCur& u) {
+    ++u.i;
+    if (u.i == it.ns) { u.part = it.lp; u.tile = it.lt; }
+    else if (++u.tile == it.tiles) { u.tile = 0; ++u.part; }
   };
   int g_rq = 0, g_use = 0;             // gate/up ring: next slot to request into, next to consume
-  auto gu_request = [&](const Item& it, int i) {                          // requests come in the order of use
-    int part, tile;
-    unit_of(it, i, part, tile);
+  auto gu_request = [&](const Item& it, UnitCur& rq) {                    // requests come in the order of use
+    const int part = rq.part, tile = rq.tile;
+    cur_next(it, rq);
     uint4* slot = m.ring + (size_t)g_rq * 2 * 32;
     if (++g_rq == Dg) g_rq = 0;
     const size_t row = (size_t)it.e * P.I + it.row0 + tile * 8 + g;
@@ -191,7 +201,8 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
 
   if ((int)blockIdx.x >= n_items) { cp_async_wait_pending(0); return; }
   Item it = load_item(blockIdx.x);
-  for (int i = 0; i < Dg - 1; ++i) { if (i < it.n_my) gu_request(it, i); cp_async_commit(); }
+  UnitCur rq = cur_begin(it);            // request cursor of the current item (of the next one once its first units are requested)
+  for (int i = 0; i < Dg - 1; ++i) { if (i < it.n_my) gu_request(it, rq); cp_async_commit(); }
   gu_finish_stage<false>(P, pg, n_books, m, Dg - 1);     // code books, tokens, z, routing lists
   pdl_launch();
 
@@ -215,12 +226,14 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     {
       uint4 fx[8];
       int frag_part = -1;
+      UnitCur use = cur_begin(it);
       for (int i = 0; i < n_my; ++i) {
-        if (i + Dg - 1 < n_my) gu_request(it, i + Dg - 1);
+        if (i + Dg - 1 < n_my) gu_request(it, rq);
         cp_async_commit();
         cp_async_wait_pending(Dg - 1);
-        int part, tile;
-        unit_of(it, i, part, tile);
+        if (i < 3) TRACE_STAMP(3, 10 + 2 * i);
+        const int part = use.part, tile = use.tile;
+        cur_next(it, use);
         const uint4* slot = m.ring + (size_t)g_use * 2 * 32;
         if (++g_use == Dg) g_use = 0;
         const int tok = g < cnt ? R.pair_token[off + g] : -1;
@@ -277,6 +290,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
         float* dst = s_parts + ((size_t)(part * fp.tps + tile) * 2) * 64 + g * 8 + 2 * c;
         *reinterpret_cast<float2*>(dst) = make_float2(acc_g[0][0] + acc_g[1][0], acc_g[0][1] + acc_g[1][1]);
         *reinterpret_cast<float2*>(dst + 64) = make_float2(acc_u[0][0] + acc_u[1][0], acc_u[0][1] + acc_u[1][1]);
+        if (i < 3) TRACE_STAMP(3, 11 + 2 * i);
       }
     }
     // what is left of the down requests; then the ring start of the other product
@@ -286,7 +300,8 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
       newest = Dd - 1;
     } else {
       if (has_next) {                    // the gate/up ring is free: the next item's first units start travelling
-        for (int i = 0; i < Dg - 1; ++i) { if (i < nx.n_my) gu_request(nx, i); cp_async_commit(); }
+        rq = cur_begin(nx);
+        for (int i = 0; i < Dg - 1; ++i) { if (i < nx.n_my) gu_request(nx, rq); cp_async_commit(); }
         newest = Dg - 1;
       }
     }
@@ -417,7 +432,8 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
         }
       }
       if (DN_DENSE && has_next) {        // all dense groups are done with: the next item's first gate/up units
-        for (int i = 0; i < Dg - 1; ++i) { if (i < nx.n_my) gu_request(nx, i); cp_async_commit(); }
+        rq = cur_begin(nx);
+        for (int i = 0; i < Dg - 1; ++i) { if (i < nx.n_my) gu_request(nx, rq); cp_async_commit(); }
       }
     }
     TRACE_STAMP(3, 8);
@@ -461,6 +477,17 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
       pos = __ldcg(P.inv_pos + t * n_slots + s);
       e = s < P.k ? __ldcg(P.topk_id + t * P.k + s) : P.E + (s - P.k);
     }
+    // the first two z_d entries of this thread (slot sj, rank rho): their positions travel with `pos`
+    const int n_here = min(kCfThreads / 32, n_slots - s0);
+    const int n_zd = lr ? n_here * r : 0;
+    int zsj[2], zrho[2], zpj[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int idx = tid + u * kCfThreads;
+      zsj[u] = idx < n_zd ? idx / r : 0;
+      zrho[u] = idx - zsj[u] * r;
+      zpj[u] = idx < n_zd ? __ldcg(P.inv_pos + t * n_slots + s0 + zsj[u]) : 0;
+    }
     float2 yv[kYv];
     uint4 a0v[kAv], a1v[kAv];
     const float* ysrc = P.ypart + (size_t)pos * P.H + 2 * h2;
@@ -480,19 +507,30 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
       a1v[i] = on ? __ldg(a1 + rg) : make_uint4(0, 0, 0, 0);
     }
     if (lr) {                            // z_d of this trip's slots: sum of the slices' parts, ascending
-      const int n_here = min(kCfThreads / 32, n_slots - s0);
-      for (int idx = tid; idx < n_here * r; idx += kCfThreads) {
+      float zv[2][16];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const float* src = P.zd_part + (size_t)zpj[u] * n_sl * r + zrho[u];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) zv[u][i] = (tid + u * kCfThreads < n_zd && i < n_sl) ? __ldcg(src + (size_t)i * r) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        if (tid + u * kCfThreads < n_zd) {
+          float acc = 0.f;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) acc += zv[u][i];
+          const float* src = P.zd_part + (size_t)zpj[u] * n_sl * r + zrho[u];
+          for (int si = 16; si < n_sl; ++si) acc += __ldcg(src + (size_t)si * r);
+          s_zd[(s0 + zsj[u]) * r + zrho[u]] = acc;
+        }
+      }
+      for (int idx = tid + 2 * kCfThreads; idx < n_zd; idx += kCfThreads) {
         const int sj = idx / r, rho = idx - sj * r;
         const int pj = __ldcg(P.inv_pos + t * n_slots + s0 + sj);
         const float* src = P.zd_part + (size_t)pj * n_sl * r + rho;
         float acc = 0.f;
-        for (int si0 = 0; si0 < n_sl; si0 += 16) {       // sixteen slices' loads in flight
-          float zv[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) zv[i] = si0 + i < n_sl ? __ldcg(src + (size_t)(si0 + i) * r) : 0.f;
-#pragma unroll
-          for (int i = 0; i < 16; ++i) acc += zv[i];
-        }
+        for (int si = 0; si < n_sl; ++si) acc += __ldcg(src + (size_t)si * r);
         s_zd[(s0 + sj) * r + rho] = acc;
       }
       __syncthreads();
