@@ -29,7 +29,8 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) per launch of the dominant kernel, from the ncu captures summarised
 # in profiles/k_gateup_mma_k_down_mma_qwen3_*.md (small case; per-launch traffic is that of the
 # full benchmark because every launch reads one layer's activated experts).
-NCU_TRAFFIC = {("qwen3", "full", "k_gateup_mma"): 8.01e6, ("qwen3", "full", "k_down_mma"): 5.36e6,
+NCU_TRAFFIC = {("qwen3", "full", "k_expert_fused"): 12.32e6,     # profiles/k_expert_fused_qwen3_b1.md
+               ("qwen3", "full", "k_gateup_mma"): 8.01e6, ("qwen3", "full", "k_down_mma"): 5.36e6,
                ("qwen3_b16", "full", "k_gateup_mma"): 42.5e6 + 0.37e6, ("qwen3_b16", "full", "k_down_mma"): 28.7e6 + 0.05e6}
 
 L2_BYTES = 126 * 1024 * 1024
