@@ -193,7 +193,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
   if (h->coop && allow_coop) {
     if (stage == 0) {
       int zsplit = 1;
-      if (!h->dn_dense && P.r > 0) while (n_pos * zsplit * 2 <= h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
+      if (!h->dn_dense && P.r > 0) while (n_pos * zsplit * 2 <= 3 * h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
       const size_t smem = coop_layout(P.K, h->n_books, T, P.H, P.I, P.r, h->plan_gu_coop, h->plan_dn_coop, !h->dn_dense, kCoopThreads / 32, P.E, P.k, P.S).total;
       // the index type is the gate/up projections' (a dense down projection has no indices)
       if (h->dn_dense && h->idx_bytes == 1) le = launch_coop(k_layer_coop<uint8_t, true>, h->sm_count, kCoopThreads, smem, st, P, xb, ob, T, h->plan_gu_coop, h->plan_dn_coop, h->n_books, h->want_dbg, h->dn_restage, zsplit);
@@ -264,7 +264,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         const int with_zd = (!h->dn_dense && P.r > 0) ? 1 : 0;
         if (P.I <= 4096) {                                // one fused block per pair (times zsplit)
           int zsplit = 1;
-          if (with_zd) while (n_pos * zsplit * 2 <= h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
+          if (with_zd) while (n_pos * zsplit * 2 <= 3 * h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
           le = launch_pdl(k_act_zdown, n_pos * zsplit, kActThreads, (size_t)P.I * sizeof(float), st, P, n_pos,
                           h->plan_gu.n_parts, with_zd, zsplit);
         } else {                                          // few pairs or a long intermediate: two wide kernels
