@@ -470,6 +470,60 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
   }
 }
 
+// Routing of a single token as far as a block of the fused kernel needs it: WHICH experts are
+// selected, in ascending id order (= the work groups).  Expert e is selected iff fewer than k
+// experts precede it in the order (logit descending, id ascending) -- one thread per expert counts
+// them, no dependent rounds; slots, affinities and the global lists are left to the one block that
+// runs route_in_block.  E <= 1024.
+__device__ void route_light_t1(const Params& P, const RouteSmem& R) {
+  const int E = P.E, k = P.k, S = P.S;
+  const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
+  unsigned int* s_key = reinterpret_cast<unsigned int*>(R.logit);
+  for (int i = tid; i < E; i += nthr) s_key[i] = logit_key(__ldcg(P.logits + i));
+  __syncthreads();
+  const int n_chunks = (E + 31) >> 5;                       // ballots of 32 experts each
+  for (int e0 = (tid >> 5) << 5; e0 < E; e0 += nthr) {      // warp-uniform trip count
+    const int e = e0 + lane;
+    bool sel = false;
+    if (e < E) {
+      const unsigned int key = s_key[e];
+      int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+      if ((E & 3) == 0) {
+#pragma unroll 4
+        for (int e2 = 0; e2 < E; e2 += 4) {
+          const uint4 v = *reinterpret_cast<const uint4*>(s_key + e2);
+          c0 += (v.x > key) | ((v.x == key) & (e2 < e));
+          c1 += (v.y > key) | ((v.y == key) & (e2 + 1 < e));
+          c2 += (v.z > key) | ((v.z == key) & (e2 + 2 < e));
+          c3 += (v.w > key) | ((v.w == key) & (e2 + 3 < e));
+        }
+      } else {
+        for (int e2 = 0; e2 < E; ++e2) c0 += (s_key[e2] > key) | ((s_key[e2] == key) & (e2 < e));
+      }
+      sel = (c0 + c1) + (c2 + c3) < k;
+    }
+    const unsigned int bal = __ballot_sync(0xffffffffu, sel);
+    if (lane == 0) R.warp_cnt[e0 >> 5] = (int)bal;
+  }
+  __syncthreads();
+  for (int e = tid; e < E; e += nthr) {
+    const unsigned int bal = (unsigned int)R.warp_cnt[e >> 5];
+    if ((bal >> (e & 31)) & 1u) {
+      int pos = __popc(bal & ((1u << (e & 31)) - 1u));
+      for (int w = 0; w < (e >> 5); ++w) pos += __popc((unsigned int)R.warp_cnt[w]);
+      R.pair_token[pos] = 0;
+      R.grp_e[pos] = e; R.grp_off[pos] = pos; R.grp_cnt[pos] = 1;
+    }
+  }
+  for (int s2 = tid; s2 < S; s2 += nthr) {
+    R.pair_token[k + s2] = 0;
+    R.grp_e[k + s2] = E + s2; R.grp_off[k + s2] = k + s2; R.grp_cnt[k + s2] = 1;
+  }
+  if (tid == 0) *R.n_grp = k + S;
+  (void)n_chunks;
+  __syncthreads();
+}
+
 // ---------------------------------------------------------------------------------------------
 // k_router_z_pdl: head of the chain.  One warp per (row of [router_w ; basis_gate ; basis_up],
 // group of four tokens).  Per (row, token) the summation order is the one of k_router_z
@@ -759,9 +813,21 @@ __device__ __forceinline__ void gu_stage_books_async(const Params& P, const Stag
   if (!DENSE) {
     uint4* dst_g = pl.repl ? m.tmp : m.cb_g;
     uint4* dst_u = pl.repl ? m.tmp + P.K : m.cb_u;
-    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_g + i, P.gate.codebook + i);
+    // Every block fetches the same few KB from L2: each starts at its own offset, so that at any
+    // moment the blocks ask for different lines (all asking for the same lines in the same order
+    // serialises on single L2 slices: 5 us instead of 1-2 for 64 KB x 148 blocks).
+    const int rot = (int)(((unsigned int)blockIdx.x * (unsigned int)P.K) / gridDim.x);
+    for (int i = tid; i < P.K; i += blockDim.x) {
+      int j = i + rot;
+      if (j >= P.K) j -= P.K;
+      cp_async16(dst_g + j, P.gate.codebook + j);
+    }
     if (n_books == 2)
-      for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst_u + i, P.up.codebook + i);
+      for (int i = tid; i < P.K; i += blockDim.x) {
+        int j = i + rot;
+        if (j >= P.K) j -= P.K;
+        cp_async16(dst_u + j, P.up.codebook + j);
+      }
   }
   cp_async_commit();
 }
@@ -775,7 +841,7 @@ __device__ __forceinline__ void gu_stage_async(const Params& P, const bf16* __re
 
 // After logits and z are complete: z as bf16 hi / lo blocks, routing, and the staged bytes landed.
 __device__ __forceinline__ void gu_route(const Params& P, int T, const StagePlan& pl, const GuSmem& m,
-                                         bool write_global, bool want_dbg) {
+                                         bool write_global, bool want_dbg, bool light = false) {
   const int tid = threadIdx.x, rb = (P.r + 7) / 8;
   float4 zv[2][2];                 // this thread's z values travel while the routing runs (up to two blocks of 8 each)
   const int nz = pl.n_lr > 0 ? T * 2 * rb : 0;
@@ -788,7 +854,7 @@ __device__ __forceinline__ void gu_route(const Params& P, int T, const StagePlan
       zv[q][1] = __ldcg(reinterpret_cast<const float4*>(zp + 4));
     }
   }
-  route_in_block(P, T, m.R, write_global, want_dbg);
+  if (light) route_light_t1(P, m.R); else route_in_block(P, T, m.R, write_global, want_dbg);
 #pragma unroll
   for (int q = 0; q < 2; ++q) {
     const int i = tid + q * blockDim.x;

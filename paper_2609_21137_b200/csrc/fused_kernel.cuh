@@ -117,7 +117,13 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
   gu_stage_async<false>(P, x, T, pg, n_books, m);
   pdl_wait();      // logits and z of this call are complete
   TRACE_STAMP(3, 1);
-  gu_route(P, T, pg, m, blockIdx.x == 0, want_dbg != 0);
+  // One block publishes the routing (slots, affinities, lists) for the weighted sum and the caller:
+  // a block without an item if there is one, else block 0.  For a single token the other blocks
+  // only need the selected experts in id order, which is much shorter to find.
+  const int min_items = (P.k + P.S) * fp.n_sl;          // every token adds at least this many
+  const int writer = (T == 1 && min_items < (int)gridDim.x) ? (int)gridDim.x - 1 : 0;
+  const bool is_writer = (int)blockIdx.x == writer;
+  gu_route(P, T, pg, m, is_writer, want_dbg != 0, T == 1 && !is_writer && P.E <= 1024);
   TRACE_STAMP(3, 2);
 
   const int n_grp = *R.n_grp, n_pos = T * (P.k + P.S), n_items = n_grp * fp.n_sl;
@@ -231,7 +237,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
         if (i + Dg - 1 < n_my) gu_request(it, rq);
         cp_async_commit();
         cp_async_wait_pending(Dg - 1);
-        if (i < 3) TRACE_STAMP(3, 10 + 2 * i);
+        if (i < 2) TRACE_STAMP(3, 10 + 2 * i);
         const int part = use.part, tile = use.tile;
         cur_next(it, use);
         const uint4* slot = m.ring + (size_t)g_use * 2 * 32;
@@ -290,7 +296,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
         float* dst = s_parts + ((size_t)(part * fp.tps + tile) * 2) * 64 + g * 8 + 2 * c;
         *reinterpret_cast<float2*>(dst) = make_float2(acc_g[0][0] + acc_g[1][0], acc_g[0][1] + acc_g[1][1]);
         *reinterpret_cast<float2*>(dst + 64) = make_float2(acc_u[0][0] + acc_u[1][0], acc_u[0][1] + acc_u[1][1]);
-        if (i < 3) TRACE_STAMP(3, 11 + 2 * i);
+        if (i < 2) TRACE_STAMP(3, 11 + 2 * i);
       }
     }
     // what is left of the down requests; then the ring start of the other product
