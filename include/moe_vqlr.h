@@ -132,7 +132,9 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
  * asynchronous up to the final wait; pageable memory works but is slower.  Weights stay on
  * the device.  Synchronous on return.  The first call for each T captures the kernel chain into
  * a CUDA graph owned by the handle (later calls replay it), so that first call is slower and
- * must not itself run inside a stream capture. */
+ * must not itself run inside a stream capture.  With pinned host buffers the two copies are part
+ * of the graph too (one launch and one wait per call) for as long as the caller passes the same
+ * two pointers; other pointers re-capture it. */
 int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T, void* out_host,
                                void* cuda_stream);
 

@@ -63,6 +63,10 @@ struct moe_vqlr_handle {
   bf16* out_stage;   // [maxT][H]
   cudaStream_t cap_stream;                 // only ever used to capture the graphs below
   cudaGraphExec_t host_graph[kMaxT + 1];   // kernel chain x_stage -> out_stage for T tokens
+  cudaGraphExec_t io_graph[kMaxT + 1];     // the same with both host copies inside, for the host buffers below
+  const void* io_x[kMaxT + 1];
+  void* io_out[kMaxT + 1];
+  bool io_graph_failed;                    // host buffers that cannot be captured (pageable): copies stay outside
   int host_graph_launches;                 // kernels in one such graph
   int64_t launches;
   int profiling;             // record an event after every stage of a call
@@ -781,6 +785,48 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
       return fail(h, MOE_VQLR_ERR_CUDA, "graph capture of the layer: %s", cudaGetErrorString(ge));
     }
   }
+  // Callers that reuse their (pinned) host buffers get the two copies inside the graph as well:
+  // one launch and one synchronisation per call.
+  if (!h->profiling && !h->io_graph_failed) {
+    if (h->io_graph[T] && (h->io_x[T] != x_host || h->io_out[T] != out_host)) {
+      cudaGraphExecDestroy(h->io_graph[T]);
+      h->io_graph[T] = nullptr;
+    }
+    if (!h->io_graph[T]) {
+      cudaPointerAttributes ax, ao;
+      const bool pinned = cudaPointerGetAttributes(&ax, x_host) == cudaSuccess && ax.type == cudaMemoryTypeHost &&
+                          cudaPointerGetAttributes(&ao, out_host) == cudaSuccess && ao.type == cudaMemoryTypeHost;
+      cudaGetLastError();
+      cudaGraph_t graph = nullptr;
+      cudaError_t ge = pinned ? cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal) : cudaErrorNotSupported;
+      if (ge == cudaSuccess) {
+        const int64_t before = h->launches;
+        cudaError_t c1 = cudaMemcpyAsync(h->x_stage, x_host, bytes, cudaMemcpyHostToDevice, h->cap_stream);
+        const int rc = c1 == cudaSuccess ? moe_vqlr_decode_layer(h, h->x_stage, T, h->out_stage, nullptr, h->cap_stream) : MOE_VQLR_ERR_CUDA;
+        cudaError_t c2 = cudaMemcpyAsync(out_host, h->out_stage, bytes, cudaMemcpyDeviceToHost, h->cap_stream);
+        h->launches = before;
+        ge = cudaStreamEndCapture(h->cap_stream, &graph);
+        if ((rc != MOE_VQLR_OK || c1 != cudaSuccess || c2 != cudaSuccess) && ge == cudaSuccess) ge = cudaErrorUnknown;
+      }
+      if (ge == cudaSuccess) ge = cudaGraphInstantiate(&h->io_graph[T], graph, 0);
+      if (graph) cudaGraphDestroy(graph);
+      if (ge != cudaSuccess) {
+        cudaGetLastError();
+        h->io_graph[T] = nullptr;
+        h->io_graph_failed = true;
+      } else {
+        h->io_x[T] = x_host;
+        h->io_out[T] = out_host;
+      }
+    }
+    if (h->io_graph[T]) {
+      cudaError_t ce2 = cudaGraphLaunch(h->io_graph[T], st);
+      if (ce2 == cudaSuccess) ce2 = cudaStreamSynchronize(st);
+      if (ce2 != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "graph launch with copies: %s", cudaGetErrorString(ce2));
+      h->launches += h->host_graph_launches;
+      return MOE_VQLR_OK;
+    }
+  }
   cudaError_t ce = cudaMemcpyAsync(h->x_stage, x_host, bytes, cudaMemcpyHostToDevice, st);
   if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "copy in: %s", cudaGetErrorString(ce));
   if (h->host_graph[T] && !h->profiling) {
@@ -802,6 +848,8 @@ int moe_vqlr_destroy(moe_vqlr_handle* h) {
   for (auto& e : h->ev)
     if (e) cudaEventDestroy(e);
   for (auto& g : h->host_graph)
+    if (g) cudaGraphExecDestroy(g);
+  for (auto& g : h->io_graph)
     if (g) cudaGraphExecDestroy(g);
   if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
   cudaError_t ce = cudaFree(h->workspace);
