@@ -128,3 +128,27 @@ def test_fused_expert_kernel_forced(shp):
         assert_routing(dbg, res)
         assert_output(bf16_tensor_to_f64(out), res.out)
     mod.close()
+
+
+def test_fused_single_token_ties_and_no_renorm():
+    """One token on the fused path: the blocks with an item find the selected experts by counting
+    ranks, one other block by the k rounds of arg-max; both must follow the rule (logit descending,
+    id ascending) when two router rows are identical, whichever side of the cut the pair falls on."""
+    from paper_2609_21137_b200 import binding
+    shp = synth.shape("tiny", T=1, E=8, k=3)
+    os.environ["MOE_VQLR_FUSED"] = "1"
+    try:
+        for seed in range(8):
+            for renorm in (True, False):
+                layer, res, _ = make_checked_layer(shp, seed=seed, tie=(6, 2), renorm_topk=renorm)
+                mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", renorm_topk=renorm)
+                x = binding.bits_to_device(layer.x, "cuda")
+                before = mod.launch_count
+                out, dbg = mod.decode(x, debug=True)
+                torch.cuda.synchronize()
+                assert mod.launch_count - before == 3
+                assert_routing(dbg, res)
+                assert_output(bf16_tensor_to_f64(out), res.out)
+                mod.close()
+    finally:
+        del os.environ["MOE_VQLR_FUSED"]
