@@ -152,3 +152,28 @@ def test_fused_single_token_ties_and_no_renorm():
                 mod.close()
     finally:
         del os.environ["MOE_VQLR_FUSED"]
+
+
+@pytest.mark.parametrize("shp", [
+    synth.LayerShape("e70", H=512, I=256, E=70, k=5, d=8, K=700, r=16, T=1),            # E not a multiple of 4 or 32
+    synth.LayerShape("e512", H=512, I=256, E=512, k=6, d=8, K=256, r=8, T=1, S=1),      # more experts than threads, replicated book
+    synth.LayerShape("e70b", H=512, I=320, E=70, k=5, d=8, K=300, r=24, T=3, mode="paper", router_bias=True),
+], ids=lambda s: s.name)
+def test_fused_odd_expert_counts(shp):
+    """The single-token routing of the fused path (rank by counting, ballots of 32 experts) on expert
+    counts that do not fill its vector loads or its warps, and the forced multi-token path with a bias."""
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    os.environ["MOE_VQLR_FUSED"] = "1"
+    try:
+        mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    finally:
+        del os.environ["MOE_VQLR_FUSED"]
+    x = binding.bits_to_device(layer.x, "cuda")
+    before = mod.launch_count
+    out, dbg = mod.decode(x, debug=True)
+    torch.cuda.synchronize()
+    assert mod.launch_count - before == 3
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out)
+    mod.close()
