@@ -664,27 +664,29 @@ __device__ __forceinline__ void router_z_finish(const Params& P, const RouterRow
   }
 }
 
-// A single token and a row of at most 2048 values: the whole row and the token are requested in
-// one go (8 + 8 loads per lane in flight) instead of two dependent passes; same summation order.
+// A single token: the row and the token are requested 2048 values at a time (8 + 8 loads per lane
+// in flight) instead of 512; same summation order.
 __device__ __forceinline__ void router_z_unit_t1(const Params& P, const bf16* __restrict__ x, int unit, int lane) {
   const RouterRow u = router_z_row(P, 1, unit);
   const int nchunk = P.H / 8;
   const uint4* x4 = reinterpret_cast<const uint4*>(x);
-  uint4 wv[8], xv[8];
-#pragma unroll
-  for (int q = 0; q < 8; ++q) {
-    const int c = q * 32 + lane;
-    wv[q] = c < nchunk ? __ldg(u.w4 + c) : make_uint4(0, 0, 0, 0);
-    xv[q] = c < nchunk ? __ldg(x4 + c) : make_uint4(0, 0, 0, 0);
-  }
   float acc = 0.f;
+  for (int c0 = 0; c0 < nchunk; c0 += 256) {
+    uint4 wv[8], xv[8];
 #pragma unroll
-  for (int q = 0; q < 8; ++q) {
-    if (q * 32 + lane < nchunk) {
-      float wf[8], xf[8];
-      unpack8(wv[q], wf);
-      unpack8(xv[q], xf);
-      acc = dot8(wf, xf, acc);
+    for (int q = 0; q < 8; ++q) {
+      const int c = c0 + q * 32 + lane;
+      wv[q] = c < nchunk ? __ldg(u.w4 + c) : make_uint4(0, 0, 0, 0);
+      xv[q] = c < nchunk ? __ldg(x4 + c) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (c0 + q * 32 + lane < nchunk) {
+        float wf[8], xf[8];
+        unpack8(wv[q], wf);
+        unpack8(xv[q], xf);
+        acc = dot8(wf, xf, acc);
+      }
     }
   }
   const float sum = warp_sum(acc);
@@ -729,7 +731,7 @@ __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params
   pdl_launch();
   const int unit = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
   if (unit >= router_z_units(P, T)) return;
-  if (T == 1 && P.H <= 2048) router_z_unit_t1(P, x, unit, threadIdx.x & 31);
+  if (T == 1) router_z_unit_t1(P, x, unit, threadIdx.x & 31);
   else if (P.H <= 2048) router_z_unit_row8(P, x, T, unit, threadIdx.x & 31);
   else router_z_unit(P, x, T, unit, threadIdx.x & 31);
 }
@@ -1183,38 +1185,51 @@ __global__ void __launch_bounds__(256) k_act(const Params P, int n_pos, int n_pa
   }
 }
 
-__global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos) {
+// wpd warps share one z_d value (a long intermediate would otherwise be one warp's serial stream
+// of dependent loads); their partial sums meet in shared memory and are added in warp order.
+__global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos, int wpd) {
+  __shared__ float s_part[8];
   pdl_launch();
   pdl_wait();
-  const int lane = threadIdx.x & 31;
-  const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  if (w >= n_pos * P.r) return;
-  const int pos = w / P.r, rho = w - pos * P.r;
-  const uint4* brow = reinterpret_cast<const uint4*>(P.down.basis + (size_t)rho * P.I);
-  const float4* prow = reinterpret_cast<const float4*>(P.p + (size_t)pos * P.I);
-  const int nchunk = P.I / 8;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int dots_per_block = 8 / wpd;
+  const int d = blockIdx.x * dots_per_block + warp / wpd, seg = warp % wpd;
+  const bool live_dot = d < n_pos * P.r;
   float acc = 0.f;
-  for (int c0 = 0; c0 < nchunk; c0 += 128) {
-    uint4 wv[4];
-    float4 pa[4], pb[4];
+  if (live_dot) {
+    const int pos = d / P.r, rho = d - pos * P.r;
+    const uint4* brow = reinterpret_cast<const uint4*>(P.down.basis + (size_t)rho * P.I);
+    const float4* prow = reinterpret_cast<const float4*>(P.p + (size_t)pos * P.I);
+    const int nchunk = P.I / 8;
+    const int per = (nchunk + wpd - 1) / wpd, c_begin = seg * per, c_end = min(nchunk, c_begin + per);
+    for (int c0 = c_begin; c0 < c_end; c0 += 128) {
+      uint4 wv[4];
+      float4 pa[4], pb[4];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int cidx = c0 + q * 32 + lane;
-      const bool live = cidx < nchunk;
-      wv[q] = live ? __ldg(brow + cidx) : make_uint4(0, 0, 0, 0);
-      pa[q] = live ? __ldcg(prow + 2 * cidx) : make_float4(0.f, 0.f, 0.f, 0.f);
-      pb[q] = live ? __ldcg(prow + 2 * cidx + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+      for (int q = 0; q < 4; ++q) {
+        const int cidx = c0 + q * 32 + lane;
+        const bool live = cidx < c_end;
+        wv[q] = live ? __ldg(brow + cidx) : make_uint4(0, 0, 0, 0);
+        pa[q] = live ? __ldcg(prow + 2 * cidx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        pb[q] = live ? __ldcg(prow + 2 * cidx + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      float wf[8];
-      unpack8(wv[q], wf);
-      const float pf[8] = {pa[q].x, pa[q].y, pa[q].z, pa[q].w, pb[q].x, pb[q].y, pb[q].z, pb[q].w};
-      acc = dot8(wf, pf, acc);
+      for (int q = 0; q < 4; ++q) {
+        float wf[8];
+        unpack8(wv[q], wf);
+        const float pf[8] = {pa[q].x, pa[q].y, pa[q].z, pa[q].w, pb[q].x, pb[q].y, pb[q].z, pb[q].w};
+        acc = dot8(wf, pf, acc);
+      }
     }
+    acc = warp_sum(acc);
   }
-  acc = warp_sum(acc);
-  if (lane == 0) P.zd[(size_t)pos * P.r + rho] = acc;
+  if (lane == 0) s_part[warp] = acc;
+  __syncthreads();
+  if (live_dot && seg == 0 && lane == 0) {
+    float sum = 0.f;
+    for (int q = 0; q < wpd; ++q) sum += s_part[warp + q];
+    P.zd[d] = sum;
+  }
 }
 
 // ---------------------------------------------------------------------------------------------

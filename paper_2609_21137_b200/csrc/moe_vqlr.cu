@@ -276,7 +276,9 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           if (grid > 4 * h->sm_count) grid = 4 * h->sm_count;
           le = launch_pdl(k_act, grid, 256, 0, st, P, n_pos, h->plan_gu.n_parts);
           if (le == cudaSuccess && with_zd) {
-            le = launch_pdl(k_zdown_pdl, (n_pos * P.r + 7) / 8, 256, 0, st, P, n_pos);
+            int wpd = 1;                                  // warps per z_d value: 2048 values of I each, at most 8
+            while (wpd < 8 && P.I > 2048 * wpd) wpd *= 2;
+            le = launch_pdl(k_zdown_pdl, (n_pos * P.r * wpd + 7) / 8, 256, 0, st, P, n_pos, wpd);
             h->launches += 1;
           }
         }
