@@ -117,7 +117,15 @@ typedef struct {
 /* Validates the configuration, allocates the handle and its device workspace on the CURRENT
  * CUDA device and returns the handle in *out (NULL on failure).  Synchronous.
  * Errors: INVALID_ARG, UNSUPPORTED (vq_dim != 8, H or I not a multiple of 8, K > 65536, k > 32,
- * max_tokens > 16), OOM, CUDA, BAD_INDEX (only with MOE_VQLR_FLAG_VALIDATE_INDICES). */
+ * max_tokens > 16), OOM, CUDA, BAD_INDEX (only with MOE_VQLR_FLAG_VALIDATE_INDICES).
+ * The weights stay where they are (borrowed); the one exception is a copy of the DOWN index map
+ * in a slice-major order (same values, at most 1/3 larger), made once here inside the workspace
+ * when the configuration can run its single-token calls as router -> one fused expert kernel ->
+ * weighted sum (Section 4's fused gate/up -> activation -> down pipeline; see
+ * moe_vqlr_workspace_bytes).  Which kernels a call runs (that path, the chain of five kernels, or
+ * the generic chain for shapes the tensor-core kernels do not cover) never changes its results
+ * beyond the summation order; MOE_VQLR_FUSED=0 in the environment at create() keeps the handle
+ * off the fused path. */
 int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out);
 
 /* Runs the layer for T tokens.  x: [T][H] bf16, device.  out: [T][H] bf16, device, written with

@@ -765,7 +765,7 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t bytes = (size_t)T * h->P.H * sizeof(bf16);
   // The kernel chain between the two staging buffers never changes for a given T, so it is
-  // captured once into a graph and replayed: one launch instead of five.
+  // captured once into a graph and replayed: one launch instead of three to six.
   if (!h->host_graph[T] && !h->profiling) {
     cudaError_t ge = cudaSuccess;
     if (!h->cap_stream) ge = cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking);
