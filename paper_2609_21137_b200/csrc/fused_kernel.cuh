@@ -113,37 +113,23 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
   const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
   const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx);
 
-  TRACE_STAMP(3, 0);
-  gu_stage_async<false>(P, x, T, pg, n_books, m);
-  pdl_wait();      // logits and z of this call are complete
-  TRACE_STAMP(3, 1);
-  // One block publishes the routing (slots, affinities, lists) for the weighted sum and the caller:
-  // a block without an item if there is one, else block 0.  For a single token the other blocks
-  // only need the selected experts in id order, which is much shorter to find.
-  const int min_items = (P.k + P.S) * fp.n_sl;          // every token adds at least this many
-  const int writer = (T == 1 && min_items < (int)gridDim.x) ? (int)gridDim.x - 1 : 0;
-  const bool is_writer = (int)blockIdx.x == writer;
-  gu_route(P, T, pg, m, is_writer, want_dbg != 0, T == 1 && !is_writer && P.E <= 1024);
-  TRACE_STAMP(3, 2);
-
-  const int n_grp = *R.n_grp, n_pos = T * (P.k + P.S), n_items = n_grp * fp.n_sl;
-  const int n_dn = (P.H / 8 - warp + kFusedWarps - 1) / kFusedWarps;    // down row tiles of this warp: warp, warp + 12, ...
-
   // One work item as this warp sees it.  Its gate/up units are an even share of the slice units
   // (part-major: consecutive units share their activation fragments) followed by an even share of
   // the cheap low-rank units.
   struct Item {
-    int e, off, cnt, si, tiles, row0, ns, n_my;
+    int e, off, cnt, gi, si, tiles, row0, ns, n_my;
     int sp, st, lp, lt;       // (part, tile) of the first slice unit and of the first low-rank unit of this warp
   };
   struct UnitCur {            // walks the warp's units in order: slice units, then low-rank units
     int i, part, tile;
   };
-  auto load_item = [&](int v) {
+  // The part of an item that does not depend on the routing (everything but the expert and its
+  // pairs) ...
+  auto item_static = [&](int v) {
     Item it;
-    const int gi = fdiv(v, fp.d_nsl);
-    it.si = v - gi * fp.n_sl;
-    it.e = R.grp_e[gi]; it.off = R.grp_off[gi]; it.cnt = R.grp_cnt[gi];
+    it.gi = fdiv(v, fp.d_nsl);
+    it.si = v - it.gi * fp.n_sl;
+    it.e = 0; it.off = 0; it.cnt = 0;
     const bool last_sl = it.si == fp.n_sl - 1;
     it.tiles = last_sl ? fp.t_last : fp.tps;
     const FastDiv d_tiles = last_sl ? fp.d_tlast : fp.d_tps;
@@ -155,6 +141,16 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     it.sp = fdiv(s0, d_tiles); it.st = s0 - it.sp * it.tiles;
     const int lq = fdiv(l0, d_tiles);
     it.lp = pg.n_slices + lq; it.lt = l0 - lq * it.tiles;
+    return it;
+  };
+  Item it = item_static(blockIdx.x);       // before the wait below: it costs a thousand clocks of cold scalar code
+  // ... and the rest, once the work groups are known.
+  auto item_bind = [&](Item& it) {
+    it.e = R.grp_e[it.gi]; it.off = R.grp_off[it.gi]; it.cnt = R.grp_cnt[it.gi];
+  };
+  auto load_item = [&](int v) {
+    Item it = item_static(v);
+    item_bind(it);
     return it;
   };
   auto cur_begin = [&](const Item& it) {
@@ -169,6 +165,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     else if (++u.tile == it.tiles) { u.tile = 0; ++u.part; }
   };
   int g_rq = 0, g_use = 0;             // gate/up ring: next slot to request into, next to consume
+  bool requests_on = true;             // off: the request code runs (and warms the instruction cache) without asking for bytes
   auto gu_request = [&](const Item& it, UnitCur& rq) {                    // requests come in the order of use
     const int part = rq.part, tile = rq.tile;
     cur_next(it, rq);
@@ -177,18 +174,23 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     const size_t row = (size_t)it.e * P.I + it.row0 + tile * 8 + g;
     if (part < pg.n_slices) {
       const int b = part * 32 + 8 * c;
-      if (b < nb) {
+      if (b < nb && requests_on) {
         cp_async_idx8<IdxT>(slot, idx_g + row * nb + b);
         cp_async_idx8<IdxT>(slot + 32, idx_u + row * nb + b);
       }
     } else {
       const int rho = (part - pg.n_slices) * 32 + 8 * c;
-      if (rho < P.r) {
+      if (rho < P.r && requests_on) {
         cp_async16(slot, P.gate.factor + row * P.r + rho);
         cp_async16(slot + 32, P.up.factor + row * P.r + rho);
       }
     }
   };
+
+  TRACE_STAMP(3, 0);
+  gu_stage_async<false>(P, x, T, pg, n_books, m);
+  const int n_pos = T * (P.k + P.S);
+  const int n_dn = (P.H / 8 - warp + kFusedWarps - 1) / kFusedWarps;    // down row tiles of this warp: warp, warp + 12, ...
   // down tile warp + 12 i of the item -> slot `slot` of this warp's down ring
   auto dn_request = [&](const Item& it, int i, int slot_i) {
     const int jt = warp + i * kFusedWarps;
@@ -204,12 +206,41 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
       if (lane * 16 < bytes) cp_async16(slot + lane * 16, src + lane * 16);
     }
   };
-
-  if ((int)blockIdx.x >= n_items) { cp_async_wait_pending(0); return; }
-  Item it = load_item(blockIdx.x);
+  // One block publishes the routing (slots, affinities, lists) for the weighted sum and the caller:
+  // a block without an item if there is one, else block 0.  For a single token the other blocks
+  // only need the selected experts in id order, which is much shorter to find.
+  const int min_items = (P.k + P.S) * fp.n_sl;          // every token adds at least this many
+  const int writer = (T == 1 && min_items < (int)gridDim.x) ? (int)gridDim.x - 1 : 0;
+  const bool is_writer = (int)blockIdx.x == writer;
+  int n_grp = 0, n_items = 0;
   UnitCur rq = cur_begin(it);            // request cursor of the current item (of the next one once its first units are requested)
-  for (int i = 0; i < Dg - 1; ++i) { if (i < it.n_my) gu_request(it, rq); cp_async_commit(); }
+  // The code that binds the item and requests its first units runs twice: a first time while the
+  // router still runs, with the requests switched off, and then for real.  Straight-line code that
+  // a block executes once per call runs at a few instructions per hundred clocks while it is not
+  // in the instruction caches, and this piece sits between the routing and the first bytes.
+#pragma unroll 1
+  for (int pass = 0; pass < 2; ++pass) {
+    if (pass == 1) {
+      pdl_wait();      // logits and z of this call are complete
+      TRACE_STAMP(3, 1);
+      gu_route(P, T, pg, m, is_writer, want_dbg != 0, T == 1 && !is_writer && P.E <= 1024);
+      TRACE_STAMP(3, 2);
+      n_grp = *R.n_grp;
+      n_items = n_grp * fp.n_sl;
+      if ((int)blockIdx.x >= n_items) { cp_async_wait_pending(0); return; }
+    }
+    requests_on = pass == 1;
+    g_rq = 0;
+    item_bind(it);
+    rq = cur_begin(it);
+    for (int i = 0; i < Dg - 1; ++i) {
+      if (i < it.n_my) gu_request(it, rq);
+      if (pass == 1) cp_async_commit();
+    }
+  }
+  TRACE_STAMP(3, 14);
   gu_finish_stage<false>(P, pg, n_books, m, Dg - 1);     // code books, tokens, z, routing lists
+  TRACE_STAMP(3, 15);
   pdl_launch();
 
   for (int v = blockIdx.x; v < n_items; v += gridDim.x) {
