@@ -489,7 +489,7 @@ __device__ void route_light_t1(const Params& P, const RouteSmem& R) {
       const unsigned int key = s_key[e];
       int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
       if ((E & 3) == 0) {
-#pragma unroll 4
+#pragma unroll 8
         for (int e2 = 0; e2 < E; e2 += 4) {
           const uint4 v = *reinterpret_cast<const uint4*>(s_key + e2);
           c0 += (v.x > key) | ((v.x == key) & (e2 < e));
