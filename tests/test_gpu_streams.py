@@ -177,3 +177,20 @@ def test_fused_odd_expert_counts(shp):
     assert_routing(dbg, res)
     assert_output(bf16_tensor_to_f64(out), res.out)
     mod.close()
+
+
+@pytest.mark.parametrize("mode", ["full", "paper"])
+def test_fused_wide_slices(mode):
+    """Slices of 15 row tiles (four k steps in the down product, the widest the fused kernel takes)."""
+    from paper_2609_21137_b200 import binding
+    shp = synth.LayerShape("wide_slices", H=512, I=2048, E=16, k=8, d=8, K=4096, r=64, T=1, mode=mode)
+    layer, res, _ = make_checked_layer(shp, 0)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    x = binding.bits_to_device(layer.x, "cuda")
+    before = mod.launch_count
+    out, dbg = mod.decode(x, debug=True)
+    torch.cuda.synchronize()
+    assert mod.launch_count - before == 3          # the fused path took it
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out)
+    mod.close()
