@@ -194,3 +194,25 @@ def test_fused_wide_slices(mode):
     assert_routing(dbg, res)
     assert_output(bf16_tensor_to_f64(out), res.out)
     mod.close()
+
+
+@pytest.mark.parametrize("mode", ["full", "paper"])
+def test_one_handle_many_batch_sizes(mode):
+    """One handle (max_tokens 16) serves calls of 1, 2, 5, 16 and again 1 tokens: the single-token
+    calls take the fused path, the others the chain, on one workspace."""
+    from paper_2609_21137_b200 import binding
+    import oracle
+    shp = synth.shape("qwen3", E=16, T=16, mode=mode)
+    layer, _, _ = make_checked_layer(shp, 0)
+    orc = oracle.OracleLayer.from_synth(layer)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", max_tokens=16)
+    for T in (1, 2, 5, 16, 1):
+        res = orc.decode_layer(layer.x[:T])
+        x = binding.bits_to_device(layer.x[:T], "cuda")
+        before = mod.launch_count
+        out, dbg = mod.decode(x, debug=True)
+        torch.cuda.synchronize()
+        assert mod.launch_count - before == (3 if T == 1 else 5)
+        assert_routing(dbg, res)
+        assert_output(bf16_tensor_to_f64(out), res.out)
+    mod.close()
