@@ -442,7 +442,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->n_books = gu_vq ? (h->two_books ? 2 : 1) : 0;
     h->plan_gu = plan_stage(I, H, r, gu_dn);
     h->plan_dn = plan_stage(H, I, r, h->dn_dense);
-    if (h->plan_gu.n_lr > 0) h->plan_gu.chunk = h->plan_gu.tiles < 4 ? h->plan_gu.tiles : 4;   // mix slice and low-rank parts
+    if (h->plan_gu.n_lr > 0) h->plan_gu.chunk = h->plan_gu.tiles < 16 ? h->plan_gu.tiles : 16;   // mix slice and low-rank parts
     h->plan_dn.n_parts = h->plan_dn.n_slices;          // the down kernel folds the low-rank groups into the slices
     // shared-memory plan: replicate a small code book eight times (conflict-free lookups), stage the
     // tokens when they fit, then take the deepest rings that still fit
