@@ -33,7 +33,7 @@ constexpr int kFastThreads = 512;
 constexpr int kDenseThreads = 384;   // dense gate/up: weight tiles in flight need more registers per thread
 constexpr int kDownThreads = 384;    // down: hi + lo activation fragments need 64 registers per thread
 constexpr int kGroupTokens = 8;      // tokens of one work group = live rows of the m16 tile
-constexpr int kMaxDepth = 4;
+constexpr int kMaxDepth = 2;
 
 // Phase stamps cost instructions in the tile loops, so they are compiled in only for tracing builds
 // (nvcc -DMOE_VQLR_TRACE); the phase-clock query then returns real data.
