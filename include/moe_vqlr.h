@@ -17,7 +17,7 @@
  *     factor_P[e] * z with z = basis_P * input computed once per token and shared by all
  *     experts (Section 3.2, "z = D^T h"); or W_P,e = dense_P[e] for a projection kept in bf16
  *     (Section 3.1 keeps the down projection uncompressed)
- *   p = silu(W_gate,e x) * (W_up,e x);   y = W_down,e p                      (SwiGLU expert)
+ *   p = phi(W_gate,e x) * (W_up,e x);    y = W_down,e p      (phi = SiLU: SwiGLU expert; or GELU)
  *   out[t] = sum_s a[t][s] * y[t][s]  +  sum over the always-on shared experts of y (weight 1)
  *
  * Symbols: H hidden size, I expert intermediate size, E routed experts, k experts per token,
@@ -72,7 +72,7 @@ enum {
   MOE_VQLR_FLAG_VALIDATE_INDICES = 1u, /* create() scans every index map once and fails with
                                          BAD_INDEX if a value >= K is found (costs one pass
                                          over the index maps; never done on the decode path) */
-  MOE_VQLR_FLAG_PERSISTENT = 2u       /* decode calls run the whole layer as ONE persistent
+  MOE_VQLR_FLAG_PERSISTENT = 2u,      /* decode calls run the whole layer as ONE persistent
                                          cooperative kernel whose phases are separated by
                                          grid-wide barriers (every wait bounded: a barrier
                                          that gives up reports MOE_VQLR_ERR_TIMEOUT through
@@ -81,6 +81,11 @@ enum {
                                          chain on B200, so off by default.  Ignored where the
                                          configuration cannot use it.  The environment
                                          variable MOE_VQLR_COOP=1 at create() sets it too. */
+  MOE_VQLR_FLAG_ACT_GELU_TANH = 4u    /* the expert activation phi of Section 2.1 (it depends
+                                         on the model): p = phi(gate) * up with
+                                         phi(g) = 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3)))
+                                         (the GELU form of GeGLU experts, e.g. the Gemma shape)
+                                         instead of the default phi = SiLU (SwiGLU experts) */
 };
 
 typedef struct {

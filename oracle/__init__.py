@@ -36,9 +36,11 @@ class _Proj(C.Structure):
 class _Layer(C.Structure):
     _fields_ = [("H", C.c_int32), ("I", C.c_int32), ("E", C.c_int32), ("k", C.c_int32),
                 ("S", C.c_int32), ("d", C.c_int32), ("K", C.c_int32), ("r", C.c_int32),
-                ("renorm_topk", C.c_int32), ("router_w", C.c_void_p),
+                ("renorm_topk", C.c_int32), ("act", C.c_int32), ("router_w", C.c_void_p),
                 ("router_bias", C.c_void_p), ("gate", _Proj), ("up", _Proj), ("down", _Proj)]
 
+
+ACTIVATIONS = {"silu": 0, "gelu_tanh": 1}     # ORACLE_ACT_* of the C file
 
 _lib = None
 
@@ -49,6 +51,8 @@ def lib():
         _lib = C.CDLL(build())
         _lib.oracle_threads.restype = C.c_int
         _lib.oracle_decode_layer.restype = C.c_int
+        _lib.oracle_activation.restype = C.c_double
+        _lib.oracle_activation.argtypes = [C.c_double, C.c_int]
         _lib.oracle_reconstruct.restype = C.c_int
         _lib.oracle_storage_bits_per_weight.restype = C.c_double
         _lib.oracle_storage_bits_per_weight.argtypes = [C.c_int] * 10
@@ -81,12 +85,13 @@ class OracleLayer:
     """Holds the arrays of one layer alive and exposes the oracle's steps."""
 
     def __init__(self, *, H, I, E, k, S, d, K, r, router_w, router_bias, gate, up, down,
-                 renorm_topk=True):
+                 renorm_topk=True, act="silu"):
         self.H, self.I, self.E, self.k, self.S, self.d, self.K, self.r = H, I, E, k, S, d, K, r
         self._keep = []
         L = _Layer()
         L.H, L.I, L.E, L.k, L.S, L.d, L.K, L.r = H, I, E, k, S, d, K, r
         L.renorm_topk = 1 if renorm_topk else 0
+        L.act = ACTIVATIONS[act]
         rw = _c(router_w, np.uint16)
         rb = _c(router_bias, np.float32)
         self._keep += [rw, rb]
@@ -114,11 +119,12 @@ class OracleLayer:
         return P
 
     @classmethod
-    def from_synth(cls, layer, renorm_topk=True) -> "OracleLayer":
+    def from_synth(cls, layer, renorm_topk=True, act=None) -> "OracleLayer":
         s = layer.shape
         return cls(H=s.H, I=s.I, E=s.E, k=s.k, S=s.S, d=s.d, K=s.K, r=s.r,
                    router_w=layer.router_w, router_bias=layer.router_bias, gate=layer.gate,
-                   up=layer.up, down=layer.down, renorm_topk=renorm_topk)
+                   up=layer.up, down=layer.down, renorm_topk=renorm_topk,
+                   act=act or getattr(s, "act", "silu"))
 
     # ---- steps -------------------------------------------------------------------------
     def router_logits(self, x_bits: np.ndarray) -> np.ndarray:
@@ -172,6 +178,13 @@ class OracleLayer:
         if rc == 2:
             raise MemoryError("oracle allocation failed")
         return LayerResult(out, logits, ids, w, counts, offsets, ptok, pslot, ypair, rc == 1)
+
+
+def activation(v, act: str = "silu") -> np.ndarray:
+    """The expert activation phi (Section 2.1) applied elementwise."""
+    a = np.atleast_1d(np.asarray(v, dtype=np.float64))
+    f = lib().oracle_activation
+    return np.array([f(float(t), ACTIVATIONS[act]) for t in a.ravel()]).reshape(a.shape)
 
 
 def topk_affinity(logits: np.ndarray, k: int, renorm: bool = True):

@@ -31,6 +31,7 @@
 #endif
 
 enum { ORACLE_PROJ_VQLR = 0, ORACLE_PROJ_DENSE = 1 };
+enum { ORACLE_ACT_SILU = 0, ORACLE_ACT_GELU_TANH = 1 };
 
 typedef struct {
   int32_t kind;
@@ -45,6 +46,7 @@ typedef struct {
 typedef struct {
   int32_t H, I, E, k, S, d, K, r;
   int32_t renorm_topk;        /* 1: affinities are a softmax over the k selected logits */
+  int32_t act;                /* expert activation phi: ORACLE_ACT_SILU or ORACLE_ACT_GELU_TANH */
   const uint16_t* router_w;   /* [E][H] bf16 */
   const float* router_bias;   /* [E] or NULL */
   oracle_proj gate, up, down;
@@ -187,14 +189,29 @@ void oracle_matvec(const double* W, const double* v, int out_dim, int in_dim, do
   }
 }
 
-/* One expert on one token (Section 2.1): g = Wg x, u = Wu x, p = silu(g) * u, y = Wd p,
- * with silu(v) = v / (1 + exp(-v)).  Wd has n_out rows (H, or fewer when rows are sampled). */
-void oracle_swiglu_expert(const double* Wg, const double* Wu, const double* Wd, const double* x,
-                          int H, int I, int n_out, double* g, double* u, double* p, double* y) {
+/* The expert activation phi of Section 2.1, which depends on the model:
+ * SiLU, phi(v) = v / (1 + exp(-v)) (SwiGLU experts), or the tanh form of GELU,
+ * phi(v) = v/2 (1 + tanh(sqrt(2/pi) (v + 0.044715 v^3))) (GeGLU experts). */
+double oracle_activation(double v, int act) {
+  if (act == ORACLE_ACT_GELU_TANH)
+    return 0.5 * v * (1.0 + tanh(sqrt(2.0 / 3.14159265358979323846) * (v + 0.044715 * v * v * v)));
+  return v / (1.0 + exp(-v));
+}
+
+/* One expert on one token (Section 2.1): g = Wg x, u = Wu x, p = phi(g) * u, y = Wd p.
+ * Wd has n_out rows (H, or fewer when rows are sampled). */
+void oracle_gated_expert(const double* Wg, const double* Wu, const double* Wd, const double* x,
+                         int H, int I, int n_out, int act, double* g, double* u, double* p, double* y) {
   oracle_matvec(Wg, x, I, H, g);
   oracle_matvec(Wu, x, I, H, u);
-  for (int i = 0; i < I; ++i) p[i] = g[i] / (1.0 + exp(-g[i])) * u[i];
+  for (int i = 0; i < I; ++i) p[i] = oracle_activation(g[i], act) * u[i];
   oracle_matvec(Wd, p, n_out, I, y);
+}
+
+/* The SwiGLU case, phi = SiLU. */
+void oracle_swiglu_expert(const double* Wg, const double* Wu, const double* Wd, const double* x,
+                          int H, int I, int n_out, double* g, double* u, double* p, double* y) {
+  oracle_gated_expert(Wg, Wu, Wd, x, H, I, n_out, ORACLE_ACT_SILU, g, u, p, y);
 }
 
 /* The whole layer.  Outputs (each may be NULL except out):
@@ -255,8 +272,8 @@ int oracle_decode_layer(const oracle_layer* L, const uint16_t* x, int T, double*
       const int t = shared ? q : pair_token[offsets[e] + q];
       const int slot = shared ? k + (e - E) : pair_slot[offsets[e] + q];
       for (int j = 0; j < H; ++j) xd[j] = bf16_to_double(x[(size_t)t * H + j]);
-      oracle_swiglu_expert(Wg, Wu, Wd, xd, H, I, n_out, g, u, p,
-                           y_pair + ((size_t)t * (k + S) + slot) * n_out);
+      oracle_gated_expert(Wg, Wu, Wd, xd, H, I, n_out, L->act, g, u, p,
+                          y_pair + ((size_t)t * (k + S) + slot) * n_out);
     }
   }
   /* weighted sum in slot order (Section 2.1: scale each selected expert's output by its

@@ -19,6 +19,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_OOM, ERR_TIMEOUT, ERR_BAD_IN
 PROJ_VQLR, PROJ_DENSE_BF16 = 0, 1
 FLAG_VALIDATE_INDICES = 1
 FLAG_PERSISTENT = 2
+FLAG_ACT_GELU_TANH = 4
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",
@@ -152,7 +153,7 @@ class MoeVqlrLayer:
     """
 
     def __init__(self, *, H, I, E, k, S=0, d=8, K=0, r=0, max_tokens=16, router_w, router_bias=None,
-                 gate, up, down, renorm_topk=True, flags=0):
+                 gate, up, down, renorm_topk=True, flags=0, act="silu"):
         self.H, self.I, self.E, self.k, self.S, self.K, self.r = H, I, E, k, S, K, r
         self.max_tokens = max_tokens
         self._keep = [router_w, router_bias, gate, up, down]
@@ -161,7 +162,9 @@ class MoeVqlrLayer:
         cfg.hidden, cfg.inter, cfg.n_experts, cfg.top_k, cfg.n_shared = H, I, E, k, S
         cfg.vq_dim, cfg.codebook_size, cfg.rank, cfg.max_tokens = d, K, r, max_tokens
         cfg.renorm_topk = 1 if renorm_topk else 0
-        cfg.flags = flags
+        if act not in ("silu", "gelu_tanh"):
+            raise ValueError(f"unknown expert activation {act!r}")
+        cfg.flags = flags | (FLAG_ACT_GELU_TANH if act == "gelu_tanh" else 0)
         cfg.router_w = router_w.data_ptr()
         cfg.router_bias = None if router_bias is None else router_bias.data_ptr()
         for name, p in (("gate", gate), ("up", up), ("down", down)):
@@ -199,7 +202,7 @@ class MoeVqlrLayer:
         return cls(H=s.H, I=s.I, E=s.E, k=s.k, S=s.S, d=s.d, K=s.K, r=s.r,
                    max_tokens=max_tokens or max(s.T, 1), router_w=up(layer.router_w),
                    router_bias=up(layer.router_bias), gate=proj(layer.gate), up=proj(layer.up),
-                   down=proj(layer.down), renorm_topk=renorm_topk, flags=flags)
+                   down=proj(layer.down), renorm_topk=renorm_topk, flags=flags, act=s.act)
 
     # -----------------------------------------------------------------------------------
     def _check(self, rc):

@@ -30,6 +30,7 @@ struct ProjDev {
 
 struct Params {
   int H, I, E, k, S, K, r, renorm;
+  int act;                 // expert activation: 0 = SiLU, 1 = GELU (tanh form)
   int n_zrows;             // rows of the stacked basis projection: (distinct gate/up bases) * r
   const bf16* router_w;
   const float* router_bias;
@@ -66,6 +67,16 @@ struct Params {
   long long* clk;          // optional phase stamps [kernel 4][block][warp 16][stamp 16], or NULL
   int clk_blocks;
 };
+
+// The model-specific expert activation phi applied to the gate output (Section 2.1):
+// p = phi(g) * u.  act is uniform over the launch.
+__device__ __forceinline__ float gated_act(float g, float u, int act) {
+  if (act == 1) {
+    const float t = tanhf(0.7978845608028654f * (g + 0.044715f * g * g * g));
+    return 0.5f * g * (1.f + t) * u;
+  }
+  return g / (1.f + expf(-g)) * u;      // silu(g) * u
+}
 
 // Optional tracing: lane 0 of a warp stores clock64() at phase `k` of kernel `kern`.
 __device__ __forceinline__ void stamp(const long long* base_c, int clk_blocks, int kern, int k) {

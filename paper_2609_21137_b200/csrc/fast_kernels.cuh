@@ -1096,7 +1096,7 @@ __device__ __forceinline__ void act_zdown_unit(const Params& P, int n_pos, int n
 #pragma unroll
       for (int q = 0; q < 6; ++q) { g0 += gv[q].x; g1 += gv[q].y; u0 += uv[q].x; u1 += uv[q].y; }
     }
-    const float p0 = g0 / (1.f + expf(-g0)) * u0, p1 = g1 / (1.f + expf(-g1)) * u1;   // silu(g) * u
+    const float p0 = gated_act(g0, u0, P.act), p1 = gated_act(g1, u1, P.act);   // phi(g) * u
     s_p[2 * i2] = p0;
     s_p[2 * i2 + 1] = p1;
     if (zs == 0) {
@@ -1176,7 +1176,7 @@ __global__ void __launch_bounds__(256) k_act(const Params P, int n_pos, int n_pa
 #pragma unroll
       for (int q = 0; q < 6; ++q) { g0 += gv[q].x; g1 += gv[q].y; u0 += uv[q].x; u1 += uv[q].y; }
     }
-    const float p0 = g0 / (1.f + expf(-g0)) * u0, p1 = g1 / (1.f + expf(-g1)) * u1;
+    const float p0 = gated_act(g0, u0, P.act), p1 = gated_act(g1, u1, P.act);
     *reinterpret_cast<float2*>(P.p + base) = make_float2(p0, p1);
     const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);
     *reinterpret_cast<__nv_bfloat162*>(P.p_hi + base) = hi;

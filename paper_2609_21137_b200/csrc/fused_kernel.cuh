@@ -346,7 +346,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     __syncthreads();
     TRACE_STAMP(3, 5);
 
-    // ---- p = silu(gate) * up for the slice's rows; parts added in ascending order -------------
+    // ---- p = phi(gate) * up for the slice's rows; parts added in ascending order -------------
     const int R_here = tiles_here * 8, R_max = fp.tps * 8, RP = 1 << fp.rp_log2;
     for (int idx = tid; idx < cnt * RP; idx += kFusedThreads) {
       const int tk = idx >> fp.rp_log2, row = idx & (RP - 1);
@@ -358,7 +358,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
           gs += src[0];
           us += src[64];
         }
-        const float pv = gs / (1.f + expf(-gs)) * us;
+        const float pv = gated_act(gs, us, P.act);
         s_pf[tk * R_max + row] = pv;
         const bf16 hi = __float2bfloat16_rn(pv);
         reinterpret_cast<bf16*>(s_ph)[(tk * 4 * JD + tile) * 8 + rr] = hi;

@@ -338,7 +338,7 @@ k_gateup(const Params P, const bf16* __restrict__ x, int T, int two_books) {
       for (int tt = 0; tt < kTokGroup; ++tt) {
         const float gs = warp_sum(g[tt]), us = warp_sum(u[tt]);
         if (lane == 0 && tt < nt)
-          P.p[(size_t)(off + q0 + tt) * P.I + i] = gs / (1.f + expf(-gs)) * us;   // silu(g) * u
+          P.p[(size_t)(off + q0 + tt) * P.I + i] = gated_act(gs, us, P.act);   // phi(g) * u
       }
     }
   }

@@ -389,6 +389,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   memset(&P, 0, sizeof P);
   P.H = H; P.I = I; P.E = E; P.k = k; P.S = S; P.K = any_vq ? K : 0; P.r = r;
   P.renorm = cfg->renorm_topk ? 1 : 0;
+  P.act = (cfg->flags & MOE_VQLR_FLAG_ACT_GELU_TANH) ? 1 : 0;
   P.router_w = static_cast<const bf16*>(cfg->router_w);
   P.router_bias = cfg->router_bias;
   P.gate = make_proj(cfg->gate, I, H);
@@ -453,11 +454,15 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->plan_gu.x_smem = 1;
     h->plan_gu.depth = 2;
     if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total > limit) h->plan_gu.x_smem = 0;
-    for (int d = kMaxDepth; d >= 2; --d) {
+    int gu_max_depth = kMaxDepth;
+    if (const char* dv = getenv("MOE_VQLR_GU_DEPTH")) gu_max_depth = atoi(dv);
+    for (int d = gu_max_depth; d >= 2; --d) {
       h->plan_gu.depth = d;
       if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total <= limit) break;
     }
-    for (int d = kMaxDepth; d >= 2; --d) {
+    int dn_max_depth = kMaxDepth;
+    if (const char* dv = getenv("MOE_VQLR_DN_DEPTH")) dn_max_depth = atoi(dv);
+    for (int d = dn_max_depth; d >= 2; --d) {
       h->plan_dn.depth = d;
       if (dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total <= limit) break;
     }

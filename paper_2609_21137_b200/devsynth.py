@@ -55,4 +55,4 @@ def make_device_layer(shp: LayerShape, seed: int, device="cuda") -> dict:
             projs[p] = dict(dense=_normal_bf16(gen, (n_exp, out_dim, in_dim), 0.02, device))
     return dict(H=H, I=I, E=E, k=shp.k, S=S, d=d, K=K if any(vq.values()) else 0, r=r,
                 max_tokens=max(T, 1), router_w=router_w, router_bias=bias, gate=projs["gate"],
-                up=projs["up"], down=projs["down"], x=x)
+                up=projs["up"], down=projs["down"], act=shp.act, x=x)

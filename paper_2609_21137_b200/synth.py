@@ -43,6 +43,7 @@ class LayerShape:
     # "dense": all three dense bf16 (the uncompressed comparison layer)
     mode: str = "full"
     per_projection_codebook: bool = False   # False: one code book aliased by all projections
+    act: str = "silu"                       # expert activation phi: "silu" (SwiGLU) or "gelu_tanh" (GeGLU)
 
     @property
     def idx_dtype(self):
@@ -71,7 +72,7 @@ SHAPES: Dict[str, LayerShape] = {
     "dsv2lite_deployed": LayerShape("dsv2lite_deployed", H=2048, I=1408, E=64, k=6, d=8, K=256, r=384, T=1,
                                     mode="paper", per_projection_codebook=True),
     "gemma4_deployed": LayerShape("gemma4_deployed", H=2816, I=704, E=128, k=8, d=8, K=256, r=384, T=1,
-                                  mode="paper", per_projection_codebook=True),
+                                  mode="paper", per_projection_codebook=True, act="gelu_tanh"),
 }
 
 

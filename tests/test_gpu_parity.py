@@ -102,3 +102,37 @@ def test_repeatable_bitwise():
     torch.cuda.synchronize()
     assert torch.equal(out1.view(torch.int16), out2.view(torch.int16))
     mod.close()
+
+
+@pytest.mark.parametrize("path", ["default", "generic", "fused", "chain", "persistent"])
+@pytest.mark.parametrize("shp", [synth.shape("tiny", T=1, act="gelu_tanh"),
+                                 synth.shape("tiny", T=5, act="gelu_tanh", mode="paper"),
+                                 synth.shape("qwen3", E=16, T=3, act="gelu_tanh")],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
+def test_gelu_expert_activation(shp, path, monkeypatch):
+    """MOE_VQLR_FLAG_ACT_GELU_TANH on every kernel path (the generic kernels, the chain, the fused
+    expert kernel, the persistent kernel): p = gelu_tanh(gate) * up as in the oracle; a path that
+    ignored the flag would miss the tolerance (SiLU and GELU differ by 15 % at gate = 1)."""
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    silu = oracle.OracleLayer.from_synth(layer, act="silu").decode_layer(layer.x)
+    assert np.max(np.abs(silu.out - res.out)) > 0.05 * np.max(np.abs(res.out))
+    kw = {}
+    if path == "generic":
+        monkeypatch.setenv("MOE_VQLR_FORCE_GENERIC", "1")
+    elif path == "fused":
+        monkeypatch.setenv("MOE_VQLR_FUSED", "1")
+    elif path == "chain":
+        monkeypatch.setenv("MOE_VQLR_FUSED", "0")
+    elif path == "persistent":
+        kw["flags"] = binding.FLAG_PERSISTENT
+    mod, (out, dbg) = run_gpu(layer, **kw)
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out, what=f"{shp.name} gelu {path}")
+    mod.close()
+
+
+def test_gelu_long_intermediate():
+    # I > 4096: the activation runs in the wide kernel of the chain
+    shp = synth.LayerShape("longI", H=256, I=4608, E=4, k=2, d=8, K=256, r=16, T=2, act="gelu_tanh")
+    _full_check(shp)

@@ -214,6 +214,44 @@ def test_single_expert_is_plain_swiglu_mlp():
     np.testing.assert_allclose(res.out, ref.numpy(), rtol=0, atol=1e-12)
 
 
+def test_activations_match_library_and_closed_forms():
+    # Section 2.1 leaves the expert activation to the model: SiLU and the tanh form of GELU
+    v = np.concatenate([np.linspace(-12, 12, 97), [0.0, 1e-9, -1e-9, 30.0, -30.0]])
+    tv = torch.from_numpy(v)
+    np.testing.assert_allclose(oracle.activation(v, "silu"), torch.nn.functional.silu(tv).numpy(),
+                               rtol=0, atol=1e-14)
+    np.testing.assert_allclose(oracle.activation(v, "gelu_tanh"),
+                               torch.nn.functional.gelu(tv, approximate="tanh").numpy(), rtol=0, atol=1e-14)
+    for act in ("silu", "gelu_tanh"):
+        a = oracle.activation(v, act)
+        np.testing.assert_allclose(a - oracle.activation(-v, act), v, rtol=0, atol=1e-13)   # phi(v) - phi(-v) = v
+        assert oracle.activation(0.0, act)[0] == 0.0
+        assert abs(oracle.activation(30.0, act)[0] - 30.0) < 1e-9 and abs(oracle.activation(-30.0, act)[0]) < 1e-9
+    # the two differ where it matters (a flag that is ignored must not pass a parity test)
+    assert abs(oracle.activation(1.0, "silu")[0] - 0.7310585786300049) < 1e-15
+    assert abs(oracle.activation(1.0, "gelu_tanh")[0] - 0.8411919906082768) < 1e-13
+    # against the exact GELU v * Phi(v) the tanh form stays within its known 5e-4 error
+    exact = v * 0.5 * (1.0 + torch.erf(tv / np.sqrt(2.0)).numpy())
+    assert np.max(np.abs(oracle.activation(v, "gelu_tanh") - exact)) < 5e-4
+
+
+def test_single_expert_with_gelu_is_plain_geglu_mlp():
+    shp = small_shape(E=1, k=1, T=2, r=3, act="gelu_tanh")
+    layer = synth.make_layer(shp, seed=8)
+    res = oracle.OracleLayer.from_synth(layer).decode_layer(layer.x)
+    W = {}
+    for p in ("gate", "up", "down"):
+        P = getattr(layer, p)
+        W[p] = torch.from_numpy(f64(P.codebook)[P.idx[0].astype(int)].reshape(P.out_dim, P.in_dim)
+                                + f64(P.factor[0]) @ f64(P.basis))
+    xt = torch.from_numpy(f64(layer.x))
+    lin = torch.nn.functional.linear
+    ref = lin(torch.nn.functional.gelu(lin(xt, W["gate"]), approximate="tanh") * lin(xt, W["up"]), W["down"])
+    np.testing.assert_allclose(res.out, ref.numpy(), rtol=0, atol=1e-12)
+    silu = oracle.OracleLayer.from_synth(layer, act="silu").decode_layer(layer.x)
+    assert np.max(np.abs(silu.out - res.out)) > 1e-3 * np.max(np.abs(res.out))
+
+
 # ------------------------------------------------------------------------------------------
 # router, affinities, grouping, combine
 # ------------------------------------------------------------------------------------------
