@@ -73,6 +73,14 @@ SHAPES: Dict[str, LayerShape] = {
                                     mode="paper", per_projection_codebook=True),
     "gemma4_deployed": LayerShape("gemma4_deployed", H=2816, I=704, E=128, k=8, d=8, K=256, r=384, T=1,
                                   mode="paper", per_projection_codebook=True, act="gelu_tanh"),
+    # the d = 8 points of the storage-rate sweep (Section 5.5: K = 256, r chosen for about 3, 4 and
+    # 5 bits per original weight on the Qwen3 shape; r rounded to a multiple of 8)
+    "qwen3_3bit": LayerShape("qwen3_3bit", H=2048, I=768, E=128, k=8, d=8, K=256, r=248, T=1,
+                             mode="paper", per_projection_codebook=True),
+    "qwen3_4bit": LayerShape("qwen3_4bit", H=2048, I=768, E=128, k=8, d=8, K=256, r=376, T=1,
+                             mode="paper", per_projection_codebook=True),
+    "qwen3_5bit": LayerShape("qwen3_5bit", H=2048, I=768, E=128, k=8, d=8, K=256, r=504, T=1,
+                             mode="paper", per_projection_codebook=True),
 }
 
 

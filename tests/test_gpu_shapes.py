@@ -47,7 +47,8 @@ def test_more_slices_than_warps_b16():
     _sampled_check(shp, rows)
 
 
-@pytest.mark.parametrize("name", ["qwen3_deployed", "qwen3_deployed_b16", "gemma4_deployed"])
+@pytest.mark.parametrize("name", ["qwen3_deployed", "qwen3_deployed_b16", "gemma4_deployed", "qwen3_3bit",
+                                  "qwen3_5bit"])
 def test_papers_deployed_operating_points(name):
     # K = 256 / uint8, r = 384 (twelve low-rank parts), separate gate and up code books, bf16 down;
     # fewer experts than the real models to keep the oracle quick (routing width is unchanged)

@@ -214,6 +214,17 @@ def test_single_expert_is_plain_swiglu_mlp():
     np.testing.assert_allclose(res.out, ref.numpy(), rtol=0, atol=1e-12)
 
 
+def test_storage_rate_sweep_shapes_hit_their_rates():
+    # Section 5.5: K = 256, d = 8, r chosen for about 3, 4 and 5 bits per original weight
+    # (here r is a multiple of 8, which moves the 3-bit point 0.022 off its target)
+    for name, target in (("qwen3_3bit", 3.0), ("qwen3_4bit", 4.0), ("qwen3_5bit", 5.0)):
+        s = synth.shape(name)
+        bits = oracle.storage_bits_per_weight(s.d, s.K, s.r, s.H, s.I, s.E)
+        closed = 8 / s.d + 16 * s.r / s.H + 16 * s.r / (s.E * s.I) + 16 * s.K * s.d / (s.E * s.H * s.I)
+        assert abs(bits - closed) < 1e-12
+        assert abs(bits - target) < 0.025, (name, bits)
+
+
 def test_activations_match_library_and_closed_forms():
     # Section 2.1 leaves the expert activation to the model: SiLU and the tanh form of GELU
     v = np.concatenate([np.linspace(-12, 12, 97), [0.0, 1e-9, -1e-9, 30.0, -30.0]])
