@@ -53,6 +53,9 @@ def parse_args():
     ap.add_argument("--mode", default="full", choices=["full", "paper", "dense"])
     ap.add_argument("--layers", type=int, default=0, help="distinct layers to rotate over (0 = auto)")
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary measurements")
+    ap.add_argument("--ablate", default="", choices=["", "z", "launch", "both"],
+                    help="switch a mechanism off (Section 5.4): z = shared projections recomputed per expert, "
+                         "launch = one gate/up and one down launch per work group")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -178,7 +181,7 @@ def run_reference(args):
 class Workload:
     """L distinct layers of one shape on the GPU, with per-layer token batches."""
 
-    def __init__(self, name: str, mode: str, n_layers: int, device):
+    def __init__(self, name: str, mode: str, n_layers: int, device, flags: int = 0):
         import torch
         from paper_2609_21137_b200 import accounting, binding, devsynth, synth
         self.torch = torch
@@ -193,7 +196,7 @@ class Workload:
         for i in range(n_layers):
             kw = devsynth.make_device_layer(shp, seed=1000 + i, device=device)
             x = kw.pop("x")
-            self.layers.append(binding.MoeVqlrLayer(**kw))
+            self.layers.append(binding.MoeVqlrLayer(flags=flags, **kw))
             self.xs.append(x)
             self.outs.append(torch.empty_like(x))
         torch.cuda.synchronize(device)
@@ -351,7 +354,10 @@ def main():
         torch.cuda.synchronize(device)
 
     peak, peak_kind = measured_peak()
-    wl = Workload(args.workload, args.mode, args.layers, device)
+    from paper_2609_21137_b200 import binding as _b
+    ablate_flags = {"": 0, "z": _b.FLAG_ABLATE_Z_PER_EXPERT, "launch": _b.FLAG_ABLATE_PER_EXPERT_LAUNCH,
+                    "both": _b.FLAG_ABLATE_Z_PER_EXPERT | _b.FLAG_ABLATE_PER_EXPERT_LAUNCH}[args.ablate]
+    wl = Workload(args.workload, args.mode, args.layers, device, flags=ablate_flags)
 
     # ---- the timed region: W warm-up steps, then exactly K steps ---------------------------
     wl.prepare(args.steps)
@@ -453,7 +459,8 @@ def main():
                 "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic",
                 "config": {"workload": f"{args.workload} (H={shp.H} I={shp.I} E={shp.E} k={shp.k} S={shp.S} "
-                                       f"K={shp.K} r={shp.r}) T={shp.T} mode={args.mode}",
+                                       f"K={shp.K} r={shp.r}) T={shp.T} mode={args.mode}"
+                                       + (f" ablate={args.ablate}" if args.ablate else ""),
                            "distinct_layers": n_layers,
                            "l2": f"rotation over {n_layers} distinct layers touches "
                                  f"{n_layers * wl.mean_bytes / 1e6:.0f} MB per pass, larger than the 126 MB L2",

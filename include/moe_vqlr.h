@@ -81,11 +81,20 @@ enum {
                                          chain on B200, so off by default.  Ignored where the
                                          configuration cannot use it.  The environment
                                          variable MOE_VQLR_COOP=1 at create() sets it too. */
-  MOE_VQLR_FLAG_ACT_GELU_TANH = 4u    /* the expert activation phi of Section 2.1 (it depends
+  MOE_VQLR_FLAG_ACT_GELU_TANH = 4u,   /* the expert activation phi of Section 2.1 (it depends
                                          on the model): p = phi(gate) * up with
                                          phi(g) = 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3)))
                                          (the GELU form of GeGLU experts, e.g. the Gemma shape)
                                          instead of the default phi = SiLU (SwiGLU experts) */
+  /* The next two switches turn OFF one mechanism each, to measure what it buys (the attribution
+   * of Section 5.4, part A of its table).  Results are unchanged.  They act on the tensor-core
+   * paths; the generic kernels and the persistent kernel ignore them. */
+  MOE_VQLR_FLAG_ABLATE_Z_PER_EXPERT = 8u, /* the shared projections z = basis * x are computed
+                                         once per selected (and shared) expert instead of once
+                                         per token: k + S times the dot products, same values */
+  MOE_VQLR_FLAG_ABLATE_PER_EXPERT_LAUNCH = 16u /* gate/up and down run as one kernel launch per
+                                         work group (expert) instead of one launch over all
+                                         activated experts; implies the chain of kernels */
 };
 
 typedef struct {

@@ -20,6 +20,8 @@ PROJ_VQLR, PROJ_DENSE_BF16 = 0, 1
 FLAG_VALIDATE_INDICES = 1
 FLAG_PERSISTENT = 2
 FLAG_ACT_GELU_TANH = 4
+FLAG_ABLATE_Z_PER_EXPERT = 8
+FLAG_ABLATE_PER_EXPERT_LAUNCH = 16
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",

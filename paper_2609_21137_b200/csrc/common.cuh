@@ -31,6 +31,7 @@ struct ProjDev {
 struct Params {
   int H, I, E, k, S, K, r, renorm;
   int act;                 // expert activation: 0 = SiLU, 1 = GELU (tanh form)
+  int z_repeat;            // 1; ablation: every basis projection is computed this many times (once per selected expert)
   int n_zrows;             // rows of the stacked basis projection: (distinct gate/up bases) * r
   const bf16* router_w;
   const float* router_bias;

@@ -193,6 +193,7 @@ struct StagePlan {
   int repl;        // code book stored eight times, entry i of copy c at slot 8 i + c: lane l reads
                    // copy l % 8, so the eight lanes of a quarter warp never share a bank group
   int W;           // warps of the launch that walks this plan (grid * warps per block)
+  int only_grp;    // -1: the launch walks every work group; >= 0 (ablation): only this one
   int tail;        // tiles % chunk: length of a shorter last chunk (0: none)
   FastDiv d_per_grp, d_per_chunk, d_chunk, d_tail, d_W;   // n_parts*tiles, n_parts*chunk, chunk, tail, W
 };
@@ -533,8 +534,14 @@ __device__ void route_light_t1(const Params& P, const RouteSmem& R) {
 constexpr int kRouterWarps = 2;
 
 // One unit = one (row, group of four tokens); executed by one warp.
-__device__ __forceinline__ int router_z_units(const Params& P, int T) {
+__host__ __device__ __forceinline__ int router_z_units(const Params& P, int T) {
   return (P.E + P.n_zrows) * ((T + kTokGroup - 1) / kTokGroup);
+}
+
+// Units of a k_router_z_pdl launch: with z_repeat > 1 (Section 5.4's variant that recomputes the
+// shared projections for every expert) the basis rows are walked z_repeat times.
+__host__ __device__ __forceinline__ int router_z_units_launched(const Params& P, int T) {
+  return (P.E + P.n_zrows * P.z_repeat) * ((T + kTokGroup - 1) / kTokGroup);
 }
 
 __device__ __forceinline__ void router_z_unit(const Params& P, const bf16* __restrict__ x, int T, int unit, int lane) {
@@ -729,8 +736,13 @@ __device__ __forceinline__ void router_z_unit_row8(const Params& P, const bf16* 
 __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
   pdl_wait();      // the previous call's kernels may still read logits / z
   pdl_launch();
-  const int unit = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
-  if (unit >= router_z_units(P, T)) return;
+  int unit = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
+  const int base_units = router_z_units(P, T);
+  if (unit >= router_z_units_launched(P, T)) return;
+  if (unit >= base_units) {          // ablation: a repeated basis row (same operands, same result, same address)
+    const int n_groups = (T + kTokGroup - 1) / kTokGroup;
+    unit = P.E * n_groups + (unit - base_units) % (P.n_zrows * n_groups);
+  }
   if (T == 1) router_z_unit_t1(P, x, unit, threadIdx.x & 31);
   else if (P.H <= 2048) router_z_unit_row8(P, x, T, unit, threadIdx.x & 31);
   else router_z_unit(P, x, T, unit, threadIdx.x & 31);
@@ -923,10 +935,12 @@ __device__ __forceinline__ void gu_issue(const Params& P, const StagePlan& pl, c
 // requested, each as one cp.async group.
 template <typename IdxT, bool DENSE>
 __device__ __forceinline__ void gu_tiles_begin(const Params& P, const StagePlan& pl, const GuSmem& m, int wid, int W, Walk& w) {
-  const int V = *m.R.n_grp * pl.n_parts * pl.tiles;
+  const int per_grp = pl.n_parts * pl.tiles;
+  int V = *m.R.n_grp * per_grp, v0 = 0;
+  if (pl.only_grp >= 0) { V = pl.only_grp < *m.R.n_grp ? per_grp : 0; v0 = pl.only_grp * per_grp; }
   const int v_begin = split_begin(V, pl, wid);         // W == pl.W by construction of the launch
   w.n_my = split_begin(V, pl, wid + 1) - v_begin;
-  w.pf.set(w.n_my > 0 ? v_begin : 0, pl);
+  w.pf.set(w.n_my > 0 ? v0 + v_begin : 0, pl);
   w.cur = w.pf;
   w.pf_slot = 0; w.cur_slot = 0;
   for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) gu_issue<IdxT, DENSE>(P, pl, m, w); cp_async_commit(); }
@@ -1287,10 +1301,12 @@ __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, c
 // Start of the walk of warp `wid` out of `W` warps (needs only the work groups, not p).
 template <typename IdxT, bool DENSE>
 __device__ __forceinline__ void dn_tiles_begin(const Params& P, const StagePlan& pl, const DnSmem& m, int wid, int W, Walk& w) {
-  const int V = m.n_grp * pl.n_parts * pl.tiles;
+  const int per_grp = pl.n_parts * pl.tiles;
+  int V = m.n_grp * per_grp, v0 = 0;
+  if (pl.only_grp >= 0) { V = pl.only_grp < m.n_grp ? per_grp : 0; v0 = pl.only_grp * per_grp; }
   const int v_begin = split_begin(V, pl, wid);         // W == pl.W by construction of the launch
   w.n_my = split_begin(V, pl, wid + 1) - v_begin;
-  w.pf.set(w.n_my > 0 ? v_begin : 0, pl);
+  w.pf.set(w.n_my > 0 ? v0 + v_begin : 0, pl);
   w.cur = w.pf;
   w.pf_slot = 0; w.cur_slot = 0;
   for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) dn_issue<IdxT, DENSE>(P, pl, m, w); cp_async_commit(); }

@@ -56,6 +56,7 @@ struct moe_vqlr_handle {
   signed char fused_dg[kMaxT + 1], fused_dd[kMaxT + 1];   // ring depths that fit for T tokens (0: the chain runs)
   signed char fused_xs[kMaxT + 1];                        // ... with the tokens staged in shared memory (else read from L2)
   StagePlan plan_gu_fused;
+  bool per_expert_launch;   // ablation: gate/up and down run as one launch per work group
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
   size_t workspace_bytes;
@@ -124,6 +125,7 @@ StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense) {
 // After the last change to a plan: the derived constants of the work-list arithmetic.
 void finish_plan(StagePlan& pl, int W) {
   pl.W = W;
+  pl.only_grp = -1;
   pl.tail = pl.tiles % pl.chunk;
   pl.d_per_grp = make_fastdiv((unsigned int)(pl.n_parts * pl.tiles));
   pl.d_per_chunk = make_fastdiv((unsigned int)(pl.n_parts * pl.chunk));
@@ -194,7 +196,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
   cudaError_t le = cudaSuccess;
   bool ran = false;
   const int n_pos = T * (P.k + P.S);
-  if (h->coop && allow_coop) {
+  if (h->coop && allow_coop && !h->per_expert_launch) {
     if (stage == 0) {
       int zsplit = 1;
       if (!h->dn_dense && P.r > 0) while (n_pos * zsplit * 2 <= 3 * h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
@@ -206,11 +208,11 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
       else le = launch_coop(k_layer_coop<uint16_t, false>, h->sm_count, kCoopThreads, smem, st, P, xb, ob, T, h->plan_gu_coop, h->plan_dn_coop, h->n_books, h->want_dbg, h->dn_restage, zsplit);
       ran = true;
     }
-  } else if (h->fused && T <= h->fused_max_T && (h->fused_forced || T * (P.k + P.S) * h->fplan.n_sl <= h->sm_count)) {
+  } else if (h->fused && !h->per_expert_launch && T <= h->fused_max_T && (h->fused_forced || T * (P.k + P.S) * h->fplan.n_sl <= h->sm_count)) {
     // one wave of (work group, slice) items at most: with more, the chain's finer parts balance better
     switch (stage) {
       case 0:
-        le = launch_pdl(k_router_z_pdl, ((P.E + P.n_zrows) * ((T + kTokGroup - 1) / kTokGroup) + kRouterWarps - 1) / kRouterWarps,
+        le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
                         32 * kRouterWarps, 0, st, P, xb, T);
         ran = true;
         break;
@@ -252,15 +254,23 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
   } else if (h->fast) {
     switch (stage) {
       case 0:
-        le = launch_pdl(k_router_z_pdl, ((P.E + P.n_zrows) * ((T + kTokGroup - 1) / kTokGroup) + kRouterWarps - 1) / kRouterWarps,
+        le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
                         32 * kRouterWarps, 0, st, P, xb, T);
         ran = true;
         break;
       case 2: {
         const size_t smem = gu_layout(P.K, h->n_books, T, P.H, P.r, h->plan_gu, (h->gu_dense ? kDenseThreads : kFastThreads) / 32, P.E, P.k, P.S).total;
-        if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, h->plan_gu, h->n_books, h->want_dbg);
-        else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, h->plan_gu, h->n_books, h->want_dbg);
-        else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, h->plan_gu, h->n_books, h->want_dbg);
+        // one launch over all work groups, or (ablation) one launch per possible work group:
+        // a launch whose group does not exist finds no units after the routing and ends
+        const int n_launch = h->per_expert_launch ? n_pos : 1;
+        for (int gi = 0; gi < n_launch && le == cudaSuccess; ++gi) {
+          StagePlan pl = h->plan_gu;
+          if (h->per_expert_launch) pl.only_grp = gi;
+          if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+        }
+        h->launches += n_launch - 1;
         ran = true;
         break;
       }
@@ -285,12 +295,19 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         ran = true;
         break;
       }
-      case 4:
-        if (h->dn_dense) le = launch_pdl(k_down_mma<uint16_t, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, h->plan_dn);
-        else if (h->idx_bytes == 1) le = launch_pdl(k_down_mma<uint8_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, h->plan_dn);
-        else le = launch_pdl(k_down_mma<uint16_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, h->plan_dn);
+      case 4: {
+        const int n_launch = h->per_expert_launch ? n_pos : 1;
+        for (int gi = 0; gi < n_launch && le == cudaSuccess; ++gi) {
+          StagePlan pl = h->plan_dn;
+          if (h->per_expert_launch) pl.only_grp = gi;
+          if (h->dn_dense) le = launch_pdl(k_down_mma<uint16_t, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else if (h->idx_bytes == 1) le = launch_pdl(k_down_mma<uint8_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else le = launch_pdl(k_down_mma<uint16_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+        }
+        h->launches += n_launch - 1;
         ran = true;
         break;
+      }
       case 5: {
         const int grid = T * ((P.H / 2 + kCombineCols - 1) / kCombineCols);
         le = launch_pdl(k_combine, grid, kCombineCols * kCombineSlots, 0, st, P, ob, T, h->plan_dn.n_parts);
@@ -390,6 +407,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   P.H = H; P.I = I; P.E = E; P.k = k; P.S = S; P.K = any_vq ? K : 0; P.r = r;
   P.renorm = cfg->renorm_topk ? 1 : 0;
   P.act = (cfg->flags & MOE_VQLR_FLAG_ACT_GELU_TANH) ? 1 : 0;
+  P.z_repeat = (cfg->flags & MOE_VQLR_FLAG_ABLATE_Z_PER_EXPERT) ? cfg->top_k + cfg->n_shared : 1;
+  h->per_expert_launch = (cfg->flags & MOE_VQLR_FLAG_ABLATE_PER_EXPERT_LAUNCH) != 0;
   P.router_w = static_cast<const bf16*>(cfg->router_w);
   P.router_bias = cfg->router_bias;
   P.gate = make_proj(cfg->gate, I, H);

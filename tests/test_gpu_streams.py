@@ -216,3 +216,37 @@ def test_one_handle_many_batch_sizes(mode):
         assert_routing(dbg, res)
         assert_output(bf16_tensor_to_f64(out), res.out)
     mod.close()
+
+
+@pytest.mark.parametrize("shp", [synth.shape("tiny", T=1), synth.shape("tiny", T=5, mode="paper"),
+                                 synth.shape("qwen3", E=16, T=1), synth.shape("dsv2lite", E=16, T=3),
+                                 synth.shape("qwen3_deployed", E=24, T=2)],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
+def test_ablation_switches_keep_results(shp):
+    """Section 5.4's mechanism switches: shared projections recomputed per expert, and one launch
+    per work group for gate/up and down.  Both leave routing and outputs as they are; the launch
+    count shows that the per-expert launches really happened."""
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    x = binding.bits_to_device(layer.x, "cuda")
+    n_pos = shp.T * (shp.k + shp.S)
+    base = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    ref_out, _ = base.decode(x, debug=True)
+    torch.cuda.synchronize()
+    for flags in (binding.FLAG_ABLATE_Z_PER_EXPERT, binding.FLAG_ABLATE_PER_EXPERT_LAUNCH,
+                  binding.FLAG_ABLATE_Z_PER_EXPERT | binding.FLAG_ABLATE_PER_EXPERT_LAUNCH):
+        mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=flags)
+        for _ in range(2):
+            before = mod.launch_count
+            out, dbg = mod.decode(x, debug=True)
+            torch.cuda.synchronize()
+            launched = mod.launch_count - before
+            assert_routing(dbg, res)
+            assert_output(bf16_tensor_to_f64(out), res.out)
+        if flags & binding.FLAG_ABLATE_PER_EXPERT_LAUNCH:
+            assert launched >= 3 + 2 * n_pos, launched
+        else:
+            # same kernels, same summation order: bitwise the unswitched result
+            assert torch.equal(out.view(torch.int16), ref_out.view(torch.int16))
+        mod.close()
+    base.close()
