@@ -98,12 +98,13 @@ enum {
 };
 
 typedef struct {
-  int32_t hidden;        /* H, multiple of vq_dim                                              */
-  int32_t inter;         /* I, multiple of vq_dim                                              */
+  int32_t hidden;        /* H, multiple of 8                                                   */
+  int32_t inter;         /* I, multiple of 8                                                   */
   int32_t n_experts;     /* E >= 1                                                             */
   int32_t top_k;         /* 1 <= k <= E, k <= 32                                               */
   int32_t n_shared;      /* S >= 0                                                             */
-  int32_t vq_dim;        /* d, must be 8                                                       */
+  int32_t vq_dim;        /* d: 8, or 4 (Section 5.5's shorter vectors: code words of 4 bf16,
+                            two indices per 8 weights; tensor-core chain for K <= 256, K even) */
   int32_t codebook_size; /* K, 1..65536                                                        */
   int32_t rank;          /* r >= 0                                                             */
   int32_t max_tokens;    /* largest T a call may pass, 1..16                                   */
@@ -130,7 +131,7 @@ typedef struct {
 
 /* Validates the configuration, allocates the handle and its device workspace on the CURRENT
  * CUDA device and returns the handle in *out (NULL on failure).  Synchronous.
- * Errors: INVALID_ARG, UNSUPPORTED (vq_dim != 8, H or I not a multiple of 8, K > 65536, k > 32,
+ * Errors: INVALID_ARG, UNSUPPORTED (vq_dim not 8 or 4, H or I not a multiple of 8, K > 65536, k > 32,
  * max_tokens > 16), OOM, CUDA, BAD_INDEX (only with MOE_VQLR_FLAG_VALIDATE_INDICES).
  * The weights stay where they are (borrowed); the one exception is a copy of the DOWN index map
  * in a slice-major order (same values, at most 1/3 larger), made once here inside the workspace

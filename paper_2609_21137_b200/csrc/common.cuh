@@ -21,7 +21,7 @@ struct ProjDev {
   int kind;
   int out_dim, in_dim;
   int zslot;               // which z slot feeds the low-rank term (gate/up), -1 if none
-  const uint4* codebook;   // [K] code words of 8 bf16
+  const uint4* codebook;   // [K] code words of 8 bf16 (d = 4: [K] words of 4 bf16, read as uint2)
   const void* idx;
   const bf16* basis;
   const bf16* factor;
@@ -31,6 +31,7 @@ struct ProjDev {
 struct Params {
   int H, I, E, k, S, K, r, renorm;
   int act;                 // expert activation: 0 = SiLU, 1 = GELU (tanh form)
+  int d;                   // VQ block length: 8 (one code word = 16 bytes) or 4 (8 bytes)
   int z_repeat;            // 1; ablation: every basis projection is computed this many times (once per selected expert)
   int n_zrows;             // rows of the stacked basis projection: (distinct gate/up bases) * r
   const bf16* router_w;

@@ -159,6 +159,16 @@ __device__ __forceinline__ uint4 ring_idx8(const uint4* smem) {
   return make_uint4(v.x, v.y, 0u, 0u);
 }
 
+// Four-value code words (d = 4): a row's uint8 indices are read two at a time as one 16-bit
+// pair (low byte = first word), i.e. with the uint16 plumbing, and the eight weights of a block are
+// two 8-byte words.  The book is stored sixteen times, word i of copy c at 8-byte slot 16 i + c:
+// lane l reads copy l % 16, so the sixteen lanes of a half warp never share a bank pair.
+__device__ __forceinline__ uint4 lookup_d4(const uint4* s_cb, uint32_t pair, int lane) {
+  const uint2* cb2 = reinterpret_cast<const uint2*>(s_cb);
+  const uint2 lo = cb2[((pair & 0xffu) << 4) | (lane & 15)], hi = cb2[((pair >> 8) << 4) | (lane & 15)];
+  return make_uint4(lo.x, lo.y, hi.x, hi.y);
+}
+
 // Division by a run-time constant as multiply-high and shift (the magic numbers come from the
 // host): exact for 0 <= n < 2^31.  A hardware-emulated 32-bit division costs about a hundred
 // clocks of dependent instructions, and the work-list arithmetic below sits on the critical path
@@ -830,16 +840,17 @@ __device__ __forceinline__ void gu_stage_books_async(const Params& P, const Stag
     // Every block fetches the same few KB from L2: each starts at its own offset, so that at any
     // moment the blocks ask for different lines (all asking for the same lines in the same order
     // serialises on single L2 slices: 5 us instead of 1-2 for 64 KB x 148 blocks).
-    const int rot = (int)(((unsigned int)blockIdx.x * (unsigned int)P.K) / gridDim.x);
-    for (int i = tid; i < P.K; i += blockDim.x) {
+    const int kw = P.d == 8 ? P.K : P.K / 2;      // 16-byte pieces of one book
+    const int rot = (int)(((unsigned int)blockIdx.x * (unsigned int)kw) / gridDim.x);
+    for (int i = tid; i < kw; i += blockDim.x) {
       int j = i + rot;
-      if (j >= P.K) j -= P.K;
+      if (j >= kw) j -= kw;
       cp_async16(dst_g + j, P.gate.codebook + j);
     }
     if (n_books == 2)
-      for (int i = tid; i < P.K; i += blockDim.x) {
+      for (int i = tid; i < kw; i += blockDim.x) {
         int j = i + rot;
-        if (j >= P.K) j -= P.K;
+        if (j >= kw) j -= kw;
         cp_async16(dst_u + j, P.up.codebook + j);
       }
   }
@@ -889,9 +900,20 @@ __device__ __forceinline__ void gu_finish_stage(const Params& P, const StagePlan
   __syncthreads();                // ... and so has everybody else's (and z, and the routing lists)
   TRACE_STAMP(1, 6);
   if (!DENSE && pl.repl) {
-    for (int i = tid; i < P.K * 8; i += blockDim.x) {
-      m.cb_g[i] = m.tmp[i >> 3];
-      if (n_books == 2) m.cb_u[i] = m.tmp[P.K + (i >> 3)];
+    if (P.d == 8) {
+      for (int i = tid; i < P.K * 8; i += blockDim.x) {
+        m.cb_g[i] = m.tmp[i >> 3];
+        if (n_books == 2) m.cb_u[i] = m.tmp[P.K + (i >> 3)];
+      }
+    } else {                        // sixteen copies of the 8-byte words
+      uint2* g2 = reinterpret_cast<uint2*>(m.cb_g);
+      uint2* u2 = reinterpret_cast<uint2*>(m.cb_u);
+      const uint2* tg = reinterpret_cast<const uint2*>(m.tmp);
+      const uint2* tu = reinterpret_cast<const uint2*>(m.tmp + P.K);
+      for (int i = tid; i < P.K * 16; i += blockDim.x) {
+        g2[i] = tg[i >> 4];
+        if (n_books == 2) u2[i] = tu[i >> 4];
+      }
     }
     __syncthreads();
   }
@@ -948,7 +970,7 @@ __device__ __forceinline__ void gu_tiles_begin(const Params& P, const StagePlan&
 }
 
 // The tile loop proper (needs code books, tokens and z in shared memory).
-template <typename IdxT, bool DENSE>
+template <typename IdxT, bool DENSE, bool D4 = false>
 __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
                                              const GuSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
@@ -1017,7 +1039,13 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
         uint32_t ig[8], iu[8];
         unpack_idx8<IdxT>(raw_g, ig);
         unpack_idx8<IdxT>(raw_u, iu);
-        if (pl.repl) {
+        if (D4) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            mma_block(acc_g[j & 1], fx[j], lookup_d4(s_cb_g, ig[j], lane));
+            mma_block(acc_u[j & 1], fx[j], lookup_d4(s_cb_u, iu[j], lane));
+          }
+        } else if (pl.repl) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             mma_block(acc_g[j & 1], fx[j], s_cb_g[(ig[j] << 3) | (lane & 7)]);
@@ -1061,7 +1089,7 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
   TRACE_STAMP(0, 15);
 }
 
-template <typename IdxT, bool DENSE>
+template <typename IdxT, bool DENSE, bool D4 = false>
 __global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
 k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {
   extern __shared__ uint4 s_u4[];
@@ -1079,7 +1107,7 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   gu_finish_stage<DENSE>(P, pl, n_books, m, pl.depth - 1);                                     // ... while the stage settles
   pdl_launch();
   TRACE_STAMP(0, 3);
-  gu_tiles_run<IdxT, DENSE>(P, x, T, pl, m, w);
+  gu_tiles_run<IdxT, DENSE, D4>(P, x, T, pl, m, w);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1314,7 +1342,7 @@ __device__ __forceinline__ void dn_tiles_begin(const Params& P, const StagePlan&
 }
 
 // The tile loop proper (needs p, z_d and the code book).
-template <typename IdxT, bool DENSE>
+template <typename IdxT, bool DENSE, bool D4 = false>
 __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const StagePlan& pl, const DnSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
   const int nb = pl.nb, D = pl.depth;
@@ -1376,7 +1404,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
       unpack_idx8<IdxT>(raw, id);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const uint4 w = s_cb[pl.repl ? ((id[j] << 3) | (lane & 7)) : id[j]];
+        const uint4 w = D4 ? lookup_d4(s_cb, id[j], lane) : s_cb[pl.repl ? ((id[j] << 3) | (lane & 7)) : id[j]];
         mma_block_hilo(acc[j & 1], fh[j], fl[j], w);      // hi product in rows 0..7 of the tile, lo in rows 8..15
       }
       if (part < pl.n_lr) {                   // warp-uniform: the low-rank group carried by this part
@@ -1409,7 +1437,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
   TRACE_STAMP(2, 15);
 }
 
-template <typename IdxT, bool DENSE>
+template <typename IdxT, bool DENSE, bool D4 = false>
 __global__ void __launch_bounds__(kDownThreads, 1)
 k_down_mma(const Params P, int T, const StagePlan pl) {
   extern __shared__ uint4 s_u4[];
@@ -1427,7 +1455,8 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   uint4* s_tmp = reinterpret_cast<uint4*>(s_base + L.cb_tmp);
   if (!DENSE) {
     uint4* dst = pl.repl ? s_tmp : s_cb;
-    for (int i = tid; i < P.K; i += blockDim.x) cp_async16(dst + i, P.down.codebook + i);
+    const int kw = D4 ? P.K / 2 : P.K;
+    for (int i = tid; i < kw; i += blockDim.x) cp_async16(dst + i, P.down.codebook + i);
   }
   cp_async_commit();
   pdl_wait();      // p (and z_d) and the routing lists are complete
@@ -1446,11 +1475,17 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   cp_async_wait_pending(D - 1);                                                                // ... the code book has landed
   __syncthreads();
   if (!DENSE && pl.repl) {
-    for (int i = tid; i < P.K * 8; i += blockDim.x) s_cb[i] = s_tmp[i >> 3];
+    if (D4) {
+      uint2* c2 = reinterpret_cast<uint2*>(s_cb);
+      const uint2* t2 = reinterpret_cast<const uint2*>(s_tmp);
+      for (int i = tid; i < P.K * 16; i += blockDim.x) c2[i] = t2[i >> 4];
+    } else {
+      for (int i = tid; i < P.K * 8; i += blockDim.x) s_cb[i] = s_tmp[i >> 3];
+    }
     __syncthreads();
   }
   TRACE_STAMP(2, 2);
-  dn_tiles_run<IdxT, DENSE>(P, T, pl, m, w);
+  dn_tiles_run<IdxT, DENSE, D4>(P, T, pl, m, w);
 }
 
 // out[t][h] = sum over slots (in slot order) of affinity * y[t][slot][h], where y is the sum of

@@ -85,7 +85,7 @@ __global__ void k_relay_down_idx(const IdxT* __restrict__ src, IdxT* __restrict_
 
 // JD = k steps of the down product (a compile-time constant: the down loop is bound by
 // instruction issue, and with JD known its predicates and index unpacking fold away).
-template <typename IdxT, bool DN_DENSE, int JD>
+template <typename IdxT, bool DN_DENSE, int JD, bool D4 = false>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePlan pg, const FusedPlan fp, int n_books,
                int want_dbg, const IdxT* __restrict__ idx_dp) {
@@ -292,7 +292,13 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
           uint32_t ig[8], iu[8];
           unpack_idx8<IdxT>(raw_g, ig);
           unpack_idx8<IdxT>(raw_u, iu);
-          if (pg.repl) {
+          if (D4) {                   // four-value code words: two 8-byte reads per block
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              mma_block(acc_g[j & 1], fx[j], lookup_d4(m.cb_g, ig[j], lane));
+              mma_block(acc_u[j & 1], fx[j], lookup_d4(m.cb_u, iu[j], lane));
+            }
+          } else if (pg.repl) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               mma_block(acc_g[j & 1], fx[j], m.cb_g[(ig[j] << 3) | (lane & 7)]);
@@ -457,7 +463,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
           for (int j = 0; j < JD; ++j) {
 #pragma unroll
             for (int u = 0; u < kU; ++u) {       // every lane runs every mma
-              const uint4 w = pg.repl ? s_cb_d[(id[u][j] << 3) | (lane & 7)] : s_cb_d[id[u][j]];
+              const uint4 w = D4 ? lookup_d4(s_cb_d, id[u][j], lane) : pg.repl ? s_cb_d[(id[u][j] << 3) | (lane & 7)] : s_cb_d[id[u][j]];
               mma_block_hilo(acc[u], fh[j], fl[j], w);
             }
           }

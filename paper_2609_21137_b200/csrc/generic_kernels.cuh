@@ -202,15 +202,36 @@ __device__ __forceinline__ void load_idx8<uint8_t>(const uint8_t* p, uint32_t (&
   id[4] = v.y & 0xffu; id[5] = (v.y >> 8) & 0xffu; id[6] = (v.y >> 16) & 0xffu; id[7] = v.y >> 24;
 }
 
-// VQ part of one row against up to kTokGroup bf16 activation rows held (swizzled) in shared
-// memory.  nb = blocks per row.
+// The eight weights of 8-value block b of a row: one code word (d = 8) or two consecutive
+// 4-value code words (d = 4, Section 5.5's shorter vectors: the row then has two indices per block).
 template <typename IdxT>
-__device__ __forceinline__ void vq_row_bf16x(const IdxT* __restrict__ idx_row, int nb,
+__device__ __forceinline__ uint4 row_block8(const IdxT* __restrict__ idx_row, int b, const uint4* __restrict__ s_cb, int d) {
+  if (d == 8) return s_cb[idx_row[b]];
+  const uint2* cb2 = reinterpret_cast<const uint2*>(s_cb);
+  const uint2 lo = cb2[idx_row[2 * b]], hi = cb2[idx_row[2 * b + 1]];
+  return make_uint4(lo.x, lo.y, hi.x, hi.y);
+}
+
+// Code book of a projection into shared memory (K words of 2 d bytes).
+__device__ __forceinline__ void stage_codebook(uint4* dst, const uint4* __restrict__ src, int K, int d) {
+  if (d == 8) {
+    for (int i = threadIdx.x; i < K; i += blockDim.x) dst[i] = __ldg(src + i);
+  } else {
+    uint2* d2 = reinterpret_cast<uint2*>(dst);
+    const uint2* s2 = reinterpret_cast<const uint2*>(src);
+    for (int i = threadIdx.x; i < K; i += blockDim.x) d2[i] = __ldg(s2 + i);
+  }
+}
+
+// VQ part of one row against up to kTokGroup bf16 activation rows held (swizzled) in shared
+// memory.  nb = 8-value blocks per row.
+template <typename IdxT>
+__device__ __forceinline__ void vq_row_bf16x(const IdxT* __restrict__ idx_row, int nb, int d,
                                              const uint4* __restrict__ s_cb,
                                              const uint4* __restrict__ s_x, int x_stride,
                                              const int (&tok)[kTokGroup], int nt,
                                              float (&acc)[kTokGroup], int lane) {
-  if ((nb & 7) == 0) {
+  if (d == 8 && (nb & 7) == 0) {
     for (int c = lane; c < (nb >> 3); c += 32) {
       uint32_t id[8];
       load_idx8<IdxT>(idx_row + c * 8, id);
@@ -231,7 +252,7 @@ __device__ __forceinline__ void vq_row_bf16x(const IdxT* __restrict__ idx_row, i
   } else {   // rows whose index run is not a multiple of eight blocks: one index at a time
     for (int b0 = lane; b0 < nb; b0 += 32) {
       float wf[8];
-      unpack8(s_cb[idx_row[b0]], wf);
+      unpack8(row_block8<IdxT>(idx_row, b0, s_cb, d), wf);
       const int b = swz(b0);
 #pragma unroll
       for (int tt = 0; tt < kTokGroup; ++tt)
@@ -290,9 +311,8 @@ k_gateup(const Params P, const bf16* __restrict__ x, int T, int two_books) {
 
   if (n_cb) {
     const uint4* src_g = P.gate.kind == MOE_VQLR_PROJ_VQLR ? P.gate.codebook : P.up.codebook;
-    for (int i = threadIdx.x; i < P.K; i += blockDim.x) s_cb_g[i] = __ldg(src_g + i);
-    if (two_books)
-      for (int i = threadIdx.x; i < P.K; i += blockDim.x) s_cb_u[i] = __ldg(P.up.codebook + i);
+    stage_codebook(s_cb_g, src_g, P.K, P.d);
+    if (two_books) stage_codebook(s_cb_u, P.up.codebook, P.K, P.d);
   }
   const int xs = (nbH + 7) & ~7;   // row stride in blocks: the swizzle permutes within groups of 8
   const uint4* x4 = reinterpret_cast<const uint4*>(x);
@@ -319,7 +339,7 @@ k_gateup(const Params P, const bf16* __restrict__ x, int T, int two_books) {
       for (int tt = 0; tt < kTokGroup; ++tt) tok[tt] = tt < nt ? P.pair_token[off + q0 + tt] : 0;
       float g[kTokGroup] = {0.f, 0.f, 0.f, 0.f}, u[kTokGroup] = {0.f, 0.f, 0.f, 0.f};
       if (P.gate.kind == MOE_VQLR_PROJ_VQLR) {
-        vq_row_bf16x<IdxT>(static_cast<const IdxT*>(P.gate.idx) + row * nbH, nbH, s_cb_g, s_x, xs,
+        vq_row_bf16x<IdxT>(static_cast<const IdxT*>(P.gate.idx) + row * (P.H / P.d), nbH, P.d, s_cb_g, s_x, xs,
                            tok, nt, g, lane);
         if (P.gate.zslot >= 0)
           lr_row(P.gate.factor + row * P.r, P.r, P.z + P.gate.zslot * P.r, 2 * P.r, tok, nt, g, lane);
@@ -327,7 +347,7 @@ k_gateup(const Params P, const bf16* __restrict__ x, int T, int two_books) {
         dense_row_bf16x(P.gate.dense + row * P.H, nbH, s_x, xs, tok, nt, g, lane);
       }
       if (P.up.kind == MOE_VQLR_PROJ_VQLR) {
-        vq_row_bf16x<IdxT>(static_cast<const IdxT*>(P.up.idx) + row * nbH, nbH, s_cb_u, s_x, xs,
+        vq_row_bf16x<IdxT>(static_cast<const IdxT*>(P.up.idx) + row * (P.H / P.d), nbH, P.d, s_cb_u, s_x, xs,
                            tok, nt, u, lane);
         if (P.up.zslot >= 0)
           lr_row(P.up.factor + row * P.r, P.r, P.z + P.up.zslot * P.r, 2 * P.r, tok, nt, u, lane);
@@ -369,8 +389,7 @@ k_down(const Params P, bf16* __restrict__ out, int T) {
   uint4* s_cb = s_u4;
   const bool vq = P.down.kind == MOE_VQLR_PROJ_VQLR;
   float* s_acc = reinterpret_cast<float*>(s_u4 + (vq ? P.K : 0));   // [warps][kMaxT]
-  if (vq)
-    for (int i = threadIdx.x; i < P.K; i += blockDim.x) s_cb[i] = __ldg(P.down.codebook + i);
+  if (vq) stage_codebook(s_cb, P.down.codebook, P.K, P.d);
   for (int i = threadIdx.x; i < (blockDim.x >> 5) * kMaxT; i += blockDim.x) s_acc[i] = 0.f;
   __syncthreads();
 
@@ -389,8 +408,8 @@ k_down(const Params P, bf16* __restrict__ out, int T) {
         const float* prow = P.p + (size_t)pos * P.I;
         float acc = 0.f;
         if (vq) {
-          const IdxT* idx_row = static_cast<const IdxT*>(P.down.idx) + row * nbI;
-          if ((nbI & 7) == 0) {
+          const IdxT* idx_row = static_cast<const IdxT*>(P.down.idx) + row * (P.I / P.d);
+          if (P.d == 8 && (nbI & 7) == 0) {
             for (int c = lane; c < (nbI >> 3); c += 32) {
               uint32_t id[8];
               load_idx8<IdxT>(idx_row + c * 8, id);
@@ -407,7 +426,7 @@ k_down(const Params P, bf16* __restrict__ out, int T) {
           } else {
             for (int b = lane; b < nbI; b += 32) {
               float wf[8];
-              unpack8(s_cb[idx_row[b]], wf);
+              unpack8(row_block8<IdxT>(idx_row, b, s_cb, P.d), wf);
               const float4 p0 = *reinterpret_cast<const float4*>(prow + b * 8);
               const float4 p1 = *reinterpret_cast<const float4*>(prow + b * 8 + 4);
               const float pf[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};

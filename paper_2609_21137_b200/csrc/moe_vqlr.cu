@@ -57,6 +57,8 @@ struct moe_vqlr_handle {
   signed char fused_xs[kMaxT + 1];                        // ... with the tokens staged in shared memory (else read from L2)
   StagePlan plan_gu_fused;
   bool per_expert_launch;   // ablation: gate/up and down run as one launch per work group
+  bool d4;                  // four-value code words on the tensor-core paths (uint8 indices read as pairs)
+  int idx_tc;               // bytes per index element as the tensor-core kernels read it (2 with d4)
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
   size_t workspace_bytes;
@@ -222,21 +224,23 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         fpl.depth_d = h->fused_dd[T];
         StagePlan pgl = h->plan_gu_fused;
         pgl.x_smem = h->fused_xs[T];
-        const size_t smem2 = fused_layout(P.K, h->n_books, T, P.H, P.r, pgl, fpl, h->dn_dense, h->idx_bytes, P.E, P.k, P.S).total;
-#define MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, JDV)                                                                       \
-  le = launch_pdl(k_expert_fused<IDXT, DENSE, JDV>, h->sm_count, kFusedThreads, smem2, st, P, xb, T, pgl, fpl, h->n_books, \
+        const size_t smem2 = fused_layout(P.K, h->n_books, T, P.H, P.r, pgl, fpl, h->dn_dense, h->idx_tc, P.E, P.k, P.S).total;
+#define MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, JDV, D4V)                                                                  \
+  le = launch_pdl(k_expert_fused<IDXT, DENSE, JDV, D4V>, h->sm_count, kFusedThreads, smem2, st, P, xb, T, pgl, fpl, h->n_books, \
                   h->want_dbg, static_cast<const IDXT*>(DENSE ? nullptr : h->idx_dp))
-#define MOE_VQLR_FUSED_JD(IDXT, DENSE)                                  \
-  switch (fpl.jd) {                                                     \
-    case 1: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 1); break;               \
-    case 2: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 2); break;               \
-    case 3: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 3); break;               \
-    default: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 4); break;              \
+#define MOE_VQLR_FUSED_JD(IDXT, DENSE, D4V)                                  \
+  switch (fpl.jd) {                                                          \
+    case 1: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 1, D4V); break;               \
+    case 2: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 2, D4V); break;               \
+    case 3: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 3, D4V); break;               \
+    default: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 4, D4V); break;              \
   }
-        if (h->dn_dense && h->idx_bytes == 1) { MOE_VQLR_FUSED_JD(uint8_t, true) }
-        else if (h->dn_dense) { MOE_VQLR_FUSED_JD(uint16_t, true) }
-        else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_JD(uint8_t, false) }
-        else { MOE_VQLR_FUSED_JD(uint16_t, false) }
+        if (h->d4 && h->dn_dense) { MOE_VQLR_FUSED_JD(uint16_t, true, true) }
+        else if (h->d4) { MOE_VQLR_FUSED_JD(uint16_t, false, true) }
+        else if (h->dn_dense && h->idx_bytes == 1) { MOE_VQLR_FUSED_JD(uint8_t, true, false) }
+        else if (h->dn_dense) { MOE_VQLR_FUSED_JD(uint16_t, true, false) }
+        else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_JD(uint8_t, false, false) }
+        else { MOE_VQLR_FUSED_JD(uint16_t, false, false) }
 #undef MOE_VQLR_FUSED_JD
 #undef MOE_VQLR_FUSED_LAUNCH
         ran = true;
@@ -267,6 +271,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           StagePlan pl = h->plan_gu;
           if (h->per_expert_launch) pl.only_grp = gi;
           if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->d4) le = launch_pdl(k_gateup_mma<uint16_t, false, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
           else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
           else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
         }
@@ -301,6 +306,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           StagePlan pl = h->plan_dn;
           if (h->per_expert_launch) pl.only_grp = gi;
           if (h->dn_dense) le = launch_pdl(k_down_mma<uint16_t, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else if (h->d4) le = launch_pdl(k_down_mma<uint16_t, false, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
           else if (h->idx_bytes == 1) le = launch_pdl(k_down_mma<uint8_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
           else le = launch_pdl(k_down_mma<uint16_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
         }
@@ -368,7 +374,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   if (k > E) return fail(nullptr, MOE_VQLR_ERR_INVALID_ARG, "top_k %d > n_experts %d", k, E);
   if (!cfg->router_w || !aligned16(cfg->router_w))
     return fail(nullptr, MOE_VQLR_ERR_INVALID_ARG, "router_w null or not 16-byte aligned");
-  if (cfg->vq_dim != kD) return fail(nullptr, MOE_VQLR_ERR_UNSUPPORTED, "vq_dim must be 8");
+  if (cfg->vq_dim != kD && cfg->vq_dim != 4) return fail(nullptr, MOE_VQLR_ERR_UNSUPPORTED, "vq_dim must be 8 or 4");
   if (H % kD || I % kD) return fail(nullptr, MOE_VQLR_ERR_UNSUPPORTED, "hidden and inter must be multiples of 8");
   if (k > kMaxK) return fail(nullptr, MOE_VQLR_ERR_UNSUPPORTED, "top_k > %d", kMaxK);
   if (maxT > kMaxT) return fail(nullptr, MOE_VQLR_ERR_UNSUPPORTED, "max_tokens > %d", kMaxT);
@@ -407,6 +413,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   P.H = H; P.I = I; P.E = E; P.k = k; P.S = S; P.K = any_vq ? K : 0; P.r = r;
   P.renorm = cfg->renorm_topk ? 1 : 0;
   P.act = (cfg->flags & MOE_VQLR_FLAG_ACT_GELU_TANH) ? 1 : 0;
+  P.d = cfg->vq_dim;
   P.z_repeat = (cfg->flags & MOE_VQLR_FLAG_ABLATE_Z_PER_EXPERT) ? cfg->top_k + cfg->n_shared : 1;
   h->per_expert_launch = (cfg->flags & MOE_VQLR_FLAG_ABLATE_PER_EXPERT_LAUNCH) != 0;
   P.router_w = static_cast<const bf16*>(cfg->router_w);
@@ -455,6 +462,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->gu_dense = gu_dn;
     h->dn_dense = P.down.kind == MOE_VQLR_PROJ_DENSE_BF16;
     bool ok = gu_vq || gu_dn;
+    const bool d4 = any_vq && cfg->vq_dim == 4;       // four-value code words: uint8 indices only, an even K
+    if (d4 && (K > 256 || (K & 1))) ok = false;
     if (gu_vq && (H % 64 != 0 || (r % 8) != 0)) ok = false;       // whole groups of eight blocks / ranks
     if (!h->dn_dense && (I % 64 != 0 || (r % 8) != 0)) ok = false;
     if (gu_vq && r > 0 && (P.gate.zslot < 0 || P.up.zslot < 0)) ok = false;
@@ -470,6 +479,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     const int gu_warps = (gu_dn ? kDenseThreads : kFastThreads) / 32;
     h->plan_gu.repl = (gu_vq && (size_t)K * 128 * h->n_books <= 72 * 1024) ? 1 : 0;
     h->plan_dn.repl = (!h->dn_dense && (size_t)K * 128 <= 72 * 1024) ? 1 : 0;
+    if (d4 && ((gu_vq && !h->plan_gu.repl) || (!h->dn_dense && !h->plan_dn.repl))) ok = false;
     h->plan_gu.x_smem = 1;
     h->plan_gu.depth = 2;
     if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total > limit) h->plan_gu.x_smem = 0;
@@ -493,13 +503,17 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     const char* force = getenv("MOE_VQLR_FORCE_GENERIC");
     if (force && force[0] == '1') ok = false;
     h->fast = ok;
+    h->d4 = ok && d4;
+    h->idx_tc = h->d4 ? 2 : h->idx_bytes;
     if (ok) {
       cudaError_t e1 = cudaSuccess, e2 = cudaSuccess;
       const int a = cudaFuncAttributeMaxDynamicSharedMemorySize;
       if (gu_dn) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (d4) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true>, (cudaFuncAttribute)a, (int)smem_gu);
       else if (h->idx_bytes == 1) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
       else e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
       if (h->dn_dense) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
+      else if (d4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
       else if (h->idx_bytes == 1) e2 = cudaFuncSetAttribute(k_down_mma<uint8_t, false>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
       else e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
       cudaError_t e3 = cudaFuncSetAttribute(k_act_zdown, (cudaFuncAttribute)a, (int)((size_t)I * sizeof(float)));
@@ -516,7 +530,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     int coop_attr = 0;
     cudaDeviceGetAttribute(&coop_attr, cudaDevAttrCooperativeLaunch, h->device);
     const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) || (coop_env && coop_env[0] == '1');
-    if (h->fast && !h->gu_dense && coop_attr && want_coop) {
+    if (h->fast && !h->d4 && !h->gu_dense && coop_attr && want_coop) {
       const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
       const int warps = kCoopThreads / 32;
       h->plan_gu_coop = h->plan_gu;
@@ -578,7 +592,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
           for (int dg = 3; dg >= 2 && !found; --dg) {
             fp.depth_g = dg;
             fp.depth_d = dd;
-            found = fused_layout(K, h->n_books, 1, H, r, pg, fp, h->dn_dense, h->idx_bytes, E, k, S).total <= limit;
+            found = fused_layout(K, h->n_books, 1, H, r, pg, fp, h->dn_dense, h->idx_tc, E, k, S).total <= limit;
           }
       }
       // many thin slices would turn the partial y into the dominant traffic: leave those shapes to the chain
@@ -603,7 +617,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
                 pgt.x_smem = xsm;
                 fp.depth_g = dg;
                 fp.depth_d = dd;
-                const size_t need = fused_layout(K, h->n_books, t, H, r, pgt, fp, h->dn_dense, h->idx_bytes, E, k, S).total;
+                const size_t need = fused_layout(K, h->n_books, t, H, r, pgt, fp, h->dn_dense, h->idx_tc, E, k, S).total;
                 if (need <= limit) {
                   fit = true;
                   h->fused_dg[t] = (signed char)dg;
@@ -616,13 +630,15 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
           maxT_fit = t;
         }
         const void* fn = nullptr;
-#define MOE_VQLR_FUSED_FN(IDXT, DENSE)                                                             \
-  fn = fp.jd == 1 ? (const void*)k_expert_fused<IDXT, DENSE, 1> : fp.jd == 2 ? (const void*)k_expert_fused<IDXT, DENSE, 2> \
-     : fp.jd == 3 ? (const void*)k_expert_fused<IDXT, DENSE, 3> : (const void*)k_expert_fused<IDXT, DENSE, 4>
-        if (h->dn_dense && h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, true); }
-        else if (h->dn_dense) { MOE_VQLR_FUSED_FN(uint16_t, true); }
-        else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, false); }
-        else { MOE_VQLR_FUSED_FN(uint16_t, false); }
+#define MOE_VQLR_FUSED_FN(IDXT, DENSE, D4V)                                                             \
+  fn = fp.jd == 1 ? (const void*)k_expert_fused<IDXT, DENSE, 1, D4V> : fp.jd == 2 ? (const void*)k_expert_fused<IDXT, DENSE, 2, D4V> \
+     : fp.jd == 3 ? (const void*)k_expert_fused<IDXT, DENSE, 3, D4V> : (const void*)k_expert_fused<IDXT, DENSE, 4, D4V>
+        if (h->d4 && h->dn_dense) { MOE_VQLR_FUSED_FN(uint16_t, true, true); }
+        else if (h->d4) { MOE_VQLR_FUSED_FN(uint16_t, false, true); }
+        else if (h->dn_dense && h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, true, false); }
+        else if (h->dn_dense) { MOE_VQLR_FUSED_FN(uint16_t, true, false); }
+        else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, false, false); }
+        else { MOE_VQLR_FUSED_FN(uint16_t, false, false); }
 #undef MOE_VQLR_FUSED_FN
         cudaError_t e1 = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
         const size_t cf_smem = ((size_t)(k + S) * (r > 0 ? r : 0) + (size_t)(k + S) * kCfCols * 2) * sizeof(float);
@@ -633,7 +649,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
           h->fused_max_T = maxT_fit;
           h->fplan = fp;
           h->plan_gu_fused = pg;
-          if (!h->dn_dense) idx_dp_bytes = (size_t)(E + S) * fp.n_sl * (H / 8) * 32 * fp.jd * h->idx_bytes;
+          if (!h->dn_dense) idx_dp_bytes = (size_t)(E + S) * fp.n_sl * (H / 8) * 32 * fp.jd * h->idx_tc;
         } else {
           cudaGetLastError();
         }
@@ -697,7 +713,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   cudaMemset(h->workspace, 0, h->workspace_bytes);
   if (h->fused && !h->dn_dense) {      // one-off: the down index map per slice
     const FusedPlan& fp = h->fplan;
-    if (h->idx_bytes == 1)
+    if (h->idx_tc == 1)
       k_relay_down_idx<uint8_t><<<h->sm_count * 8, 256>>>(static_cast<const uint8_t*>(P.down.idx), static_cast<uint8_t*>(h->idx_dp), E + S, H, I / kD, fp.tps, fp.n_sl, fp.jd);
     else
       k_relay_down_idx<uint16_t><<<h->sm_count * 8, 256>>>(static_cast<const uint16_t*>(P.down.idx), static_cast<uint16_t*>(h->idx_dp), E + S, H, I / kD, fp.tps, fp.n_sl, fp.jd);
@@ -715,7 +731,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     const moe_vqlr_proj* projs[3] = {&cfg->gate, &cfg->up, &cfg->down};
     for (int i = 0; i < 3; ++i) {
       if (projs[i]->kind != MOE_VQLR_PROJ_VQLR) continue;
-      const size_t n = (size_t)(E + S) * H * I / kD;
+      const size_t n = (size_t)(E + S) * H * I / cfg->vq_dim;
       if (h->idx_bytes == 1) k_max_index<uint8_t><<<h->sm_count * 4, 256>>>(static_cast<const uint8_t*>(projs[i]->idx), n, d_max);
       else k_max_index<uint16_t><<<h->sm_count * 4, 256>>>(static_cast<const uint16_t*>(projs[i]->idx), n, d_max);
     }

@@ -81,6 +81,13 @@ SHAPES: Dict[str, LayerShape] = {
                              mode="paper", per_projection_codebook=True),
     "qwen3_5bit": LayerShape("qwen3_5bit", H=2048, I=768, E=128, k=8, d=8, K=256, r=504, T=1,
                              mode="paper", per_projection_codebook=True),
+    # the (4, 256, 256) point on the OLMoE shape: four-value code words (generic kernels)
+    "olmoe_deployed": LayerShape("olmoe_deployed", H=2048, I=1024, E=64, k=8, d=4, K=256, r=256, T=1,
+                                 mode="paper", per_projection_codebook=True),
+    "olmoe_deployed_b8": LayerShape("olmoe_deployed_b8", H=2048, I=1024, E=64, k=8, d=4, K=256, r=256, T=8,
+                                    mode="paper", per_projection_codebook=True),
+    "olmoe_deployed_b16": LayerShape("olmoe_deployed_b16", H=2048, I=1024, E=64, k=8, d=4, K=256, r=256,
+                                     T=16, mode="paper", per_projection_codebook=True),
 }
 
 

@@ -136,3 +136,16 @@ def test_gelu_long_intermediate():
     # I > 4096: the activation runs in the wide kernel of the chain
     shp = synth.LayerShape("longI", H=256, I=4608, E=4, k=2, d=8, K=256, r=16, T=2, act="gelu_tanh")
     _full_check(shp)
+
+
+@pytest.mark.parametrize("shp", [synth.shape("tiny", d=4, T=1), synth.shape("tiny", d=4, T=5, mode="paper"),
+                                 synth.LayerShape("ragged4", H=8 * 37, I=8 * 53, E=13, k=3, S=1, d=4, K=100, r=7, T=5),
+                                 synth.LayerShape("books4", H=256, I=192, E=8, k=2, d=4, K=512, r=8, T=3,
+                                                  per_projection_codebook=True),
+                                 synth.LayerShape("olmoe_like", H=2048, I=1024, E=12, k=8, d=4, K=256, r=256,
+                                                  T=4, mode="paper", per_projection_codebook=True)],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
+def test_four_value_code_words(shp):
+    """d = 4 (Section 5.5): code words of four values, two indices per eight weights; uint8 and
+    uint16 indices, shared and separate code books, the shape of the paper's (4, 256, 256) point."""
+    _full_check(shp)

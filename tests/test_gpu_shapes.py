@@ -109,7 +109,7 @@ def test_error_codes():
     torch.cuda.synchronize()
     mod.close()
     # unsupported shapes and options
-    for kw, code in ((dict(d=4), binding.ERR_UNSUPPORTED), (dict(max_tokens=17), binding.ERR_UNSUPPORTED),
+    for kw, code in ((dict(d=2), binding.ERR_UNSUPPORTED), (dict(d=16), binding.ERR_UNSUPPORTED), (dict(max_tokens=17), binding.ERR_UNSUPPORTED),
                      (dict(k=9), binding.ERR_INVALID_ARG), (dict(H=260), binding.ERR_UNSUPPORTED)):
         with pytest.raises(binding.MoeVqlrError) as err:
             args = dict(H=256, I=128, E=8, k=2, S=0, d=8, K=256, r=16, max_tokens=4)

@@ -107,8 +107,10 @@ def test_persistent_kernel(shp):
 @pytest.mark.parametrize("shp", [synth.shape("tiny", T=5), synth.shape("tiny", T=2, mode="paper"),
                                  synth.shape("qwen3", E=16, T=3), synth.shape("qwen3", E=16, T=9, mode="paper"),
                                  synth.shape("qwen3", E=16, T=16, I=832), synth.shape("dsv2lite", E=16, T=1),
-                                 synth.shape("dsv2lite", E=16, T=2, mode="paper")],
-                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}-I{s.I}")
+                                 synth.shape("dsv2lite", E=16, T=2, mode="paper"),
+                                 synth.shape("tiny", T=2, d=4), synth.shape("tiny", T=1, d=4, mode="paper"),
+                                 synth.shape("olmoe_deployed", E=12, T=3), synth.shape("olmoe_deployed", E=12, T=1)],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}-I{s.I}-d{s.d}")
 def test_fused_expert_kernel_forced(shp):
     """Router -> one kernel per (work group, slice of I) -> weighted sum, forced also where the
     items would not fill the GPU: three launches per call, the chain's results."""

@@ -199,8 +199,9 @@ def test_exact_codebook_rank0_reproduces_dense_bf16_expert():
         np.testing.assert_allclose(comp.out[t], acc.numpy(), rtol=0, atol=1e-12)
 
 
-def test_single_expert_is_plain_swiglu_mlp():
-    shp = small_shape(E=1, k=1, T=2, r=3)
+@pytest.mark.parametrize("d", [8, 4, 2])
+def test_single_expert_is_plain_swiglu_mlp(d):
+    shp = small_shape(E=1, k=1, T=2, r=3, d=d)
     layer = synth.make_layer(shp, seed=8)
     orc = oracle.OracleLayer.from_synth(layer)
     res = orc.decode_layer(layer.x)
