@@ -969,8 +969,11 @@ __device__ __forceinline__ void gu_tiles_begin(const Params& P, const StagePlan&
   TRACE_STAMP(1, 7);
 }
 
-// The tile loop proper (needs code books, tokens and z in shared memory).
-template <typename IdxT, bool DENSE, bool D4 = false>
+// The tile loop proper (needs code books, tokens and z in shared memory).  LRF: there are at least
+// as many low-rank groups (32 ranks each) as slices; slice s then carries the groups s, s + n_slices,
+// ... besides its own blocks and no group is a part of its own (fewer, fatter units and fewer
+// partial tiles; with fewer groups than slices the units that carry one would lag the others).
+template <typename IdxT, bool DENSE, bool D4 = false, bool LRF = false>
 __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
                                              const GuSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
@@ -1002,9 +1005,22 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
     if (++cur_slot == D) cur_slot = 0;
     const int off = R.grp_off[grp], n_tok = R.grp_cnt[grp];
     const int tok = g < n_tok ? R.pair_token[off + g] : -1;
-    const bool is_lr = part >= pl.n_slices;
+    const bool is_lr = !LRF && part >= pl.n_slices;
     float acc_g[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     float acc_u[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    // LRF: the factor bytes of the slice's first low-rank group are requested now and used after
+    // the slice's own mma's
+    const bool has_lr = LRF && part < pl.n_lr;
+    size_t lr_row = 0;
+    uint4 lf_g = {0, 0, 0, 0}, lf_u = {0, 0, 0, 0};
+    if (LRF && has_lr) {
+      lr_row = (size_t)R.grp_e[grp] * P.I + jt * 8 + g;
+      const int rho = part * 32 + 8 * c;
+      if (rho < P.r) {
+        lf_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho));
+        lf_u = __ldg(reinterpret_cast<const uint4*>(P.up.factor + lr_row * P.r + rho));
+      }
+    }
     if (!is_lr) {
       const int b0 = part * 32 + (DENSE ? c : 8 * c);
       if (frag_grp != grp || frag_part != part) {
@@ -1077,6 +1093,27 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
       acc_g[0][0] += acc_g[0][2]; acc_g[0][1] += acc_g[0][3];
       acc_u[0][0] += acc_u[0][2]; acc_u[0][1] += acc_u[0][3];
     }
+    if (LRF && has_lr) {
+      for (int lg = part; lg < pl.n_lr; lg += pl.n_slices) {
+        const int rho = lg * 32 + 8 * c;
+        if (lg != part) {                   // further groups of this slice (ranks beyond 32 * n_slices)
+          lf_g = lf_u = make_uint4(0, 0, 0, 0);
+          if (rho < P.r) {
+            lf_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho));
+            lf_u = __ldg(reinterpret_cast<const uint4*>(P.up.factor + lr_row * P.r + rho));
+          }
+        }
+        uint4 zgh = {0, 0, 0, 0}, zgl = {0, 0, 0, 0}, zuh = {0, 0, 0, 0}, zul = {0, 0, 0, 0};
+        if (rho < P.r && tok >= 0) {
+          const int ig2 = (tok * 2 + P.gate.zslot) * rb + (rho >> 3), iu2 = (tok * 2 + P.up.zslot) * rb + (rho >> 3);
+          zgh = s_zh[ig2]; zgl = s_zl[ig2]; zuh = s_zh[iu2]; zul = s_zl[iu2];
+        }
+        mma_block_hilo(acc_g[0], zgh, zgl, lf_g);    // hi product in the accumulators' first halves, lo in the second
+        mma_block_hilo(acc_u[0], zuh, zul, lf_u);
+      }
+      acc_g[0][0] += acc_g[0][2]; acc_g[0][1] += acc_g[0][3];
+      acc_u[0][0] += acc_u[0][2]; acc_u[0][1] += acc_u[0][3];
+    }
     TRACE_STAMP(0, 6 + 3 * i);
     // partial tile of this part: token g of the group, rows 2c and 2c+1 of the tile
     if (g < n_tok) {
@@ -1089,7 +1126,7 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
   TRACE_STAMP(0, 15);
 }
 
-template <typename IdxT, bool DENSE, bool D4 = false>
+template <typename IdxT, bool DENSE, bool D4 = false, bool LRF = false>
 __global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
 k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {
   extern __shared__ uint4 s_u4[];
@@ -1107,7 +1144,7 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   gu_finish_stage<DENSE>(P, pl, n_books, m, pl.depth - 1);                                     // ... while the stage settles
   pdl_launch();
   TRACE_STAMP(0, 3);
-  gu_tiles_run<IdxT, DENSE, D4>(P, x, T, pl, m, w);
+  gu_tiles_run<IdxT, DENSE, D4, LRF>(P, x, T, pl, m, w);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -59,6 +59,7 @@ struct moe_vqlr_handle {
   bool per_expert_launch;   // ablation: gate/up and down run as one launch per work group
   bool d4;                  // four-value code words on the tensor-core paths (uint8 indices read as pairs)
   int idx_tc;               // bytes per index element as the tensor-core kernels read it (2 with d4)
+  bool lrf;                 // chain gate/up: the low-rank groups ride on the slices (at least one per slice)
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
   size_t workspace_bytes;
@@ -271,8 +272,11 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           StagePlan pl = h->plan_gu;
           if (h->per_expert_launch) pl.only_grp = gi;
           if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->d4 && h->lrf) le = launch_pdl(k_gateup_mma<uint16_t, false, true, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
           else if (h->d4) le = launch_pdl(k_gateup_mma<uint16_t, false, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->idx_bytes == 1 && h->lrf) le = launch_pdl(k_gateup_mma<uint8_t, false, false, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
           else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->lrf) le = launch_pdl(k_gateup_mma<uint16_t, false, false, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
           else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
         }
         h->launches += n_launch - 1;
@@ -473,6 +477,12 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->plan_dn = plan_stage(H, I, r, h->dn_dense);
     if (h->plan_gu.n_lr > 0) h->plan_gu.chunk = h->plan_gu.tiles < 16 ? h->plan_gu.tiles : 16;   // mix slice and low-rank parts
     h->plan_dn.n_parts = h->plan_dn.n_slices;          // the down kernel folds the low-rank groups into the slices
+    {
+      const char* coop_env = getenv("MOE_VQLR_COOP");      // the persistent kernel walks the groups as parts of their own
+      const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) || (coop_env && coop_env[0] == '1');
+      h->lrf = gu_vq && !want_coop && h->plan_gu.n_lr >= h->plan_gu.n_slices;
+    }
+    if (h->lrf) h->plan_gu.n_parts = h->plan_gu.n_slices;   // ... and so does gate/up where every slice gets a group
     // shared-memory plan: replicate a small code book eight times (conflict-free lookups), stage the
     // tokens when they fit, then take the deepest rings that still fit
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
@@ -509,8 +519,11 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       cudaError_t e1 = cudaSuccess, e2 = cudaSuccess;
       const int a = cudaFuncAttributeMaxDynamicSharedMemorySize;
       if (gu_dn) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (d4 && h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true, true>, (cudaFuncAttribute)a, (int)smem_gu);
       else if (d4) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (h->idx_bytes == 1 && h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false, false, true>, (cudaFuncAttribute)a, (int)smem_gu);
       else if (h->idx_bytes == 1) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, false, true>, (cudaFuncAttribute)a, (int)smem_gu);
       else e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
       if (h->dn_dense) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
       else if (d4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
@@ -530,7 +543,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     int coop_attr = 0;
     cudaDeviceGetAttribute(&coop_attr, cudaDevAttrCooperativeLaunch, h->device);
     const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) || (coop_env && coop_env[0] == '1');
-    if (h->fast && !h->d4 && !h->gu_dense && coop_attr && want_coop) {
+    if (h->fast && !h->d4 && !h->lrf && !h->gu_dense && coop_attr && want_coop) {
       const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
       const int warps = kCoopThreads / 32;
       h->plan_gu_coop = h->plan_gu;
@@ -576,6 +589,10 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       memset(&fp, 0, sizeof fp);
       StagePlan pg = h->plan_gu;
       pg.x_smem = 1;
+      if (h->lrf) {                                  // the fused kernel walks the low-rank groups as parts of their own
+        pg.n_parts = pg.n_slices + pg.n_lr;
+        finish_plan(pg, pg.W);
+      }
       bool found = false;
       for (int tps = (tiles + target - 1) / target; tps >= 1 && !found; --tps) {
         if (tps > 4 * kFusedMaxJd) tps = 4 * kFusedMaxJd;
