@@ -758,6 +758,64 @@ __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params
   else router_z_unit(P, x, T, unit, threadIdx.x & 31);
 }
 
+// k_router_zmma_pdl: head of the chain for 9..16 tokens.  The shared projections z = basis * x
+// (Section 4.2) run on the tensor cores: one block per eight basis rows, each of its eight warps
+// takes an eighth of H with the tokens as the sixteen rows of the m16n8k16 tile (tokens 0..7 in
+// rows 0..7, 8..15 in rows 8..15), and the warps' partial tiles meet in shared memory and are added
+// in warp order.  The remaining blocks compute the router logits with the exact FMA chains of
+// k_router_z_pdl, one (row, group of four tokens) per warp.  H must be a multiple of 256, r of 8.
+constexpr int kZmmaWarps = 8;
+
+__host__ __device__ __forceinline__ int zmma_blocks(const Params& P) { return P.n_zrows / 8 * P.z_repeat; }
+
+__global__ void __launch_bounds__(32 * kZmmaWarps) k_router_zmma_pdl(const Params P, const bf16* __restrict__ x, int T) {
+  __shared__ float s_red[kZmmaWarps][128];
+  pdl_wait();      // the previous call's kernels may still read logits / z
+  pdl_launch();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n_units = P.E * ((T + kTokGroup - 1) / kTokGroup), n_logit_blocks = (n_units + kZmmaWarps - 1) / kZmmaWarps;
+  if ((int)blockIdx.x < n_logit_blocks) {      // the logits blocks come first: their FMA chains take longest
+    const int unit = (int)blockIdx.x * kZmmaWarps + warp;
+    if (unit >= n_units) return;
+    if (P.H <= 2048) router_z_unit_row8(P, x, T, unit, lane);
+    else router_z_unit(P, x, T, unit, lane);
+    return;
+  }
+  const int g = lane >> 2, c = lane & 3;
+  const int q0 = (((int)blockIdx.x - n_logit_blocks) % (P.n_zrows / 8)) * 8;   // a repeated tile (ablation) recomputes the same rows
+  const int slot = q0 / P.r, rho0 = q0 - slot * P.r;
+  const bf16* basis = (slot == P.gate.zslot && P.gate.basis) ? P.gate.basis : P.up.basis;
+  const int nblk = P.H / 8, per = nblk / kZmmaWarps;
+  const uint4* w4 = reinterpret_cast<const uint4*>(basis + (size_t)(rho0 + g) * P.H) + warp * per + c;
+  const uint4* xa4 = reinterpret_cast<const uint4*>(x + (size_t)g * P.H) + warp * per + c;
+  const uint4* xb4 = reinterpret_cast<const uint4*>(x + (size_t)(g + 8) * P.H) + warp * per + c;
+  const bool live_a = g < T, live_b = g + 8 < T;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int s = 0; s < per; s += 16) {                              // four steps of 32 values with their loads in flight
+    uint4 wv[4], av[4], bv[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const bool in = s + 4 * u < per;
+      wv[u] = in ? __ldg(w4 + s + 4 * u) : make_uint4(0, 0, 0, 0);
+      av[u] = (in && live_a) ? __ldg(xa4 + s + 4 * u) : make_uint4(0, 0, 0, 0);
+      bv[u] = (in && live_b) ? __ldg(xb4 + s + 4 * u) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) mma_block_hilo(acc, av[u], bv[u], wv[u]);
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) s_red[warp][lane * 4 + i] = acc[i];
+  __syncthreads();
+  if (threadIdx.x < 128) {
+    float sum = 0.f;
+#pragma unroll
+    for (int w = 0; w < kZmmaWarps; ++w) sum += s_red[w][threadIdx.x];
+    const int l2 = threadIdx.x >> 2, i = threadIdx.x & 3;
+    const int tok = (l2 >> 2) + ((i & 2) ? 8 : 0), row = 2 * (l2 & 3) + (i & 1);
+    if (tok < T) P.z[((size_t)tok * 2 + slot) * P.r + rho0 + row] = sum;
+  }
+}
+
 // Splits `total` units evenly over `parts` warps: first unit of warp `idx` = floor(total * idx / parts),
 // in 32-bit arithmetic (parts < 65536).
 __device__ __forceinline__ int split_begin(int total, int parts, int idx) {

@@ -196,6 +196,8 @@ T* carve(char*& cur, size_t n) {
 // Enqueues the kernel of one stage (nothing for a stage this configuration does not have).
 cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, bf16* ob, cudaStream_t st, bool allow_coop) {
   const Params& P = h->P;
+  // more than eight tokens: the basis projections run on the tensor cores, in the router kernel's launch
+  const bool z_by_mma = h->fast && T > 8 && P.n_zrows > 0 && P.H % 256 == 0 && P.r % 8 == 0;
   cudaError_t le = cudaSuccess;
   bool ran = false;
   const int n_pos = T * (P.k + P.S);
@@ -215,8 +217,12 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
     // one wave of (work group, slice) items at most: with more, the chain's finer parts balance better
     switch (stage) {
       case 0:
-        le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
-                        32 * kRouterWarps, 0, st, P, xb, T);
+        if (z_by_mma)
+          le = launch_pdl(k_router_zmma_pdl, zmma_blocks(P) + (P.E * ((T + kTokGroup - 1) / kTokGroup) + kZmmaWarps - 1) / kZmmaWarps,
+                          32 * kZmmaWarps, 0, st, P, xb, T);
+        else
+          le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
+                          32 * kRouterWarps, 0, st, P, xb, T);
         ran = true;
         break;
       case 2: {
@@ -259,8 +265,12 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
   } else if (h->fast) {
     switch (stage) {
       case 0:
-        le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
-                        32 * kRouterWarps, 0, st, P, xb, T);
+        if (z_by_mma)
+          le = launch_pdl(k_router_zmma_pdl, zmma_blocks(P) + (P.E * ((T + kTokGroup - 1) / kTokGroup) + kZmmaWarps - 1) / kZmmaWarps,
+                          32 * kZmmaWarps, 0, st, P, xb, T);
+        else
+          le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
+                          32 * kRouterWarps, 0, st, P, xb, T);
         ran = true;
         break;
       case 2: {
