@@ -1027,11 +1027,12 @@ __device__ __forceinline__ void gu_tiles_begin(const Params& P, const StagePlan&
   TRACE_STAMP(1, 7);
 }
 
-// The tile loop proper (needs code books, tokens and z in shared memory).  LRF: there are at least
+// The tile loop proper (needs code books, tokens and z in shared memory).  LRF > 0: there are at least
 // as many low-rank groups (32 ranks each) as slices; slice s then carries the groups s, s + n_slices,
 // ... besides its own blocks and no group is a part of its own (fewer, fatter units and fewer
 // partial tiles; with fewer groups than slices the units that carry one would lag the others).
-template <typename IdxT, bool DENSE, bool D4 = false, bool LRF = false>
+// LRF = 2: some slices carry two or more groups; the second one's bytes are requested early as well.
+template <typename IdxT, bool DENSE, bool D4 = false, int LRF = 0>
 __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
                                              const GuSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
@@ -1063,20 +1064,24 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
     if (++cur_slot == D) cur_slot = 0;
     const int off = R.grp_off[grp], n_tok = R.grp_cnt[grp];
     const int tok = g < n_tok ? R.pair_token[off + g] : -1;
-    const bool is_lr = !LRF && part >= pl.n_slices;
+    const bool is_lr = LRF == 0 && part >= pl.n_slices;
     float acc_g[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     float acc_u[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     // LRF: the factor bytes of the slice's first low-rank group are requested now and used after
     // the slice's own mma's
-    const bool has_lr = LRF && part < pl.n_lr;
+    const bool has_lr = LRF > 0 && part < pl.n_lr;
     size_t lr_row = 0;
-    uint4 lf_g = {0, 0, 0, 0}, lf_u = {0, 0, 0, 0};
-    if (LRF && has_lr) {
+    uint4 lf_g = {0, 0, 0, 0}, lf_u = {0, 0, 0, 0}, lf2_g = {0, 0, 0, 0}, lf2_u = {0, 0, 0, 0};   // first and second group
+    if (LRF > 0 && has_lr) {
       lr_row = (size_t)R.grp_e[grp] * P.I + jt * 8 + g;
-      const int rho = part * 32 + 8 * c;
+      const int rho = part * 32 + 8 * c, rho2 = rho + pl.n_slices * 32;
       if (rho < P.r) {
         lf_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho));
         lf_u = __ldg(reinterpret_cast<const uint4*>(P.up.factor + lr_row * P.r + rho));
+      }
+      if (LRF == 2 && part + pl.n_slices < pl.n_lr && rho2 < P.r) {
+        lf2_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho2));
+        lf2_u = __ldg(reinterpret_cast<const uint4*>(P.up.factor + lr_row * P.r + rho2));
       }
     }
     if (!is_lr) {
@@ -1151,10 +1156,12 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
       acc_g[0][0] += acc_g[0][2]; acc_g[0][1] += acc_g[0][3];
       acc_u[0][0] += acc_u[0][2]; acc_u[0][1] += acc_u[0][3];
     }
-    if (LRF && has_lr) {
+    if (LRF > 0 && has_lr) {
       for (int lg = part; lg < pl.n_lr; lg += pl.n_slices) {
         const int rho = lg * 32 + 8 * c;
-        if (lg != part) {                   // further groups of this slice (ranks beyond 32 * n_slices)
+        if (LRF == 2 && lg == part + pl.n_slices) {     // the second group was requested with the first
+          lf_g = lf2_g; lf_u = lf2_u;
+        } else if (lg != part) {            // further groups of this slice (ranks beyond 64 * n_slices)
           lf_g = lf_u = make_uint4(0, 0, 0, 0);
           if (rho < P.r) {
             lf_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho));
@@ -1184,7 +1191,7 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
   TRACE_STAMP(0, 15);
 }
 
-template <typename IdxT, bool DENSE, bool D4 = false, bool LRF = false>
+template <typename IdxT, bool DENSE, bool D4 = false, int LRF = 0>
 __global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
 k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {
   extern __shared__ uint4 s_u4[];

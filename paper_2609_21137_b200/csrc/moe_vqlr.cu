@@ -60,6 +60,7 @@ struct moe_vqlr_handle {
   bool d4;                  // four-value code words on the tensor-core paths (uint8 indices read as pairs)
   int idx_tc;               // bytes per index element as the tensor-core kernels read it (2 with d4)
   bool lrf;                 // chain gate/up: the low-rank groups ride on the slices (at least one per slice)
+  bool lrf2;                // ... and some slices carry two or more
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
   size_t workspace_bytes;
@@ -282,11 +283,14 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           StagePlan pl = h->plan_gu;
           if (h->per_expert_launch) pl.only_grp = gi;
           if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->d4 && h->lrf) le = launch_pdl(k_gateup_mma<uint16_t, false, true, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->d4 && h->lrf2) le = launch_pdl(k_gateup_mma<uint16_t, false, true, 2>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->d4 && h->lrf) le = launch_pdl(k_gateup_mma<uint16_t, false, true, 1>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
           else if (h->d4) le = launch_pdl(k_gateup_mma<uint16_t, false, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->idx_bytes == 1 && h->lrf) le = launch_pdl(k_gateup_mma<uint8_t, false, false, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->idx_bytes == 1 && h->lrf2) le = launch_pdl(k_gateup_mma<uint8_t, false, false, 2>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->idx_bytes == 1 && h->lrf) le = launch_pdl(k_gateup_mma<uint8_t, false, false, 1>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
           else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->lrf) le = launch_pdl(k_gateup_mma<uint16_t, false, false, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->lrf2) le = launch_pdl(k_gateup_mma<uint16_t, false, false, 2>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          else if (h->lrf) le = launch_pdl(k_gateup_mma<uint16_t, false, false, 1>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
           else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
         }
         h->launches += n_launch - 1;
@@ -491,6 +495,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       const char* coop_env = getenv("MOE_VQLR_COOP");      // the persistent kernel walks the groups as parts of their own
       const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) || (coop_env && coop_env[0] == '1');
       h->lrf = gu_vq && !want_coop && h->plan_gu.n_lr >= h->plan_gu.n_slices;
+      h->lrf2 = h->lrf && h->plan_gu.n_lr > h->plan_gu.n_slices;
     }
     if (h->lrf) h->plan_gu.n_parts = h->plan_gu.n_slices;   // ... and so does gate/up where every slice gets a group
     // shared-memory plan: replicate a small code book eight times (conflict-free lookups), stage the
@@ -529,11 +534,14 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       cudaError_t e1 = cudaSuccess, e2 = cudaSuccess;
       const int a = cudaFuncAttributeMaxDynamicSharedMemorySize;
       if (gu_dn) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (d4 && h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true, true>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (d4 && h->lrf2) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true, 2>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (d4 && h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true, 1>, (cudaFuncAttribute)a, (int)smem_gu);
       else if (d4) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (h->idx_bytes == 1 && h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false, false, true>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (h->idx_bytes == 1 && h->lrf2) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false, false, 2>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (h->idx_bytes == 1 && h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false, false, 1>, (cudaFuncAttribute)a, (int)smem_gu);
       else if (h->idx_bytes == 1) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, false, true>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (h->lrf2) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, false, 2>, (cudaFuncAttribute)a, (int)smem_gu);
+      else if (h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, false, 1>, (cudaFuncAttribute)a, (int)smem_gu);
       else e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
       if (h->dn_dense) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
       else if (d4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);

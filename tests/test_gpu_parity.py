@@ -48,6 +48,14 @@ def test_rank_zero_and_two_codebooks():
                                  per_projection_codebook=True))
 
 
+def test_more_rank_groups_than_slices():
+    # the chain's gate/up kernel lets the slices carry the low-rank groups: two and three groups on
+    # one slice (the third fetched late), uint16 and uint8 indices, four-value code words
+    _full_check(synth.LayerShape("lr2_u16", H=256, I=192, E=8, k=2, d=8, K=512, r=64, T=3))
+    _full_check(synth.LayerShape("lr3_u8", H=256, I=192, E=8, k=2, d=8, K=256, r=88, T=5, mode="paper"))
+    _full_check(synth.LayerShape("lr2_d4", H=512, I=192, E=8, k=2, d=4, K=256, r=128, T=4))
+
+
 def test_topk_equals_E_and_single_expert():
     _full_check(synth.LayerShape("kE", H=128, I=64, E=4, k=4, d=8, K=64, r=4, T=4))
     _full_check(synth.LayerShape("E1", H=128, I=64, E=1, k=1, d=8, K=64, r=4, T=2))
