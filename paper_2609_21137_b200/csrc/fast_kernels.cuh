@@ -1610,27 +1610,52 @@ __device__ __forceinline__ void combine_unit(const Params& P, bf16* __restrict__
   const int col = threadIdx.x % kCombineCols, sl = threadIdx.x / kCombineCols, n_sl = blockDim.x / kCombineCols;
   const int t = unit / blocks_per_tok, h2 = (unit - t * blocks_per_tok) * kCombineCols + col;
   const size_t part_stride = (size_t)n_pos * P.H;
-  for (int s = sl; s < n_slots; s += n_sl) {
+  // fewer slots than slot lanes (few experts per token): lps lanes share one slot's parts, lane q of
+  // them adds the parts q, q + lps, ...; the partial sums are added in (slot, q) order below
+  const int lps = n_slots < n_sl ? n_sl / n_slots : 1;
+  const int n_rows = n_slots * lps;
+  if (lps == 1) {
+    for (int s = sl; s < n_slots; s += n_sl) {
+      const int pos = __ldcg(P.inv_pos + t * n_slots + s);
+      const float w = __ldcg(P.pair_w + pos);
+      float y0 = 0.f, y1 = 0.f;
+      if (h2 < H2) {
+        const float* src = P.ypart + (size_t)pos * P.H + 2 * h2;
+        for (int part0 = 0; part0 < n_parts; part0 += 4) {
+          float2 v[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            v[q] = part0 + q < n_parts ? __ldcg(reinterpret_cast<const float2*>(src + (part0 + q) * part_stride)) : make_float2(0.f, 0.f);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { y0 += v[q].x; y1 += v[q].y; }
+        }
+      }
+      s_y[s][col] = make_float2(w * y0, w * y1);
+    }
+  } else if (sl < n_rows) {
+    const int s = sl / lps, q0 = sl - s * lps;
     const int pos = __ldcg(P.inv_pos + t * n_slots + s);
     const float w = __ldcg(P.pair_w + pos);
     float y0 = 0.f, y1 = 0.f;
     if (h2 < H2) {
-      const float* src = P.ypart + (size_t)pos * P.H + 2 * h2;
-      for (int part0 = 0; part0 < n_parts; part0 += 4) {
+      const float* src = P.ypart + (size_t)pos * P.H + 2 * h2 + q0 * part_stride;
+      const size_t stride = part_stride * lps;
+      const int n_mine = (n_parts - q0 + lps - 1) / lps;
+      for (int i0 = 0; i0 < n_mine; i0 += 4) {
         float2 v[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-          v[q] = part0 + q < n_parts ? __ldcg(reinterpret_cast<const float2*>(src + (part0 + q) * part_stride)) : make_float2(0.f, 0.f);
+          v[q] = i0 + q < n_mine ? __ldcg(reinterpret_cast<const float2*>(src + (i0 + q) * stride)) : make_float2(0.f, 0.f);
 #pragma unroll
         for (int q = 0; q < 4; ++q) { y0 += v[q].x; y1 += v[q].y; }
       }
     }
-    s_y[s][col] = make_float2(w * y0, w * y1);
+    s_y[sl][col] = make_float2(w * y0, w * y1);
   }
   __syncthreads();
   if (sl == 0 && h2 < H2) {
     float a0 = 0.f, a1 = 0.f;
-    for (int s = 0; s < n_slots; ++s) { a0 += s_y[s][col].x; a1 += s_y[s][col].y; }
+    for (int s = 0; s < n_rows; ++s) { a0 += s_y[s][col].x; a1 += s_y[s][col].y; }
     *reinterpret_cast<__nv_bfloat162*>(out + (size_t)t * P.H + 2 * h2) = __floats2bfloat162_rn(a0, a1);
   }
 }
