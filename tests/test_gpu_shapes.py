@@ -121,11 +121,12 @@ def test_error_codes():
         assert err.value.status == code, kw
 
 
-def test_index_validation_flag_finds_bad_index():
+@pytest.mark.parametrize("d", [8, 4])
+def test_index_validation_flag_finds_bad_index(d):
     from paper_2609_21137_b200 import binding
-    layer = synth.make_layer(synth.shape("tiny", K=200), seed=0)
+    layer = synth.make_layer(synth.shape("tiny", K=200, d=d), seed=0)
     binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_VALIDATE_INDICES).close()
-    layer.up.idx[3, 7, 5] = 200
+    layer.up.idx[3, 7, layer.up.idx.shape[2] - 1] = 200      # the last index of a row: inside the scan for either d
     with pytest.raises(binding.MoeVqlrError) as err:
         binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_VALIDATE_INDICES)
     assert err.value.status == binding.ERR_BAD_INDEX

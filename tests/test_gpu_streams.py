@@ -222,7 +222,7 @@ def test_one_handle_many_batch_sizes(mode):
 
 @pytest.mark.parametrize("shp", [synth.shape("tiny", T=1), synth.shape("tiny", T=5, mode="paper"),
                                  synth.shape("qwen3", E=16, T=1), synth.shape("dsv2lite", E=16, T=3),
-                                 synth.shape("qwen3_deployed", E=24, T=2)],
+                                 synth.shape("qwen3_deployed", E=24, T=2), synth.shape("qwen3", E=16, T=12)],
                          ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
 def test_ablation_switches_keep_results(shp):
     """Section 5.4's mechanism switches: shared projections recomputed per expert, and one launch
