@@ -140,7 +140,9 @@ typedef struct {
  * moe_vqlr_workspace_bytes).  Which kernels a call runs (that path, the chain of five kernels, or
  * the generic chain for shapes the tensor-core kernels do not cover) never changes its results
  * beyond the summation order; MOE_VQLR_FUSED=0 in the environment at create() keeps the handle
- * off the fused path. */
+ * off the fused path, and MOE_VQLR_PCB=1 makes calls with two or more tokens evaluate the VQ term of
+ * gate/up through per-token projection code books T[b][k] = <x_b, codebook[k]> (Section 4.2; K <=
+ * 256, vq_dim 8; measured slower than the reconstructing tensor-core kernel on B200, hence opt-in). */
 int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out);
 
 /* Runs the layer for T tokens.  x: [T][H] bf16, device.  out: [T][H] bf16, device, written with

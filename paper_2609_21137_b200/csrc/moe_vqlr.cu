@@ -16,6 +16,7 @@
 #include "fast_kernels.cuh"
 #include "coop_kernel.cuh"
 #include "fused_kernel.cuh"
+#include "pcb_kernel.cuh"
 
 #include <cstdlib>
 
@@ -61,6 +62,10 @@ struct moe_vqlr_handle {
   int idx_tc;               // bytes per index element as the tensor-core kernels read it (2 with d4)
   bool lrf;                 // chain gate/up: the low-rank groups ride on the slices (at least one per slice)
   bool lrf2;                // ... and some slices carry two or more
+  bool pcb;                 // gate/up through the projection code book is available (K <= 256, uint8, d = 8)
+  int pcb_min_T;            // ... and used from this many tokens on
+  int pcb_Q;                // table pieces per token = ceil(H / 8 / 64)
+  size_t smem_lr;           // dynamic shared memory of k_gateup_lr
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
   size_t workspace_bytes;
@@ -276,6 +281,21 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         break;
       case 2: {
         const size_t smem = gu_layout(P.K, h->n_books, T, P.H, P.r, h->plan_gu, (h->gu_dense ? kDenseThreads : kFastThreads) / 32, P.E, P.k, P.S).total;
+        if (h->pcb && T >= h->pcb_min_T && !h->per_expert_launch) {
+          // projection code book: routing + low-rank term, then the table kernel
+          StagePlan pl = h->plan_gu;
+          pl.x_smem = 0; pl.repl = 0;
+          le = launch_pdl(k_gateup_lr, h->sm_count, kFastThreads, h->smem_lr, st, P, xb, T, pl, h->want_dbg);
+          if (le == cudaSuccess) {
+            int bpc = h->sm_count / (T * h->pcb_Q);
+            if (bpc < 1) bpc = 1;
+            le = launch_pdl(k_gateup_pcb, T * h->pcb_Q * bpc, kPcbThreads, pcb_smem_bytes(P.K), st, P, xb, T, h->pcb_Q, bpc,
+                            h->plan_gu.n_lr > 0 ? 1 : 0);
+            h->launches += 1;
+          }
+          ran = true;
+          break;
+        }
         // one launch over all work groups, or (ablation) one launch per possible work group:
         // a launch whose group does not exist finds no units after the routing and ends
         const int n_launch = h->per_expert_launch ? n_pos : 1;
@@ -299,15 +319,17 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
       }
       case 3: {
         const int with_zd = (!h->dn_dense && P.r > 0) ? 1 : 0;
+        const int gu_parts = (h->pcb && T >= h->pcb_min_T && !h->per_expert_launch) ? h->pcb_Q + (h->plan_gu.n_lr > 0 ? 1 : 0)
+                                                                                     : h->plan_gu.n_parts;
         if (P.I <= 4096) {                                // one fused block per pair (times zsplit)
           int zsplit = 1;
           if (with_zd) while (n_pos * zsplit * 2 <= 3 * h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
           le = launch_pdl(k_act_zdown, n_pos * zsplit, kActThreads, (size_t)P.I * sizeof(float), st, P, n_pos,
-                          h->plan_gu.n_parts, with_zd, zsplit);
+                          gu_parts, with_zd, zsplit);
         } else {                                          // few pairs or a long intermediate: two wide kernels
           int grid = (n_pos * (P.I / 2) + 255) / 256;
           if (grid > 4 * h->sm_count) grid = 4 * h->sm_count;
-          le = launch_pdl(k_act, grid, 256, 0, st, P, n_pos, h->plan_gu.n_parts);
+          le = launch_pdl(k_act, grid, 256, 0, st, P, n_pos, gu_parts);
           if (le == cudaSuccess && with_zd) {
             int wpd = 1;                                  // warps per z_d value: 2048 values of I each, at most 8
             while (wpd < 8 && P.I > 2048 * wpd) wpd *= 2;
@@ -552,6 +574,32 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     }
   }
 
+  // ---- gate/up through the projection code book (several tokens, small code book) ---------------
+  h->pcb = false;
+  h->pcb_min_T = 0;
+  h->pcb_Q = 0;
+  h->smem_lr = 0;
+  {
+    const char* penv = getenv("MOE_VQLR_PCB");            // 1: from two tokens on; otherwise off (measured slower than the tensor-core kernel)
+    const bool gu_vq2 = P.gate.kind == MOE_VQLR_PROJ_VQLR && P.up.kind == MOE_VQLR_PROJ_VQLR;
+    const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
+    if (h->fast && gu_vq2 && !h->d4 && cfg->vq_dim == kD && h->idx_bytes == 1 && H % 16 == 0 && I % kPcbRows == 0 &&
+        pcb_smem_bytes(K) <= limit && penv && penv[0] == '1') {
+      StagePlan pl = h->plan_gu;
+      pl.x_smem = 0; pl.repl = 0;
+      h->smem_lr = gu_layout(K, 0, maxT, H, r, pl, kFastThreads / 32, E, k, S).total;
+      if (h->smem_lr <= limit &&
+          cudaFuncSetAttribute(k_gateup_lr, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_lr) == cudaSuccess &&
+          cudaFuncSetAttribute(k_gateup_pcb, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pcb_smem_bytes(K)) == cudaSuccess) {
+        h->pcb = true;
+        h->pcb_Q = (H / 8 + kPcbPiece - 1) / kPcbPiece;
+        h->pcb_min_T = 2;
+      } else {
+        cudaGetLastError();
+      }
+    }
+  }
+
   // ---- the same chain as one persistent cooperative kernel --------------------------------------
   h->coop = false;
   h->dn_restage = 0;
@@ -719,8 +767,10 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     P.p_hi = carve<bf16>(cur, n_pos * I);
     P.p_lo = carve<bf16>(cur, n_pos * I);
     P.zd = carve<float>(cur, n_pos * (r > 0 ? r : 1));
-    P.gpart = carve<float>(cur, h->fast ? (size_t)h->plan_gu.n_parts * n_pos * I : 1);
-    P.upart = carve<float>(cur, h->fast ? (size_t)h->plan_gu.n_parts * n_pos * I : 1);
+    size_t gu_parts_max = h->plan_gu.n_parts;
+    if (h->pcb && (size_t)h->pcb_Q + 1 > gu_parts_max) gu_parts_max = (size_t)h->pcb_Q + 1;
+    P.gpart = carve<float>(cur, h->fast ? gu_parts_max * n_pos * I : 1);
+    P.upart = carve<float>(cur, h->fast ? gu_parts_max * n_pos * I : 1);
     {
       int y_parts = h->fast ? h->plan_dn.n_parts : 0;
       if (h->fused && h->fplan.n_sl > y_parts) y_parts = h->fplan.n_sl;

@@ -252,3 +252,29 @@ def test_ablation_switches_keep_results(shp):
             assert torch.equal(out.view(torch.int16), ref_out.view(torch.int16))
         mod.close()
     base.close()
+
+
+@pytest.mark.parametrize("shp", [synth.shape("tiny", T=5), synth.shape("tiny", T=2, mode="paper", K=100),
+                                 synth.shape("dsv2lite", E=16, T=8), synth.shape("qwen3_deployed", E=24, T=16),
+                                 synth.LayerShape("ragged_piece", H=8 * 48, I=128, E=6, k=2, S=1, d=8, K=256, r=40, T=3),
+                                 synth.LayerShape("r0_books", H=1024, I=64, E=8, k=3, d=8, K=64, r=0, T=4,
+                                                  per_projection_codebook=True)],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
+def test_projection_code_book_path(shp, monkeypatch):
+    """MOE_VQLR_PCB=1: gate/up through per-token tables T[b][k] = <x_b, codebook[k]> (Section 4.2)
+    with the low-rank term in a kernel of its own: six launches per call, the oracle's results; one
+    and several table pieces, a ragged piece, small code books, rank 0, separate books."""
+    from paper_2609_21137_b200 import binding
+    monkeypatch.setenv("MOE_VQLR_PCB", "1")
+    monkeypatch.setenv("MOE_VQLR_FUSED", "0")
+    layer, res, _ = make_checked_layer(shp, 0)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    x = binding.bits_to_device(layer.x, "cuda")
+    for _ in range(2):
+        before = mod.launch_count
+        out, dbg = mod.decode(x, debug=True)
+        torch.cuda.synchronize()
+        assert mod.launch_count - before == 6
+        assert_routing(dbg, res)
+        assert_output(bf16_tensor_to_f64(out), res.out)
+    mod.close()
