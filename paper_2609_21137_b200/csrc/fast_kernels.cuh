@@ -1217,7 +1217,7 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
 // bf16 hi + lo for the down kernel's fragments, then z_d = basis_down * p when the down
 // projection is compressed.  Parts are added in ascending order.
 // ---------------------------------------------------------------------------------------------
-constexpr int kActThreads = 384;
+constexpr int kActThreads = 512;
 
 // grid = n_pos * zsplit blocks: block (pos, zs) rebuilds p[pos] (cheap, from L2) and computes the
 // z_d rows rho = zs, zs + zsplit, ...; only zs == 0 writes p_hi / p_lo.
