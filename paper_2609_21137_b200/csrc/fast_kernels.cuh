@@ -1381,6 +1381,9 @@ __global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos, in
 // are the bf16 hi + lo halves of p.  The warp of slice s also adds the low-rank groups s,
 // s + n_slices, ... (32 ranks each; A = z_d as hi + lo), so the parts are the slices alone.
 // ---------------------------------------------------------------------------------------------
+constexpr int kDnVqTiles = 2;     // a compressed down unit covers this many 8-row tiles of H (one set of p fragments,
+                                  // one request group, one step of the work cursor for 16 rows); the plan's tiles count them
+
 struct DnLayout {
   size_t ring, grp, cb_tmp, total;
   int slot_u4;      // uint4 per lane per ring slot: 2 (indices, factor) or 8 (a dense 256-value slice)
@@ -1389,7 +1392,7 @@ struct DnLayout {
 __host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& pl, int warps, int max_groups) {
   DnLayout L;
   size_t o = vq ? (size_t)K * 16 * (pl.repl ? 8 : 1) : 0;
-  L.slot_u4 = vq ? 2 : 8;
+  L.slot_u4 = vq ? 2 * kDnVqTiles : 8;
   L.ring = o;   o += (size_t)warps * pl.depth * L.slot_u4 * 32 * 16;
   L.grp = o;    o += ((size_t)max_groups * 12 + 15) / 16 * 16;
   L.cb_tmp = o; o += (vq && pl.repl) ? (size_t)K * 16 : 0;
@@ -1412,7 +1415,7 @@ __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, c
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3, nb = pl.nb;
   uint4* ring = m.ring;
   const Cursor& pf = w.pf;
-  const size_t row = (size_t)m.grp_e[pf.grp] * P.H + pf.jt * 8 + g;
+  const size_t row = (size_t)m.grp_e[pf.grp] * P.H + pf.jt * (DENSE ? 8 : 8 * kDnVqTiles) + g;
   if (DENSE) {
     const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I) + pf.part * 32 + c;
 #pragma unroll
@@ -1421,8 +1424,13 @@ __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, c
   } else {
     const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
     const int b = pf.part * 32 + 8 * c, rho = pf.part * 32 + 8 * c;
-    if (b < nb) cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_d + row * nb + b);
-    if (pf.part < pl.n_lr && rho < P.r) cp_async16(ring + (w.pf_slot * 2 + 1) * 32, P.down.factor + row * P.r + rho);
+#pragma unroll
+    for (int sub = 0; sub < kDnVqTiles; ++sub) {
+      const size_t rs = row + 8 * sub;
+      uint4* slot = ring + (size_t)(w.pf_slot * kDnVqTiles + sub) * 2 * 32;
+      if (b < nb) cp_async_idx8<IdxT>(slot, idx_d + rs * nb + b);
+      if (pf.part < pl.n_lr && rho < P.r) cp_async16(slot + 32, P.down.factor + rs * P.r + rho);
+    }
   }
   w.pf.next(pl);
   if (++w.pf_slot == pl.depth) w.pf_slot = 0;
@@ -1473,7 +1481,6 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
     const int pos = g < n_tok ? off + g : -1;
     const int b0 = part * 32 + (DENSE ? c : 8 * c);
     const int rho0 = part * 32 + 8 * c;
-    float acc[4][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // four independent chains
     if (frag_grp != grp || frag_part != part) {
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -1492,6 +1499,10 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
       }
       frag_grp = grp; frag_part = part;
     }
+#pragma unroll
+    for (int sub = 0; sub < (DENSE ? 1 : kDnVqTiles); ++sub) {
+    const int row0 = DENSE ? jt * 8 : (jt * kDnVqTiles + sub) * 8;      // first row of this 8-row tile
+    float acc[4][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // four independent chains
     if (DENSE) {
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -1500,8 +1511,9 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
       }
     } else {
       // mma.sync needs the whole warp: out-of-range block groups use index 0 and zero fragments
+      const uint4* uslot = ring + (size_t)(slot * kDnVqTiles + sub) * 2 * 32;
       uint4 raw = {0, 0, 0, 0};
-      if (b0 < nb) raw = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32);
+      if (b0 < nb) raw = ring_idx8<IdxT>(uslot);
       uint32_t id[8];
       unpack_idx8<IdxT>(raw, id);
 #pragma unroll
@@ -1510,9 +1522,9 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
         mma_block_hilo(acc[j & 1], fh[j], fl[j], w);      // hi product in rows 0..7 of the tile, lo in rows 8..15
       }
       if (part < pl.n_lr) {                   // warp-uniform: the low-rank group carried by this part
-        const uint4 f = rho0 < P.r ? ring[(slot * 2 + 1) * 32] : make_uint4(0, 0, 0, 0);
+        const uint4 f = rho0 < P.r ? uslot[32] : make_uint4(0, 0, 0, 0);
         mma_block_hilo(acc[2], zh, zl, f);
-        const size_t row = (size_t)s_grp_e[grp] * P.H + jt * 8 + g;
+        const size_t row = (size_t)s_grp_e[grp] * P.H + row0 + g;
         for (int lg = part + pl.n_slices; lg < pl.n_lr; lg += pl.n_slices) {   // more rank groups than slices
           const int rho = lg * 32 + 8 * c;
           uint4 f2 = {0, 0, 0, 0}, zh2 = {0, 0, 0, 0}, zl2 = {0, 0, 0, 0};
@@ -1527,13 +1539,14 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
         }
       }
     }
-    if (i < 5) TRACE_STAMP(2, 5 + 2 * i);
     if (pos >= 0) {
-      const size_t at = ((size_t)part * n_pos + pos) * P.H + jt * 8 + 2 * c;
+      const size_t at = ((size_t)part * n_pos + pos) * P.H + row0 + 2 * c;
       *reinterpret_cast<float2*>(P.ypart + at) =
           make_float2(((acc[0][0] + acc[0][2]) + (acc[1][0] + acc[1][2])) + ((acc[2][0] + acc[2][2]) + (acc[3][0] + acc[3][2])),
                       ((acc[0][1] + acc[0][3]) + (acc[1][1] + acc[1][3])) + ((acc[2][1] + acc[2][3]) + (acc[3][1] + acc[3][3])));
     }
+    }
+    if (i < 5) TRACE_STAMP(2, 5 + 2 * i);
   }
   cp_async_wait_pending(0);
   TRACE_STAMP(2, 15);

@@ -505,7 +505,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     const bool d4 = any_vq && cfg->vq_dim == 4;       // four-value code words: uint8 indices only, an even K
     if (d4 && (K > 256 || (K & 1))) ok = false;
     if (gu_vq && (H % 64 != 0 || (r % 8) != 0)) ok = false;       // whole groups of eight blocks / ranks
-    if (!h->dn_dense && (I % 64 != 0 || (r % 8) != 0)) ok = false;
+    if (!h->dn_dense && (I % 64 != 0 || (r % 8) != 0 || H % (8 * kDnVqTiles) != 0)) ok = false;
     if (gu_vq && r > 0 && (P.gate.zslot < 0 || P.up.zslot < 0)) ok = false;
     if (k + S > kMaxK + 8) ok = false;                            // k_combine keeps one partial per slot in shared memory
     h->n_books = gu_vq ? (h->two_books ? 2 : 1) : 0;
@@ -513,6 +513,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->plan_dn = plan_stage(H, I, r, h->dn_dense);
     if (h->plan_gu.n_lr > 0) h->plan_gu.chunk = h->plan_gu.tiles < 16 ? h->plan_gu.tiles : 16;   // mix slice and low-rank parts
     h->plan_dn.n_parts = h->plan_dn.n_slices;          // the down kernel folds the low-rank groups into the slices
+    if (!h->dn_dense) h->plan_dn.tiles = H / (8 * kDnVqTiles);      // a compressed down unit covers kDnVqTiles row tiles
+    h->plan_dn.chunk = h->plan_dn.tiles;
     {
       const char* coop_env = getenv("MOE_VQLR_COOP");      // the persistent kernel walks the groups as parts of their own
       const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) || (coop_env && coop_env[0] == '1');
