@@ -29,7 +29,7 @@ __host__ __device__ inline CoopLayout coop_layout(int K, int n_books, int T, int
   L.cb_u = n_books == 2 ? gu_book : 0;
   size_t o = coop_max((size_t)n_books * gu_book, dn_book);
   L.x = o;      o += pg.x_smem ? (size_t)T * (H / 8 + 1) * 16 : 0;
-  L.dn_slot_u4 = dn_vq ? 2 * kDnVqTiles : 8;
+  L.dn_slot_u4 = dn_vq ? 2 * pd.tpu : 8;
   // the ring serves the gate/up walk, then the down walk (whose first units are requested while
   // the activation phase still runs, hence a scratch region of its own for that phase and the combine)
   size_t region = (size_t)warps * pg.depth * 2 * 32 * 16;

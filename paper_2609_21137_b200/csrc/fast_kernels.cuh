@@ -204,6 +204,8 @@ struct StagePlan {
                    // copy l % 8, so the eight lanes of a quarter warp never share a bank group
   int W;           // warps of the launch that walks this plan (grid * warps per block)
   int only_grp;    // -1: the launch walks every work group; >= 0 (ablation): only this one
+  int tpu;         // compressed down stage: 8-row tiles of H per unit (one set of p fragments, one request group and
+                   // one step of the work cursor for 8 * tpu rows); `tiles` then counts units.  1 elsewhere
   int tail;        // tiles % chunk: length of a shorter last chunk (0: none)
   FastDiv d_per_grp, d_per_chunk, d_chunk, d_tail, d_W;   // n_parts*tiles, n_parts*chunk, chunk, tail, W
 };
@@ -1381,9 +1383,6 @@ __global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos, in
 // are the bf16 hi + lo halves of p.  The warp of slice s also adds the low-rank groups s,
 // s + n_slices, ... (32 ranks each; A = z_d as hi + lo), so the parts are the slices alone.
 // ---------------------------------------------------------------------------------------------
-constexpr int kDnVqTiles = 2;     // a compressed down unit covers this many 8-row tiles of H (one set of p fragments,
-                                  // one request group, one step of the work cursor for 16 rows); the plan's tiles count them
-
 struct DnLayout {
   size_t ring, grp, cb_tmp, total;
   int slot_u4;      // uint4 per lane per ring slot: 2 (indices, factor) or 8 (a dense 256-value slice)
@@ -1392,7 +1391,7 @@ struct DnLayout {
 __host__ __device__ inline DnLayout dn_layout(int K, bool vq, const StagePlan& pl, int warps, int max_groups) {
   DnLayout L;
   size_t o = vq ? (size_t)K * 16 * (pl.repl ? 8 : 1) : 0;
-  L.slot_u4 = vq ? 2 * kDnVqTiles : 8;
+  L.slot_u4 = vq ? 2 * pl.tpu : 8;
   L.ring = o;   o += (size_t)warps * pl.depth * L.slot_u4 * 32 * 16;
   L.grp = o;    o += ((size_t)max_groups * 12 + 15) / 16 * 16;
   L.cb_tmp = o; o += (vq && pl.repl) ? (size_t)K * 16 : 0;
@@ -1410,12 +1409,12 @@ struct DnSmem {
 };
 
 // Streams the bytes of the prefetch cursor's unit into the ring and advances that cursor.
-template <typename IdxT, bool DENSE>
+template <typename IdxT, bool DENSE, int TPU = 2>
 __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, const DnSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3, nb = pl.nb;
   uint4* ring = m.ring;
   const Cursor& pf = w.pf;
-  const size_t row = (size_t)m.grp_e[pf.grp] * P.H + pf.jt * (DENSE ? 8 : 8 * kDnVqTiles) + g;
+  const size_t row = (size_t)m.grp_e[pf.grp] * P.H + pf.jt * (DENSE ? 8 : 8 * TPU) + g;
   if (DENSE) {
     const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + row * P.I) + pf.part * 32 + c;
 #pragma unroll
@@ -1425,9 +1424,9 @@ __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, c
     const IdxT* idx_d = static_cast<const IdxT*>(P.down.idx);
     const int b = pf.part * 32 + 8 * c, rho = pf.part * 32 + 8 * c;
 #pragma unroll
-    for (int sub = 0; sub < kDnVqTiles; ++sub) {
+    for (int sub = 0; sub < TPU; ++sub) {
       const size_t rs = row + 8 * sub;
-      uint4* slot = ring + (size_t)(w.pf_slot * kDnVqTiles + sub) * 2 * 32;
+      uint4* slot = ring + (size_t)(w.pf_slot * TPU + sub) * 2 * 32;
       if (b < nb) cp_async_idx8<IdxT>(slot, idx_d + rs * nb + b);
       if (pf.part < pl.n_lr && rho < P.r) cp_async16(slot + 32, P.down.factor + rs * P.r + rho);
     }
@@ -1437,7 +1436,7 @@ __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, c
 }
 
 // Start of the walk of warp `wid` out of `W` warps (needs only the work groups, not p).
-template <typename IdxT, bool DENSE>
+template <typename IdxT, bool DENSE, int TPU = 2>
 __device__ __forceinline__ void dn_tiles_begin(const Params& P, const StagePlan& pl, const DnSmem& m, int wid, int W, Walk& w) {
   const int per_grp = pl.n_parts * pl.tiles;
   int V = m.n_grp * per_grp, v0 = 0;
@@ -1447,12 +1446,12 @@ __device__ __forceinline__ void dn_tiles_begin(const Params& P, const StagePlan&
   w.pf.set(w.n_my > 0 ? v0 + v_begin : 0, pl);
   w.cur = w.pf;
   w.pf_slot = 0; w.cur_slot = 0;
-  for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) dn_issue<IdxT, DENSE>(P, pl, m, w); cp_async_commit(); }
+  for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) dn_issue<IdxT, DENSE, TPU>(P, pl, m, w); cp_async_commit(); }
   TRACE_STAMP(2, 3);
 }
 
 // The tile loop proper (needs p, z_d and the code book).
-template <typename IdxT, bool DENSE, bool D4 = false>
+template <typename IdxT, bool DENSE, bool D4 = false, int TPU = 2>
 __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const StagePlan& pl, const DnSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
   const int nb = pl.nb, D = pl.depth;
@@ -1463,7 +1462,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
   const int *s_grp_e = m.grp_e, *s_grp_off = m.grp_off, *s_grp_cnt = m.grp_cnt;
   Cursor& cur = w.cur;
   int& cur_slot = w.cur_slot;
-  auto issue = [&]() { dn_issue<IdxT, DENSE>(P, pl, m, w); };
+  auto issue = [&]() { dn_issue<IdxT, DENSE, TPU>(P, pl, m, w); };
 
   uint4 fh[8], fl[8];
   uint4 zh = {0, 0, 0, 0}, zl = {0, 0, 0, 0};     // z_d fragments of the low-rank group this part carries
@@ -1500,8 +1499,8 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
       frag_grp = grp; frag_part = part;
     }
 #pragma unroll
-    for (int sub = 0; sub < (DENSE ? 1 : kDnVqTiles); ++sub) {
-    const int row0 = DENSE ? jt * 8 : (jt * kDnVqTiles + sub) * 8;      // first row of this 8-row tile
+    for (int sub = 0; sub < (DENSE ? 1 : TPU); ++sub) {
+    const int row0 = DENSE ? jt * 8 : (jt * TPU + sub) * 8;      // first row of this 8-row tile
     float acc[4][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // four independent chains
     if (DENSE) {
 #pragma unroll
@@ -1511,7 +1510,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
       }
     } else {
       // mma.sync needs the whole warp: out-of-range block groups use index 0 and zero fragments
-      const uint4* uslot = ring + (size_t)(slot * kDnVqTiles + sub) * 2 * 32;
+      const uint4* uslot = ring + (size_t)(slot * TPU + sub) * 2 * 32;
       uint4 raw = {0, 0, 0, 0};
       if (b0 < nb) raw = ring_idx8<IdxT>(uslot);
       uint32_t id[8];
@@ -1552,7 +1551,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
   TRACE_STAMP(2, 15);
 }
 
-template <typename IdxT, bool DENSE, bool D4 = false>
+template <typename IdxT, bool DENSE, bool D4 = false, int TPU = 2>
 __global__ void __launch_bounds__(kDownThreads, 1)
 k_down_mma(const Params P, int T, const StagePlan pl) {
   extern __shared__ uint4 s_u4[];
@@ -1586,7 +1585,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   m.cb = s_cb; m.ring = ring; m.slot_u4 = L.slot_u4;
   m.grp_e = s_grp_e; m.grp_off = s_grp_off; m.grp_cnt = s_grp_cnt; m.n_grp = n_grp;
   Walk w;
-  dn_tiles_begin<IdxT, DENSE>(P, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps, w);   // index bytes travel ...
+  dn_tiles_begin<IdxT, DENSE, TPU>(P, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps, w);   // index bytes travel ...
   cp_async_wait_pending(D - 1);                                                                // ... the code book has landed
   __syncthreads();
   if (!DENSE && pl.repl) {
@@ -1600,7 +1599,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
     __syncthreads();
   }
   TRACE_STAMP(2, 2);
-  dn_tiles_run<IdxT, DENSE, D4>(P, T, pl, m, w);
+  dn_tiles_run<IdxT, DENSE, D4, TPU>(P, T, pl, m, w);
 }
 
 // out[t][h] = sum over slots (in slot order) of affinity * y[t][slot][h], where y is the sum of

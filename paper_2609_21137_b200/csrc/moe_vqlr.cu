@@ -128,6 +128,7 @@ StagePlan plan_stage(int out_dim, int in_dim, int r, bool dense) {
   pl.chunk = pl.tiles;
   pl.x_smem = 1;
   pl.repl = 0;
+  pl.tpu = 1;
   return pl;
 }
 
@@ -346,9 +347,12 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           StagePlan pl = h->plan_dn;
           if (h->per_expert_launch) pl.only_grp = gi;
           if (h->dn_dense) le = launch_pdl(k_down_mma<uint16_t, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else if (h->d4) le = launch_pdl(k_down_mma<uint16_t, false, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else if (h->idx_bytes == 1) le = launch_pdl(k_down_mma<uint8_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else le = launch_pdl(k_down_mma<uint16_t, false>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else if (h->d4 && pl.tpu == 4) le = launch_pdl(k_down_mma<uint16_t, false, true, 4>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else if (h->d4) le = launch_pdl(k_down_mma<uint16_t, false, true, 2>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else if (h->idx_bytes == 1 && pl.tpu == 4) le = launch_pdl(k_down_mma<uint8_t, false, false, 4>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else if (h->idx_bytes == 1) le = launch_pdl(k_down_mma<uint8_t, false, false, 2>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else if (pl.tpu == 4) le = launch_pdl(k_down_mma<uint16_t, false, false, 4>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          else le = launch_pdl(k_down_mma<uint16_t, false, false, 2>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
         }
         h->launches += n_launch - 1;
         ran = true;
@@ -505,7 +509,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     const bool d4 = any_vq && cfg->vq_dim == 4;       // four-value code words: uint8 indices only, an even K
     if (d4 && (K > 256 || (K & 1))) ok = false;
     if (gu_vq && (H % 64 != 0 || (r % 8) != 0)) ok = false;       // whole groups of eight blocks / ranks
-    if (!h->dn_dense && (I % 64 != 0 || (r % 8) != 0 || H % (8 * kDnVqTiles) != 0)) ok = false;
+    if (!h->dn_dense && (I % 64 != 0 || (r % 8) != 0 || H % 16 != 0)) ok = false;
     if (gu_vq && r > 0 && (P.gate.zslot < 0 || P.up.zslot < 0)) ok = false;
     if (k + S > kMaxK + 8) ok = false;                            // k_combine keeps one partial per slot in shared memory
     h->n_books = gu_vq ? (h->two_books ? 2 : 1) : 0;
@@ -513,7 +517,10 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->plan_dn = plan_stage(H, I, r, h->dn_dense);
     if (h->plan_gu.n_lr > 0) h->plan_gu.chunk = h->plan_gu.tiles < 16 ? h->plan_gu.tiles : 16;   // mix slice and low-rank parts
     h->plan_dn.n_parts = h->plan_dn.n_slices;          // the down kernel folds the low-rank groups into the slices
-    if (!h->dn_dense) h->plan_dn.tiles = H / (8 * kDnVqTiles);      // a compressed down unit covers kDnVqTiles row tiles
+    if (!h->dn_dense && H % 16 == 0) {                  // a compressed down unit covers two or four row tiles (four where
+      h->plan_dn.tpu = (H % 32 == 0 && h->plan_dn.n_slices * (H / 32) >= 256) ? 4 : 2;   // a group still has many units)
+      h->plan_dn.tiles = H / (8 * h->plan_dn.tpu);
+    }
     h->plan_dn.chunk = h->plan_dn.tiles;
     {
       const char* coop_env = getenv("MOE_VQLR_COOP");      // the persistent kernel walks the groups as parts of their own
@@ -568,9 +575,12 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       else if (h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, false, 1>, (cudaFuncAttribute)a, (int)smem_gu);
       else e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
       if (h->dn_dense) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else if (d4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else if (h->idx_bytes == 1) e2 = cudaFuncSetAttribute(k_down_mma<uint8_t, false>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
+      else if (d4 && h->plan_dn.tpu == 4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, true, 4>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
+      else if (d4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, true, 2>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
+      else if (h->idx_bytes == 1 && h->plan_dn.tpu == 4) e2 = cudaFuncSetAttribute(k_down_mma<uint8_t, false, false, 4>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
+      else if (h->idx_bytes == 1) e2 = cudaFuncSetAttribute(k_down_mma<uint8_t, false, false, 2>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
+      else if (h->plan_dn.tpu == 4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, false, 4>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
+      else e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, false, 2>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
       cudaError_t e3 = cudaFuncSetAttribute(k_act_zdown, (cudaFuncAttribute)a, (int)((size_t)I * sizeof(float)));
       if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) { cudaGetLastError(); h->fast = false; }
     }
@@ -616,6 +626,11 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       const int warps = kCoopThreads / 32;
       h->plan_gu_coop = h->plan_gu;
       h->plan_dn_coop = h->plan_dn;
+      if (!h->dn_dense) {                               // the persistent kernel's down walk is built for two tiles per unit
+        h->plan_dn_coop.tpu = 2;
+        h->plan_dn_coop.tiles = H / 16;
+        h->plan_dn_coop.chunk = h->plan_dn_coop.tiles;
+      }
       bool fits = false;
       for (int xs = 1; xs >= 0 && !fits; --xs)
         for (int d = kMaxDepth; d >= 2 && !fits; --d) {

@@ -151,7 +151,8 @@ def test_gelu_long_intermediate():
                                  synth.LayerShape("books4", H=256, I=192, E=8, k=2, d=4, K=512, r=8, T=3,
                                                   per_projection_codebook=True),
                                  synth.LayerShape("olmoe_like", H=2048, I=1024, E=12, k=8, d=4, K=256, r=256,
-                                                  T=4, mode="paper", per_projection_codebook=True)],
+                                                  T=4, mode="paper", per_projection_codebook=True),
+                                 synth.LayerShape("olmoe_full", H=2048, I=1024, E=6, k=2, d=4, K=256, r=32, T=3)],
                          ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
 def test_four_value_code_words(shp):
     """d = 4 (Section 5.5): code words of four values, two indices per eight weights; uint8 and
