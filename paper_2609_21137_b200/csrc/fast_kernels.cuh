@@ -1378,6 +1378,63 @@ __global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos, in
   }
 }
 
+// The same with four consecutive ranks per unit (many pairs: the pair's p values, two thirds of the
+// bytes of a dot product, are loaded once for four basis rows).
+__global__ void __launch_bounds__(256) k_zdown4_pdl(const Params P, int n_pos, int wpd) {
+  // one unit = (pair, four consecutive ranks): the pair's p values are loaded once for the four rows
+  __shared__ float s_part[8][4];
+  pdl_launch();
+  pdl_wait();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int units_per_block = 8 / wpd, rq = P.r / 4;
+  const int d = blockIdx.x * units_per_block + warp / wpd, seg = warp % wpd;
+  const bool live_unit = d < n_pos * rq;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  int pos = 0, rho = 0;
+  if (live_unit) {
+    pos = d / rq; rho = (d - pos * rq) * 4;
+    const uint4* brow = reinterpret_cast<const uint4*>(P.down.basis + (size_t)rho * P.I);
+    const float4* prow = reinterpret_cast<const float4*>(P.p + (size_t)pos * P.I);
+    const int nchunk = P.I / 8;
+    const int per = (nchunk + wpd - 1) / wpd, c_begin = seg * per, c_end = min(nchunk, c_begin + per);
+    for (int c0 = c_begin; c0 < c_end; c0 += 64) {
+      uint4 wv[2][4];
+      float4 pa[2], pb[2];
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int cidx = c0 + q * 32 + lane;
+        const bool live = cidx < c_end;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) wv[q][j] = live ? __ldg(brow + (size_t)j * nchunk + cidx) : make_uint4(0, 0, 0, 0);
+        pa[q] = live ? __ldcg(prow + 2 * cidx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        pb[q] = live ? __ldcg(prow + 2 * cidx + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const float pf[8] = {pa[q].x, pa[q].y, pa[q].z, pa[q].w, pb[q].x, pb[q].y, pb[q].z, pb[q].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float wf[8];
+          unpack8(wv[q][j], wf);
+          acc[j] = dot8(wf, pf, acc[j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[j] = warp_sum(acc[j]);
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) s_part[warp][j] = acc[j];
+  }
+  __syncthreads();
+  if (live_unit && seg == 0 && lane < 4) {
+    float sum = 0.f;
+    for (int q = 0; q < wpd; ++q) sum += s_part[warp + q][lane];
+    P.zd[(size_t)pos * P.r + rho + lane] = sum;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // k_down_mma: partial y tiles for every (work group, slice of I, 8-row tile of H); activations
 // are the bf16 hi + lo halves of p.  The warp of slice s also adds the low-rank groups s,

@@ -334,7 +334,10 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           if (le == cudaSuccess && with_zd) {
             int wpd = 1;                                  // warps per z_d value: 2048 values of I each, at most 8
             while (wpd < 8 && P.I > 2048 * wpd) wpd *= 2;
-            le = launch_pdl(k_zdown_pdl, (n_pos * P.r * wpd + 7) / 8, 256, 0, st, P, n_pos, wpd);
+            if (n_pos * (P.r / 4) * wpd >= 32 * h->sm_count)       // enough warps left with four ranks per unit
+              le = launch_pdl(k_zdown4_pdl, (n_pos * (P.r / 4) * wpd + 7) / 8, 256, 0, st, P, n_pos, wpd);
+            else
+              le = launch_pdl(k_zdown_pdl, (n_pos * P.r * wpd + 7) / 8, 256, 0, st, P, n_pos, wpd);
             h->launches += 1;
           }
         }

@@ -158,3 +158,9 @@ def test_four_value_code_words(shp):
     """d = 4 (Section 5.5): code words of four values, two indices per eight weights; uint8 and
     uint16 indices, shared and separate code books, the shape of the paper's (4, 256, 256) point."""
     _full_check(shp)
+
+
+def test_long_intermediate_many_pairs():
+    # I > 4096 and many (token, expert) pairs: z_d comes from the kernel that takes four ranks per warp
+    shp = synth.LayerShape("longI_b16", H=256, I=4608, E=6, k=3, d=8, K=256, r=128, T=16, router_bias=True)
+    _full_check(shp)
