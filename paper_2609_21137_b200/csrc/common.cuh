@@ -84,7 +84,15 @@ __device__ __forceinline__ float gated_act(float g, float u, int act) {
 __device__ __forceinline__ void stamp(const long long* base_c, int clk_blocks, int kern, int k) {
   long long* base = const_cast<long long*>(base_c);
   if (base && (threadIdx.x & 31) == 0 && k < 16 && (int)blockIdx.x < clk_blocks && (threadIdx.x >> 5) < 16)
-    base[(((size_t)kern * clk_blocks + blockIdx.x) * 16 + (threadIdx.x >> 5)) * 16 + k] = clock64();
+  {
+#ifdef MOE_VQLR_TRACE_GLOBAL      // nanoseconds of the device-wide timer: comparable across SMs and kernels
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+#else
+    const long long t = clock64();
+#endif
+    base[(((size_t)kern * clk_blocks + blockIdx.x) * 16 + (threadIdx.x >> 5)) * 16 + k] = t;
+  }
 }
 
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }

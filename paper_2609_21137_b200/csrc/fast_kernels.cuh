@@ -684,18 +684,18 @@ __device__ __forceinline__ void router_z_finish(const Params& P, const RouterRow
 }
 
 // A single token: the row and the token are requested 2048 values at a time (8 + 8 loads per lane
-// in flight) instead of 512; same summation order.
-__device__ __forceinline__ void router_z_unit_t1(const Params& P, const bf16* __restrict__ x, int unit, int lane) {
-  const RouterRow u = router_z_row(P, 1, unit);
+// in flight) instead of 512; same summation order.  wv holds chunks 0..255 of the row, requested by
+// the caller before it waited for the previous kernel (weights do not depend on it).
+__device__ __forceinline__ void router_z_finish_t1(const Params& P, const RouterRow& u, const bf16* __restrict__ x, int lane, uint4 (&wv)[8]) {
   const int nchunk = P.H / 8;
   const uint4* x4 = reinterpret_cast<const uint4*>(x);
   float acc = 0.f;
   for (int c0 = 0; c0 < nchunk; c0 += 256) {
-    uint4 wv[8], xv[8];
+    uint4 xv[8];
+    if (c0 > 0) router_z_load8(u, c0, nchunk, lane, wv);
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
       const int c = c0 + q * 32 + lane;
-      wv[q] = c < nchunk ? __ldg(u.w4 + c) : make_uint4(0, 0, 0, 0);
       xv[q] = c < nchunk ? __ldg(x4 + c) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
@@ -712,13 +712,10 @@ __device__ __forceinline__ void router_z_unit_t1(const Params& P, const bf16* __
   if (lane == 0) u.dst[0] = sum + u.bias;
 }
 
-// Up to four tokens and a row of at most 2048 values: the whole weight row is requested first (the
-// DRAM round trip), the tokens' chunks follow from L1 / L2; same summation order.
-__device__ __forceinline__ void router_z_unit_row8(const Params& P, const bf16* __restrict__ x, int T, int unit, int lane) {
-  const RouterRow u = router_z_row(P, T, unit);
+// Up to four tokens and a row of at most 2048 values: the whole weight row (wv, requested before
+// the wait) is the DRAM round trip, the tokens' chunks follow from L1 / L2; same summation order.
+__device__ __forceinline__ void router_z_finish_row8(const Params& P, const RouterRow& u, const bf16* __restrict__ x, int lane, uint4 (&wv)[8]) {
   const int nchunk = P.H / 8;
-  uint4 wv[8];
-  router_z_load8(u, 0, nchunk, lane, wv);
   float acc[kTokGroup] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
   for (int q = 0; q < 8; ++q) {
@@ -745,19 +742,40 @@ __device__ __forceinline__ void router_z_unit_row8(const Params& P, const bf16* 
   }
 }
 
+__device__ __forceinline__ void router_z_unit_row8(const Params& P, const bf16* __restrict__ x, int T, int unit, int lane) {
+  const RouterRow u = router_z_row(P, T, unit);
+  uint4 wv[8];
+  router_z_load8(u, 0, P.H / 8, lane, wv);
+  router_z_finish_row8(P, u, x, lane, wv);
+}
+
+// The weight row of a unit is requested BEFORE the wait for the previous kernel of the stream: the
+// weights never depend on it (only the tokens and the logits / z buffers do), so the DRAM round
+// trip of the row overlaps the previous kernel's tail.
 __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
-  pdl_wait();      // the previous call's kernels may still read logits / z
-  pdl_launch();
   int unit = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
-  const int base_units = router_z_units(P, T);
-  if (unit >= router_z_units_launched(P, T)) return;
-  if (unit >= base_units) {          // ablation: a repeated basis row (same operands, same result, same address)
+  const int base_units = router_z_units(P, T), lane = threadIdx.x & 31;
+  const bool has = unit < router_z_units_launched(P, T);
+  if (has && unit >= base_units) {          // ablation: a repeated basis row (same operands, same result, same address)
     const int n_groups = (T + kTokGroup - 1) / kTokGroup;
     unit = P.E * n_groups + (unit - base_units) % (P.n_zrows * n_groups);
   }
-  if (T == 1) router_z_unit_t1(P, x, unit, threadIdx.x & 31);
-  else if (P.H <= 2048) router_z_unit_row8(P, x, T, unit, threadIdx.x & 31);
-  else router_z_unit(P, x, T, unit, threadIdx.x & 31);
+  const bool early = has && (T == 1 || P.H <= 2048);
+  RouterRow u;
+  uint4 wv[8];
+  TRACE_STAMP(0, 8);
+  if (early) {
+    u = router_z_row(P, T, unit);
+    router_z_load8(u, 0, P.H / 8, lane, wv);
+  }
+  pdl_wait();      // the previous call's kernels may still read logits / z; the tokens are its output
+  pdl_launch();
+  TRACE_STAMP(0, 9);
+  if (!has) return;
+  if (T == 1) router_z_finish_t1(P, u, x, lane, wv);
+  else if (P.H <= 2048) router_z_finish_row8(P, u, x, lane, wv);
+  else router_z_unit(P, x, T, unit, lane);
+  TRACE_STAMP(0, 10);
 }
 
 // k_router_zmma_pdl: head of the chain for 9..16 tokens.  The shared projections z = basis * x
@@ -916,6 +934,7 @@ __device__ __forceinline__ void gu_stage_books_async(const Params& P, const Stag
   }
   cp_async_commit();
 }
+
 
 template <bool DENSE>
 __device__ __forceinline__ void gu_stage_async(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,

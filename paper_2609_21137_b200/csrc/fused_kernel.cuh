@@ -506,7 +506,9 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
   const int tid = threadIdx.x, col = tid & 7, q = (tid >> 3) & 3, sl = tid >> 5;
   const int units_per_tok = H2 / kCfCols;
   const int t = blockIdx.x / units_per_tok, h2 = (blockIdx.x - t * units_per_tok) * kCfCols + col;
+  TRACE_STAMP(2, 8);
   pdl_wait();
+  TRACE_STAMP(2, 9);
   pdl_launch();
   // Every load of a thread is requested before the first one is used: the kernel is a handful of
   // dependent round trips long, not a loop of them.
@@ -619,6 +621,7 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
     for (int s = 0; s < n_slots; ++s) { a0 += s_y[s * kCfCols + tid].x; a1 += s_y[s * kCfCols + tid].y; }
     *reinterpret_cast<__nv_bfloat162*>(out + (size_t)t * P.H + 2 * h2) = __floats2bfloat162_rn(a0, a1);
   }
+  TRACE_STAMP(2, 10);
 }
 
 }  // namespace

@@ -23,8 +23,11 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <map>
+#include <mutex>
 #include <new>
 #include <string>
+#include <utility>
 
 namespace {
 
@@ -96,6 +99,22 @@ int fail(moe_vqlr_handle* h, int code, const char* fmt, ...) {
   va_end(ap);
   if (h) h->error = buf; else g_create_error = buf;
   return code;
+}
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize belongs to the kernel (per device), not to a handle:
+// it is only ever raised, so that a handle with a smaller need cannot lower it under a live one.
+std::mutex g_attr_mu;
+std::map<std::pair<int, const void*>, size_t> g_attr_max;
+cudaError_t raise_dyn_smem(const void* fn, size_t bytes) {
+  int dev = 0;
+  cudaError_t ce = cudaGetDevice(&dev);
+  if (ce != cudaSuccess) return ce;
+  std::lock_guard<std::mutex> lock(g_attr_mu);
+  size_t& cur = g_attr_max[std::make_pair(dev, fn)];
+  if (bytes <= cur) return cudaSuccess;
+  ce = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (ce == cudaSuccess) cur = bytes;
+  return ce;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -493,14 +512,13 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     return rc;
   }
   if (h->idx_bytes == 1) {
-    cudaFuncSetAttribute(k_gateup<uint8_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_gu_max);
-    cudaFuncSetAttribute(k_down<uint8_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_down);
+    raise_dyn_smem((const void*)k_gateup<uint8_t>, (size_t)smem_gu_max);
+    raise_dyn_smem((const void*)k_down<uint8_t>, (size_t)h->smem_down);
   } else {
-    cudaFuncSetAttribute(k_gateup<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_gu_max);
-    cudaFuncSetAttribute(k_down<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_down);
+    raise_dyn_smem((const void*)k_gateup<uint16_t>, (size_t)smem_gu_max);
+    raise_dyn_smem((const void*)k_down<uint16_t>, (size_t)h->smem_down);
   }
-  cudaFuncSetAttribute(k_route, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                       (int)((size_t)maxT * E * 4 + (2 * (size_t)E + 1) * 4));
+  raise_dyn_smem((const void*)k_route, (size_t)maxT * E * 4 + (2 * (size_t)E + 1) * 4);
 
   // ---- tensor-core chain: eligibility, plans, shared-memory budgets -------------------------
   {
@@ -566,25 +584,24 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->idx_tc = h->d4 ? 2 : h->idx_bytes;
     if (ok) {
       cudaError_t e1 = cudaSuccess, e2 = cudaSuccess;
-      const int a = cudaFuncAttributeMaxDynamicSharedMemorySize;
-      if (gu_dn) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (d4 && h->lrf2) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true, 2>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (d4 && h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true, 1>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (d4) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, true>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (h->idx_bytes == 1 && h->lrf2) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false, false, 2>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (h->idx_bytes == 1 && h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false, false, 1>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (h->idx_bytes == 1) e1 = cudaFuncSetAttribute(k_gateup_mma<uint8_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (h->lrf2) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, false, 2>, (cudaFuncAttribute)a, (int)smem_gu);
-      else if (h->lrf) e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false, false, 1>, (cudaFuncAttribute)a, (int)smem_gu);
-      else e1 = cudaFuncSetAttribute(k_gateup_mma<uint16_t, false>, (cudaFuncAttribute)a, (int)smem_gu);
-      if (h->dn_dense) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, true>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else if (d4 && h->plan_dn.tpu == 4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, true, 4>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else if (d4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, true, 2>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else if (h->idx_bytes == 1 && h->plan_dn.tpu == 4) e2 = cudaFuncSetAttribute(k_down_mma<uint8_t, false, false, 4>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else if (h->idx_bytes == 1) e2 = cudaFuncSetAttribute(k_down_mma<uint8_t, false, false, 2>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else if (h->plan_dn.tpu == 4) e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, false, 4>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      else e2 = cudaFuncSetAttribute(k_down_mma<uint16_t, false, false, 2>, (cudaFuncAttribute)a, (int)h->smem_fast_dn);
-      cudaError_t e3 = cudaFuncSetAttribute(k_act_zdown, (cudaFuncAttribute)a, (int)((size_t)I * sizeof(float)));
+      if (gu_dn) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, true>, (size_t)smem_gu);
+      else if (d4 && h->lrf2) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, true, 2>, (size_t)smem_gu);
+      else if (d4 && h->lrf) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, true, 1>, (size_t)smem_gu);
+      else if (d4) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, true>, (size_t)smem_gu);
+      else if (h->idx_bytes == 1 && h->lrf2) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint8_t, false, false, 2>, (size_t)smem_gu);
+      else if (h->idx_bytes == 1 && h->lrf) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint8_t, false, false, 1>, (size_t)smem_gu);
+      else if (h->idx_bytes == 1) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint8_t, false>, (size_t)smem_gu);
+      else if (h->lrf2) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, false, 2>, (size_t)smem_gu);
+      else if (h->lrf) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, false, 1>, (size_t)smem_gu);
+      else e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false>, (size_t)smem_gu);
+      if (h->dn_dense) e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, true>, (size_t)h->smem_fast_dn);
+      else if (d4 && h->plan_dn.tpu == 4) e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, false, true, 4>, (size_t)h->smem_fast_dn);
+      else if (d4) e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, false, true, 2>, (size_t)h->smem_fast_dn);
+      else if (h->idx_bytes == 1 && h->plan_dn.tpu == 4) e2 = raise_dyn_smem((const void*)k_down_mma<uint8_t, false, false, 4>, (size_t)h->smem_fast_dn);
+      else if (h->idx_bytes == 1) e2 = raise_dyn_smem((const void*)k_down_mma<uint8_t, false, false, 2>, (size_t)h->smem_fast_dn);
+      else if (h->plan_dn.tpu == 4) e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, false, false, 4>, (size_t)h->smem_fast_dn);
+      else e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, false, false, 2>, (size_t)h->smem_fast_dn);
+      cudaError_t e3 = raise_dyn_smem((const void*)k_act_zdown, (size_t)((size_t)I * sizeof(float)));
       if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) { cudaGetLastError(); h->fast = false; }
     }
   }
@@ -604,8 +621,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
       pl.x_smem = 0; pl.repl = 0;
       h->smem_lr = gu_layout(K, 0, maxT, H, r, pl, kFastThreads / 32, E, k, S).total;
       if (h->smem_lr <= limit &&
-          cudaFuncSetAttribute(k_gateup_lr, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_lr) == cudaSuccess &&
-          cudaFuncSetAttribute(k_gateup_pcb, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pcb_smem_bytes(K)) == cudaSuccess) {
+          raise_dyn_smem((const void*)k_gateup_lr, (size_t)h->smem_lr) == cudaSuccess &&
+          raise_dyn_smem((const void*)k_gateup_pcb, (size_t)pcb_smem_bytes(K)) == cudaSuccess) {
         h->pcb = true;
         h->pcb_Q = (H / 8 + kPcbPiece - 1) / kPcbPiece;
         h->pcb_min_T = 2;
@@ -650,7 +667,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
         const void* fn = h->dn_dense ? (h->idx_bytes == 1 ? (const void*)k_layer_coop<uint8_t, true> : (const void*)k_layer_coop<uint16_t, true>)
                          : h->idx_bytes == 1 ? (const void*)k_layer_coop<uint8_t, false> : (const void*)k_layer_coop<uint16_t, false>;
         int per_sm = 0;
-        cudaError_t e1 = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_coop);
+        cudaError_t e1 = raise_dyn_smem((const void*)fn, (size_t)h->smem_coop);
         if (e1 == cudaSuccess) e1 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kCoopThreads, h->smem_coop);
         if (e1 == cudaSuccess && per_sm >= 1) h->coop = true; else cudaGetLastError();
       }
@@ -743,10 +760,10 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
         else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, false, false); }
         else { MOE_VQLR_FUSED_FN(uint16_t, false, false); }
 #undef MOE_VQLR_FUSED_FN
-        cudaError_t e1 = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+        cudaError_t e1 = raise_dyn_smem((const void*)fn, (size_t)smem_max);
         const size_t cf_smem = ((size_t)(k + S) * (r > 0 ? r : 0) + (size_t)(k + S) * kCfCols * 2) * sizeof(float);
         if (e1 == cudaSuccess && cf_smem > 48 * 1024)
-          e1 = cf_smem <= limit ? cudaFuncSetAttribute(k_combine_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cf_smem) : cudaErrorInvalidValue;
+          e1 = cf_smem <= limit ? raise_dyn_smem((const void*)k_combine_fused, (size_t)cf_smem) : cudaErrorInvalidValue;
         if (e1 == cudaSuccess && maxT_fit >= 1) {
           h->fused = true;
           h->fused_max_T = maxT_fit;

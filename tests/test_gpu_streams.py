@@ -278,3 +278,23 @@ def test_projection_code_book_path(shp, monkeypatch):
         assert_routing(dbg, res)
         assert_output(bf16_tensor_to_f64(out), res.out)
     mod.close()
+
+
+def test_two_live_handles_of_one_kernel_with_different_shared_memory_needs():
+    """The shared-memory limit of a kernel belongs to the kernel, not to a handle: a second handle
+    of the same shape with a smaller need (fewer tokens) must not lower it under the first one."""
+    from paper_2609_21137_b200 import binding
+    shp = synth.shape("qwen3_b16", E=32)
+    layer, res, _ = make_checked_layer(shp, 0)
+    big = binding.MoeVqlrLayer.from_synth(layer, device="cuda", max_tokens=16)
+    small = binding.MoeVqlrLayer.from_synth(layer, device="cuda", max_tokens=1)     # same template instances
+    x = binding.bits_to_device(layer.x, "cuda")
+    out, dbg = big.decode(x, debug=True)            # would fail with ERR_CUDA if the limit had dropped
+    torch.cuda.synchronize()
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out)
+    out1 = small.decode(x[:1])
+    torch.cuda.synchronize()
+    assert torch.isfinite(out1.float()).all()
+    small.close()
+    big.close()
