@@ -76,7 +76,8 @@ enum {
                                          cooperative kernel whose phases are separated by
                                          grid-wide barriers (every wait bounded: a barrier
                                          that gives up reports MOE_VQLR_ERR_TIMEOUT through
-                                         the status word) instead of the chain of five
+                                         the status word, see moe_vqlr_last_status) instead
+                                         of the chain of five
                                          kernels.  Same results; measured slower than the
                                          chain on B200, so off by default.  Ignored where the
                                          configuration cannot use it.  The environment
@@ -92,9 +93,16 @@ enum {
   MOE_VQLR_FLAG_ABLATE_Z_PER_EXPERT = 8u, /* the shared projections z = basis * x are computed
                                          once per selected (and shared) expert instead of once
                                          per token: k + S times the dot products, same values */
-  MOE_VQLR_FLAG_ABLATE_PER_EXPERT_LAUNCH = 16u /* gate/up and down run as one kernel launch per
+  MOE_VQLR_FLAG_ABLATE_PER_EXPERT_LAUNCH = 16u, /* gate/up and down run as one kernel launch per
                                          work group (expert) instead of one launch over all
                                          activated experts; implies the chain of kernels */
+  MOE_VQLR_FLAG_TEST_BARRIER_TIMEOUT = 32u /* test switch, only with MOE_VQLR_FLAG_PERSISTENT: the
+                                         persistent kernel's grid barrier waits for one arrival
+                                         more than will ever come and gives up after 2000 polls
+                                         (about a millisecond), so that the report of a bounded
+                                         wait that ran out (MOE_VQLR_ERR_TIMEOUT through the status
+                                         word) can be exercised without hanging the GPU.  The
+                                         call's output is invalid by construction. */
 };
 
 typedef struct {
@@ -162,6 +170,20 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
  * two pointers; other pointers re-capture it. */
 int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T, void* out_host,
                                void* cuda_stream);
+
+/* The status word of the handle: conditions that only the kernels can detect while a call runs.
+ * Returns MOE_VQLR_OK, or the code a kernel of an earlier call recorded, and clears the word:
+ *   MOE_VQLR_ERR_TIMEOUT      a bounded device-side wait gave up (the grid barrier of the persistent
+ *                             kernel, MOE_VQLR_FLAG_PERSISTENT); that call's output is invalid.  The
+ *                             handle then leaves the persistent kernel for good and runs the chain
+ *                             of kernels, so later calls are correct.
+ *   MOE_VQLR_ERR_INVALID_ARG  a token selected an expert whose router logit is NaN or infinite
+ *                             (non-finite x or router weights); ids stay in range, out is garbage.
+ * The word lives in host memory that the kernels write directly, so reading it copies nothing, but
+ * it is only meaningful once the caller has synchronized the stream of the calls in question.
+ * moe_vqlr_decode_layer_host, which synchronizes anyway, checks it itself and returns the code.
+ * moe_vqlr_last_error() then holds a description. */
+int moe_vqlr_last_status(moe_vqlr_handle* h);
 
 /* Frees the workspace and the handle.  The caller must first make sure no call on this handle
  * is still running on the device.  NULL is accepted. */

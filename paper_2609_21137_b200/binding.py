@@ -22,9 +22,10 @@ FLAG_PERSISTENT = 2
 FLAG_ACT_GELU_TANH = 4
 FLAG_ABLATE_Z_PER_EXPERT = 8
 FLAG_ABLATE_PER_EXPERT_LAUNCH = 16
+FLAG_TEST_BARRIER_TIMEOUT = 32
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
-           "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_launch_count",
+           "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_last_status", "moe_vqlr_launch_count",
            "moe_vqlr_workspace_bytes", "moe_vqlr_set_profiling", "moe_vqlr_last_stage_times",
            "moe_vqlr_stage_count", "moe_vqlr_stage_name", "moe_vqlr_route_noalloc",
            "moe_vqlr_run_stage", "moe_vqlr_phase_clocks", "moe_vqlr_probe_lookup_rate"]
@@ -75,6 +76,8 @@ def _load():
     lib.moe_vqlr_destroy.argtypes = [C.c_void_p]
     lib.moe_vqlr_last_error.restype = C.c_char_p
     lib.moe_vqlr_last_error.argtypes = [C.c_void_p]
+    lib.moe_vqlr_last_status.restype = C.c_int
+    lib.moe_vqlr_last_status.argtypes = [C.c_void_p]
     lib.moe_vqlr_launch_count.restype = C.c_int64
     lib.moe_vqlr_launch_count.argtypes = [C.c_void_p]
     lib.moe_vqlr_workspace_bytes.restype = C.c_int64
@@ -261,6 +264,11 @@ class MoeVqlrLayer:
         buf = np.zeros(n, np.int64)
         got = int(_lib.moe_vqlr_phase_clocks(self._h, buf.ctypes.data_as(C.c_void_p), n))
         return buf.reshape(4, -1, 16, 16) if got == n else None
+
+    def last_status(self) -> int:
+        """Status word of the handle (0, or the code a kernel recorded); reading clears it.
+        Synchronize the stream of the calls in question first."""
+        return int(_lib.moe_vqlr_last_status(self._h))
 
     def set_profiling(self, on: bool) -> None:
         self._check(_lib.moe_vqlr_set_profiling(self._h, 1 if on else 0))

@@ -64,7 +64,9 @@ struct Params {
   float* ypart;            // [parts][maxT*(k+S)][H]  partial down tiles, by pair position
   float* zd_part;          // [maxT*(k+S)][slices][r] partial z_d of the fused kernel's slices
   int* inv_pos;            // [maxT][k+S]       pair position of (token, slot)
-  int* status;             // [1]
+  int* status;             // [1] in pinned host memory mapped into the device: 0, or the code a kernel recorded
+  int spin_limit;          // polls after which a device-side wait gives up (MOE_VQLR_ERR_TIMEOUT)
+  int bar_fault;           // test switch: the persistent kernel's barriers wait for one arrival too many
   unsigned int* grid_bar;  // [2] arrivals and generation of the cooperative kernel's grid barrier
   long long* clk;          // optional phase stamps [kernel 4][block][warp 16][stamp 16], or NULL
   int clk_blocks;
@@ -79,6 +81,11 @@ __device__ __forceinline__ float gated_act(float g, float u, int act) {
   }
   return g / (1.f + expf(-g)) * u;      // silu(g) * u
 }
+
+// Records a device-detected condition for the host (moe_vqlr_last_status).  The word lives in
+// host memory, so it is a plain store: whichever block writes last wins, and every writer of a call
+// reports a failure of that call.
+__device__ __forceinline__ void set_status(const Params& P, int code) { *reinterpret_cast<volatile int*>(P.status) = code; }
 
 // Optional tracing: lane 0 of a warp stores clock64() at phase `k` of kernel `kern`.
 __device__ __forceinline__ void stamp(const long long* base_c, int clk_blocks, int kern, int k) {

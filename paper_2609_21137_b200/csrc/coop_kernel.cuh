@@ -5,15 +5,16 @@
 // code book, tokens and routing lists stay in shared memory across the phases.
 //
 // The grid barrier is a counter + generation pair in global memory.  Co-residency of all blocks
-// is guaranteed by the cooperative launch.  Every wait is bounded: after kGridSyncSpinLimit
-// polls the block records MOE_VQLR_ERR_TIMEOUT in the status word and leaves the kernel.
+// is guaranteed by the cooperative launch.  Every wait is bounded: after Params::spin_limit
+// polls (kGridSyncSpinLimit unless a test shortens it) the block records MOE_VQLR_ERR_TIMEOUT in
+// the status word and leaves the kernel.
 #pragma once
 #include "fast_kernels.cuh"
 
 namespace {
 
 constexpr int kCoopThreads = 384;
-constexpr long long kGridSyncSpinLimit = 1LL << 19;     // x ~0.4 us per poll (an L2 round trip): gives up after ~0.2 s
+constexpr int kGridSyncSpinLimit = 1 << 19;     // x ~0.4 us per poll (an L2 round trip): gives up after ~0.2 s
 
 struct CoopLayout {
   size_t cb_u, x, ring, scratch, z, route, tmp, total;
@@ -57,16 +58,17 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
 // are then out of step and the handle must not be used for further persistent launches.
 constexpr unsigned int kCoopBarriers = 4;
 
-__device__ __forceinline__ bool grid_sync(unsigned int* bar, unsigned int target, int* status) {
+__device__ __forceinline__ bool grid_sync(const Params& P, unsigned int* bar, unsigned int target) {
   __shared__ int s_ok;
   __syncthreads();
   if (threadIdx.x == 0) {
     bool ok = true;
     __threadfence();
     asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
-    long long spins = 0;
+    int spins = 0;
+    target += (unsigned int)P.bar_fault;       // test switch: an arrival that never comes
     while ((int)(ld_acquire_u32(bar) - target) < 0) {
-      if (++spins > kGridSyncSpinLimit) { ok = false; atomicExch(status, MOE_VQLR_ERR_TIMEOUT); break; }
+      if (++spins > P.spin_limit) { ok = false; set_status(P, MOE_VQLR_ERR_TIMEOUT); break; }
     }
     s_ok = ok ? 1 : 0;
   }
@@ -121,7 +123,7 @@ k_layer_coop(const Params P, const bf16* __restrict__ x, bf16* __restrict__ out,
     for (int unit = staged ? unit0 + W : unit0; unit < n_units; unit += W) router_z_unit(P, x, T, unit, lane);
   }
   TRACE_STAMP(3, 1);
-  if (!grid_sync(bar, bar_base + 1u * gridDim.x, P.status)) return;
+  if (!grid_sync(P, bar, bar_base + 1u * gridDim.x)) return;
   TRACE_STAMP(3, 2);
 
   // ---- phase B: routing (every block), gate/up partial tiles
@@ -134,7 +136,7 @@ k_layer_coop(const Params P, const bf16* __restrict__ x, bf16* __restrict__ out,
     gu_tiles_run<IdxT, false>(P, x, T, pg, m, w);
   }
   TRACE_STAMP(3, 4);
-  if (!grid_sync(bar, bar_base + 2u * gridDim.x, P.status)) return;
+  if (!grid_sync(P, bar, bar_base + 2u * gridDim.x)) return;
   TRACE_STAMP(3, 5);
 
   // ---- phase C: sum of parts, SwiGLU, z_d; meanwhile a down code book of its own streams in
@@ -161,7 +163,7 @@ k_layer_coop(const Params P, const bf16* __restrict__ x, bf16* __restrict__ out,
   }
   cp_async_wait_pending(pd.depth - 1);      // the code book (the walk's groups may still travel)
   TRACE_STAMP(3, 6);
-  if (!grid_sync(bar, bar_base + 3u * gridDim.x, P.status)) return;
+  if (!grid_sync(P, bar, bar_base + 3u * gridDim.x)) return;
   TRACE_STAMP(3, 7);
   if (!DN_DENSE && dn_restage && pd.repl) {
     for (int i = tid; i < P.K * 8; i += blockDim.x) m.cb_g[i] = m.tmp[i >> 3];
@@ -171,7 +173,7 @@ k_layer_coop(const Params P, const bf16* __restrict__ x, bf16* __restrict__ out,
   // ---- phase D: down partial tiles (work groups are still in shared memory)
   dn_tiles_run<IdxT, DN_DENSE>(P, T, pd, dm, dw);
   TRACE_STAMP(3, 8);
-  if (!grid_sync(bar, bar_base + 4u * gridDim.x, P.status)) return;
+  if (!grid_sync(P, bar, bar_base + 4u * gridDim.x)) return;
   TRACE_STAMP(3, 9);
   if (blockIdx.x == 0 && tid == 0) bar[1] = bar_epoch + 1u;   // this launch is past its last barrier
 

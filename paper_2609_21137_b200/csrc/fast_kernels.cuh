@@ -316,6 +316,7 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
     unsigned int taken = 0;          // bit j: expert lane + 32 j already selected (E <= 1024)
     unsigned int sel_key = 0;
     int sel_e = 0;
+    bool bad = false;                // fewer than k experts with a finite logit
     if (E <= 256) {                  // keys live in registers
       unsigned int key[8];
 #pragma unroll
@@ -328,7 +329,7 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
           if (!((taken >> j) & 1u) && key[j] > bk) { bk = key[j]; bi = lane + 32 * j; }   // ascending e: '>' keeps the lower id
         const unsigned int mk = __reduce_max_sync(0xffffffffu, bk);
         int win = __reduce_min_sync(0xffffffffu, bk == mk ? bi : 0x7fffffff);
-        if (win >= E) win = s;       // only NaN / -inf left: stay in bounds
+        if (win >= E) { win = s; bad = true; }     // only NaN / -inf left: stay in bounds, report it
         if (lane == (win & 31)) taken |= 1u << (win >> 5);
         if (lane == s) { sel_key = mk; sel_e = win; }
       }
@@ -342,12 +343,16 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
         }
         const unsigned int mk = __reduce_max_sync(0xffffffffu, bk);
         int win = __reduce_min_sync(0xffffffffu, bk == mk ? bi : 0x7fffffff);
-        if (win >= E) win = s;
+        if (win >= E) { win = s; bad = true; }
         if (lane == (win & 31)) taken |= 1u << (win >> 5);
         if (lane == s) { sel_key = mk; sel_e = win; }
       }
     }
     const float sel_l = key_logit(sel_key);
+    // a selected logit that is not finite (NaN sorts above every number here, -inf is only taken
+    // when nothing else is left): the ids stay in bounds, the call is reported as invalid
+    if (lane < k && !(fabsf(sel_l) <= 3.402823466e38f)) bad = true;
+    if (__any_sync(0xffffffffu, bad) && write_global && lane == 0) set_status(P, MOE_VQLR_ERR_INVALID_ARG);
     const float lmax = __shfl_sync(0xffffffffu, sel_l, 0);
     const float ev = lane < k ? expf(sel_l - lmax) : 0.f;
     float denom = ev;

@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(32 * kMaxT) k_route(const Params P, int T) {
       }
       if (bi >= E) {   // only NaN / -inf logits left: keep memory safe and report it
         bi = s;
-        if (lane == 0) atomicExch(P.status, MOE_VQLR_ERR_INVALID_ARG);
+        if (lane == 0) set_status(P, MOE_VQLR_ERR_INVALID_ARG);
       }
       if (lane == s) sel_l = bv;
       if (lane == 0) s_id[t * k + s] = bi;

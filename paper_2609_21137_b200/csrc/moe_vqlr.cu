@@ -72,6 +72,7 @@ struct moe_vqlr_handle {
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
   size_t workspace_bytes;
+  int* status_host;          // the status word: pinned host memory that the kernels write through a mapped pointer
   bf16* x_stage;     // [maxT][H] device staging for the host-buffer entry point
   bf16* out_stage;   // [maxT][H]
   cudaStream_t cap_stream;                 // only ever used to capture the graphs below
@@ -426,6 +427,25 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
   return le;
 }
 
+// Reads and clears the status word (the stream must have been synchronized).  After a device-side
+// timeout the persistent kernel's barrier counters are out of step: they are cleared and the handle
+// goes back to the chain of kernels (graphs captured with the persistent kernel are dropped).
+int take_status(moe_vqlr_handle* h) {
+  const int code = *static_cast<volatile int*>(h->status_host);
+  if (code == MOE_VQLR_OK) return MOE_VQLR_OK;
+  *h->status_host = 0;
+  if (h->coop) {
+    cudaMemset(h->P.grid_bar, 0, 2 * sizeof(unsigned int));
+    h->coop = false;
+    h->P.bar_fault = 0;
+    for (auto& g : h->host_graph) if (g) { cudaGraphExecDestroy(g); g = nullptr; }
+    for (auto& g : h->io_graph) if (g) { cudaGraphExecDestroy(g); g = nullptr; }
+  }
+  return fail(h, code, "a kernel of an earlier call on this handle reported: %s",
+              code == MOE_VQLR_ERR_TIMEOUT ? "a bounded device-side wait gave up (results of that call are invalid)"
+              : code == MOE_VQLR_ERR_INVALID_ARG ? "non-finite router logits" : "error");
+}
+
 }  // namespace
 
 extern "C" {
@@ -458,6 +478,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   h->launches = 0;
   h->want_dbg = 0;
   h->workspace = nullptr;
+  h->status_host = nullptr;
   h->profiling = 0;
   h->cap_stream = nullptr;
   for (auto& g : h->host_graph) g = nullptr;
@@ -781,6 +802,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   const char* clk_env = getenv("MOE_VQLR_PHASE_CLOCKS");
   const bool want_clk = clk_env && clk_env[0] == '1';
   const size_t n_pos = (size_t)maxT * (k + S);
+  unsigned int* idx_max = nullptr;      // scratch of the index validation
   auto plan = [&](char* base) {
     char* cur = base;
     P.logits = carve<float>(cur, (size_t)maxT * E);
@@ -816,7 +838,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     P.zd_part = carve<float>(cur, (h->fused && !h->dn_dense && r > 0) ? n_pos * h->fplan.n_sl * r : 1);
     h->idx_dp = carve<char>(cur, idx_dp_bytes > 0 ? idx_dp_bytes : 1);
     P.inv_pos = carve<int>(cur, n_pos);
-    P.status = carve<int>(cur, 1);
+    idx_max = carve<unsigned int>(cur, 1);
     P.grid_bar = carve<unsigned int>(cur, 2);
     if (want_clk) { P.clk = carve<long long>(cur, (size_t)4 * h->sm_count * 16 * 16); P.clk_blocks = h->sm_count; }
     h->x_stage = carve<bf16>(cur, (size_t)maxT * H);
@@ -833,6 +855,23 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   }
   plan(static_cast<char*>(h->workspace));
   cudaMemset(h->workspace, 0, h->workspace_bytes);
+  // the status word: host memory the device can write, so that reading it costs the host nothing
+  ce = cudaHostAlloc(reinterpret_cast<void**>(&h->status_host), sizeof(int), cudaHostAllocMapped);
+  if (ce == cudaSuccess) {
+    *h->status_host = 0;
+    ce = cudaHostGetDevicePointer(reinterpret_cast<void**>(&P.status), h->status_host, 0);
+  }
+  if (ce != cudaSuccess) {
+    rc = fail(nullptr, MOE_VQLR_ERR_OOM, "status word (mapped host memory): %s", cudaGetErrorString(ce));
+    cudaGetLastError();
+    if (h->status_host) cudaFreeHost(h->status_host);
+    cudaFree(h->workspace);
+    delete h;
+    return rc;
+  }
+  P.spin_limit = kGridSyncSpinLimit;
+  P.bar_fault = 0;
+  if ((cfg->flags & MOE_VQLR_FLAG_TEST_BARRIER_TIMEOUT) && h->coop) { P.spin_limit = 2000; P.bar_fault = 1; }
   if (h->fused && !h->dn_dense) {      // one-off: the down index map per slice
     const FusedPlan& fp = h->fplan;
     if (h->idx_tc == 1)
@@ -842,6 +881,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     ce = cudaDeviceSynchronize();
     if (ce != cudaSuccess) {
       rc = fail(nullptr, MOE_VQLR_ERR_CUDA, "re-laying the down index map: %s", cudaGetErrorString(ce));
+      cudaFreeHost(h->status_host);
       cudaFree(h->workspace);
       delete h;
       return rc;
@@ -849,7 +889,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   }
 
   if (cfg->flags & MOE_VQLR_FLAG_VALIDATE_INDICES) {
-    unsigned int* d_max = reinterpret_cast<unsigned int*>(P.status);
+    unsigned int* d_max = idx_max;
     const moe_vqlr_proj* projs[3] = {&cfg->gate, &cfg->up, &cfg->down};
     for (int i = 0; i < 3; ++i) {
       if (projs[i]->kind != MOE_VQLR_PROJ_VQLR) continue;
@@ -859,10 +899,10 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     }
     unsigned int mx = 0;
     ce = cudaMemcpy(&mx, d_max, sizeof mx, cudaMemcpyDeviceToHost);
-    cudaMemset(P.status, 0, sizeof(int));
     if (ce != cudaSuccess || mx >= (unsigned int)K) {
       rc = ce != cudaSuccess ? fail(nullptr, MOE_VQLR_ERR_CUDA, "index validation: %s", cudaGetErrorString(ce))
                              : fail(nullptr, MOE_VQLR_ERR_BAD_INDEX, "index %u >= codebook_size %d", mx, K);
+      cudaFreeHost(h->status_host);
       cudaFree(h->workspace);
       delete h;
       return rc;
@@ -871,6 +911,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   ce = cudaDeviceSynchronize();
   if (ce != cudaSuccess) {
     rc = fail(nullptr, MOE_VQLR_ERR_CUDA, "create: %s", cudaGetErrorString(ce));
+    cudaFreeHost(h->status_host);
     cudaFree(h->workspace);
     delete h;
     return rc;
@@ -988,7 +1029,7 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
       if (ce2 == cudaSuccess) ce2 = cudaStreamSynchronize(st);
       if (ce2 != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "graph launch with copies: %s", cudaGetErrorString(ce2));
       h->launches += h->host_graph_launches;
-      return MOE_VQLR_OK;
+      return take_status(h);
     }
   }
   cudaError_t ce = cudaMemcpyAsync(h->x_stage, x_host, bytes, cudaMemcpyHostToDevice, st);
@@ -1004,7 +1045,12 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
   ce = cudaMemcpyAsync(out_host, h->out_stage, bytes, cudaMemcpyDeviceToHost, st);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
   if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "copy out: %s", cudaGetErrorString(ce));
-  return MOE_VQLR_OK;
+  return take_status(h);
+}
+
+int moe_vqlr_last_status(moe_vqlr_handle* h) {
+  if (!h) return MOE_VQLR_ERR_INVALID_ARG;
+  return take_status(h);
 }
 
 int moe_vqlr_destroy(moe_vqlr_handle* h) {
@@ -1016,6 +1062,7 @@ int moe_vqlr_destroy(moe_vqlr_handle* h) {
   for (auto& g : h->io_graph)
     if (g) cudaGraphExecDestroy(g);
   if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
+  if (h->status_host) cudaFreeHost(h->status_host);
   cudaError_t ce = cudaFree(h->workspace);
   delete h;
   return ce == cudaSuccess ? MOE_VQLR_OK : MOE_VQLR_ERR_CUDA;

@@ -298,3 +298,70 @@ def test_two_live_handles_of_one_kernel_with_different_shared_memory_needs():
     assert torch.isfinite(out1.float()).all()
     small.close()
     big.close()
+
+
+def test_bounded_wait_that_runs_out_is_reported_and_the_handle_recovers():
+    """The persistent kernel's grid barrier is the library's only device-side spin.  With the test
+    switch it waits for an arrival that never comes and gives up after 2000 polls: every block
+    RETURNS (nothing traps, nothing hangs), the status word says MOE_VQLR_ERR_TIMEOUT, and the
+    handle leaves the persistent kernel, so that the next call is correct."""
+    from paper_2609_21137_b200 import binding
+    shp = synth.shape("tiny", T=2)
+    layer, res, _ = make_checked_layer(shp, 0)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda",
+                                          flags=binding.FLAG_PERSISTENT | binding.FLAG_TEST_BARRIER_TIMEOUT)
+    x = binding.bits_to_device(layer.x, "cuda")
+    assert mod.last_status() == binding.OK
+    before = mod.launch_count
+    mod.decode(x)
+    torch.cuda.synchronize()
+    assert mod.launch_count - before == 1                  # it was the persistent kernel that ran
+    assert mod.last_status() == binding.ERR_TIMEOUT
+    assert mod.last_status() == binding.OK                 # reading clears it
+    out, dbg = mod.decode(x, debug=True)                   # now the chain of kernels
+    torch.cuda.synchronize()
+    assert mod.last_status() == binding.OK
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out)
+    # the host-buffer entry point reports the code by itself
+    mod2 = binding.MoeVqlrLayer.from_synth(layer, device="cuda",
+                                           flags=binding.FLAG_PERSISTENT | binding.FLAG_TEST_BARRIER_TIMEOUT)
+    xh = x.cpu().pin_memory()
+    oh = torch.empty((shp.T, shp.H), dtype=torch.bfloat16).pin_memory()
+    with pytest.raises(binding.MoeVqlrError) as err:
+        mod2.decode_host(xh, oh)
+    assert err.value.status == binding.ERR_TIMEOUT
+    mod2.decode_host(xh, oh)
+    assert_output(bf16_tensor_to_f64(oh), res.out)
+    # and a fresh handle is unaffected
+    fresh = binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_PERSISTENT)
+    out3 = fresh.decode(x)
+    torch.cuda.synchronize()
+    assert fresh.last_status() == binding.OK
+    assert_output(bf16_tensor_to_f64(out3), res.out)
+    for m in (mod, mod2, fresh):
+        m.close()
+
+
+@pytest.mark.parametrize("path", ["default", "generic"])
+def test_non_finite_logits_are_reported(path, monkeypatch):
+    """A NaN in the tokens makes every router logit NaN: the ids stay in range and the status word
+    reports MOE_VQLR_ERR_INVALID_ARG."""
+    from paper_2609_21137_b200 import binding
+    if path == "generic":
+        monkeypatch.setenv("MOE_VQLR_FORCE_GENERIC", "1")
+    shp = synth.shape("tiny", T=2)
+    layer, _, _ = make_checked_layer(shp, 0)
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    xb = layer.x.copy()
+    xb[1, 3] = 0x7FC0                                      # bf16 NaN in token 1
+    x = binding.bits_to_device(xb, "cuda")
+    _, dbg = mod.decode(x, debug=True)
+    torch.cuda.synchronize()
+    ids = dbg["topk_id"].cpu().numpy()
+    assert ids.min() >= 0 and ids.max() < shp.E
+    assert mod.last_status() == binding.ERR_INVALID_ARG
+    mod.decode(binding.bits_to_device(layer.x, "cuda"))
+    torch.cuda.synchronize()
+    assert mod.last_status() == binding.OK
+    mod.close()
