@@ -27,12 +27,24 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) per launch of the dominant kernel, from the ncu captures summarised
-# in profiles/k_gateup_mma_k_down_mma_qwen3_*.md (small case; per-launch traffic is that of the
-# full benchmark because every launch reads one layer's activated experts).
-NCU_TRAFFIC = {("qwen3", "full", "k_expert_fused"): 12.32e6,     # profiles/k_expert_fused_qwen3_b1.md
-               ("qwen3", "full", "k_gateup_mma"): 8.01e6, ("qwen3", "full", "k_down_mma"): 5.36e6,
-               ("qwen3_b16", "full", "k_gateup_mma"): 42.5e6 + 0.37e6, ("qwen3_b16", "full", "k_down_mma"): 28.7e6 + 0.05e6}
+# DRAM bytes (read + write) per launch of the dominant kernels come from the ncu captures
+# summarised under profiles/; the table profiles/dram_traffic.md lists them with their source.
+def ncu_traffic_table():
+    """{(workload, mode, kernel): (bytes per launch, source)} parsed from profiles/dram_traffic.md."""
+    table = {}
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.md")) as f:
+            for line in f:
+                cells = [c.strip() for c in line.strip().strip("|").split("|")]
+                if len(cells) >= 5 and cells[0] not in ("workload", "") and not set(cells[0]) <= set("-: "):
+                    try:
+                        table[(cells[0], cells[1], cells[2].strip("`"))] = (float(cells[3]), cells[4])
+                    except ValueError:
+                        pass
+    except OSError:
+        pass
+    return table
+
 
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
@@ -254,6 +266,45 @@ class Workload:
             self.g_rem.replay()
         return self.reps * self.n_full + self.n_rem
 
+    def timed_regions(self, regions: int):
+        """`regions` timed regions of exactly reps * L + rem calls each, every one bracketed by its own
+        pair of CUDA events on the launching stream; returns (list of ms, launches per region)."""
+        torch = self.torch
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(regions)]
+        n = 0
+        for e0, e1 in ev:
+            e0.record()
+            n = self.timed_region()
+            e1.record()
+        torch.cuda.synchronize(self.device)
+        return [e0.elapsed_time(e1) for e0, e1 in ev], n
+
+    def run_cold_l2(self, samples: int = 48):
+        """One layer call at a time with the L2 flushed before it (a 256 MB buffer is overwritten):
+        device time of the isolated call in microseconds, per sample."""
+        torch = self.torch
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=self.device)
+        graphs = []
+        for j in range(len(self.layers)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self.layers[j].decode(self.xs[j], out=self.outs[j])
+            graphs.append(g)
+        for g in graphs:
+            g.replay()
+        out = []
+        for i in range(samples):
+            flush.fill_(i & 0xFF)
+            torch.cuda.synchronize(self.device)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graphs[i % len(graphs)].replay()
+            e1.record()
+            torch.cuda.synchronize(self.device)
+            out.append(e0.elapsed_time(e1) * 1e3)
+        del flush
+        return out
+
     def run_timed(self, steps: int, warmup: int):
         """Device time of `steps` back-to-back calls in milliseconds (CUDA events on the stream)."""
         torch = self.torch
@@ -296,6 +347,10 @@ class Workload:
         shp = self.shp
         xh = [x.cpu().pin_memory() for x in self.xs]
         oh = [torch.empty((shp.T, shp.H), dtype=torch.bfloat16).pin_memory() for _ in self.xs]
+        # every handle's first host call captures its graphs: do that for ALL layers before the clock
+        # starts, then the requested warm-up
+        for j in range(len(self.layers)):
+            self.layers[j].decode_host(xh[j], oh[j])
         for i in range(warmup):
             j = i % len(self.layers)
             self.layers[j].decode_host(xh[j], oh[j])
@@ -315,6 +370,47 @@ class Workload:
         self.g_full = self.g_rem = None
         self.layers, self.xs, self.outs = [], [], []
         self.torch.cuda.empty_cache()
+
+
+def percentiles(values):
+    v = sorted(values)
+    def q(p):
+        if len(v) == 1:
+            return v[0]
+        pos = p * (len(v) - 1)
+        lo = int(pos)
+        hi = min(lo + 1, len(v) - 1)
+        return v[lo] + (v[hi] - v[lo]) * (pos - lo)
+    return {"median": q(0.5), "p2_5": q(0.025), "p97_5": q(0.975), "min": v[0], "max": v[-1], "n": len(v)}
+
+
+def stage_roofline(wl, workload, mode, peak, peak_kind):
+    """Roofline block of the dominant kernel of a workload: every stage's kernel is replayed alone,
+    back to back over the rotating layers inside a captured graph and timed with CUDA events; the
+    dominant one is the byte-carrying stage that takes longest."""
+    shp = wl.shp
+    stage_ms = wl.run_stage_profile()
+    gu_bytes = sum(b.gateup_kernel for b in wl.bytes) / len(wl.bytes)
+    dn_bytes = sum(b.down_kernel for b in wl.bytes) / len(wl.bytes)
+    stage_bytes = {"gateup": gu_bytes, "down": dn_bytes}
+    kernel_names = {"gateup": "k_gateup_mma", "down": "k_down_mma"}
+    if stage_ms.get("down", 0.0) == 0.0 and stage_ms.get("zdown", 0.0) == 0.0:
+        # the fused expert kernel ran as the "gateup" stage: it streams gate/up and the down indices (or the
+        # dense down matrix); the low-rank factor of a compressed down projection is read by the weighted sum
+        lr_down = 2 * shp.H * shp.r if mode == "full" else 0
+        n_act = sum(b.n_active for b in wl.bytes) / len(wl.bytes)
+        stage_bytes = {"gateup": gu_bytes + dn_bytes - n_act * lr_down}
+        kernel_names = {"gateup": "k_expert_fused"}
+    dominant = max(stage_bytes, key=lambda st: stage_ms.get(st, 0.0))
+    dom_ms = stage_ms[dominant]
+    achieved = stage_bytes[dominant] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
+    traffic, source = ncu_traffic_table().get((workload, mode, kernel_names[dominant]), (None, None))
+    return {"bound": "hbm", "kernel": kernel_names[dominant], "achieved": achieved, "peak": peak,
+            "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+            "traffic": traffic, "traffic_source": source,
+            "algorithmic_bytes_per_launch": stage_bytes[dominant], "us_per_launch": dom_ms * 1e3,
+            "how": "each stage's kernel replayed back to back over the rotating layers in a captured graph, CUDA events",
+            "stage_us": {k_: v * 1e3 for k_, v in stage_ms.items()}}
 
 
 def measure(name, mode, steps, warmup, device, n_layers=0):
@@ -359,52 +455,46 @@ def main():
                     "both": _b.FLAG_ABLATE_Z_PER_EXPERT | _b.FLAG_ABLATE_PER_EXPERT_LAUNCH}[args.ablate]
     wl = Workload(args.workload, args.mode, args.layers, device, flags=ablate_flags)
 
-    # ---- the timed region: W warm-up steps, then exactly K steps ---------------------------
+    # ---- the timed regions: W warm-up steps, then R regions of exactly K steps each -----------
+    # A region of few steps lasts well under a millisecond and one sample of it is noisy, so the
+    # region is repeated (about a second of device time, 5..400 regions, each with its own pair of
+    # CUDA events) and the median region is the value, with the 2.5 / 97.5 percentiles beside it.
     wl.prepare(args.steps)
     wl.warm(args.warmup)
     barrier()
     with ClockSampler(local_rank) as clocks:
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        launches = wl.timed_region()
-        e1.record()
-        torch.cuda.synchronize(device)
-        ms = e0.elapsed_time(e1)
+        first_ms, launches = wl.timed_regions(1)
+        regions = int(max(5, min(400, 1000.0 / max(first_ms[0], 1e-3))))
+        barrier()
+        region_ms, launches = wl.timed_regions(regions)
         barrier()
         t_end = time.time() + 0.8      # keep the same load running so the sampler sees its clocks
         while time.time() < t_end:
             wl.g_full.replay()
             torch.cuda.synchronize(device)
-    ms = max_over_ranks(ms, world, device)
+    per_step_us = percentiles([m * 1e3 / args.steps for m in region_ms])
+    ms = max_over_ranks(per_step_us["median"] * args.steps / 1e3, world, device)
     shp = wl.shp
     ms_per_step = ms / args.steps
     us_per_layer_token = ms_per_step * 1e3 / (shp.T * world)
     layer_gbs = wl.mean_bytes / (ms_per_step * 1e-3) / 1e9
+    timing = {"regions": regions, "steps_per_region": args.steps,
+              "us_per_step": {k_: v for k_, v in per_step_us.items()},
+              "first_region_us_per_step": first_ms[0] * 1e3 / args.steps,
+              "how": "every region is exactly `steps` layer calls between two CUDA events on the launching stream; "
+                     "value = median region (max over ranks), percentiles over the regions of rank 0"}
 
     # ---- per-stage profile for the roofline of the dominant kernel -------------------------
-    stage_ms = wl.run_stage_profile()
-    gu_bytes = sum(b.gateup_kernel for b in wl.bytes) / len(wl.bytes)
-    dn_bytes = sum(b.down_kernel for b in wl.bytes) / len(wl.bytes)
-    stage_bytes = {"gateup": gu_bytes, "down": dn_bytes}
-    kernel_names = {"gateup": "k_gateup_mma", "down": "k_down_mma"}
-    if stage_ms.get("down", 0.0) == 0.0 and stage_ms.get("zdown", 0.0) == 0.0:
-        # the fused expert kernel ran as the "gateup" stage: it streams gate/up and the down indices (or the
-        # dense down matrix); the low-rank factor of a compressed down projection is read by the weighted sum
-        lr_down = 2 * shp.H * shp.r if args.mode == "full" else 0
-        n_act = sum(b.n_active for b in wl.bytes) / len(wl.bytes)
-        stage_bytes = {"gateup": gu_bytes + dn_bytes - n_act * lr_down}
-        kernel_names = {"gateup": "k_expert_fused"}
-    dominant = max(stage_bytes, key=lambda s: stage_ms.get(s, 0.0))
-    dom_ms = stage_ms[dominant]
-    achieved = stage_bytes[dominant] / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": kernel_names[dominant], "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                "traffic": NCU_TRAFFIC.get((args.workload, args.mode, kernel_names[dominant])), "algorithmic_bytes_per_launch": stage_bytes[dominant],
-                "us_per_launch": dom_ms * 1e3,
-                "how": "each stage's kernel replayed back to back over the rotating layers in a captured graph, CUDA events",
-                "stage_us": {k_: v * 1e3 for k_, v in stage_ms.items()},
-                "layer": {"algorithmic_bytes": wl.mean_bytes, "gbs": layer_gbs, "frac_of_measured": layer_gbs / peak,
-                          "frac_of_nominal_8TBs": layer_gbs / NOMINAL_HBM_GBS}}
+    roofline = stage_roofline(wl, args.workload, args.mode, peak, peak_kind)
+    roofline["layer"] = {"algorithmic_bytes": wl.mean_bytes, "gbs": layer_gbs, "frac_of_measured": layer_gbs / peak,
+                         "frac_of_nominal_8TBs": layer_gbs / NOMINAL_HBM_GBS}
+
+    # ---- one isolated call with a cold L2 ---------------------------------------------------
+    cold = None
+    if rank == 0 and not args.no_extras:
+        cs = percentiles(wl.run_cold_l2())
+        cold = {"us_per_layer": cs, "how": "a 256 MB buffer is overwritten before every call (L2 is 126 MB); one call "
+                                           "(its kernels captured as one graph) between two CUDA events; 48 samples over the layers"}
 
     # ---- second bound: shared-memory lookup rate (measured live by a probe kernel) ----------
     lookup_bound = None
@@ -428,11 +518,14 @@ def main():
     e2e_ms, h2d, d2h = wl.run_e2e(e2e_steps, max(3, min(args.warmup, 20)))
     e2e_ms = max_over_ranks(e2e_ms, world, device)
     e2e = {"value": e2e_ms * 1e3 / e2e_steps / (shp.T * world), "unit": "us", "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+           "how": "moe_vqlr_decode_layer_host with pinned host buffers, one call after the other, wall clock around "
+                  "the loop; every handle made one call before the clock started (its first call captures graphs)"}
     n_layers = len(wl.layers)
     wl.close()
 
     extras = []
+    roofline_b16 = None
     if rank == 0 and world == 1 and not args.no_extras:
         todo = [("qwen3", "paper"), ("qwen3", "dense"), ("qwen3_b16", "full"), ("qwen3_b16", "paper"),
                 ("qwen3_b16", "dense"), ("qwen3_deployed", "paper"), ("qwen3_deployed_b16", "paper")]
@@ -442,6 +535,11 @@ def main():
                 w2, r2, _ = measure(name, mode, 960, 96, device)
                 r2["frac_of_measured"] = r2["gbs"] / peak
                 r2["frac_of_nominal_8TBs"] = r2["gbs"] / NOMINAL_HBM_GBS
+                if (name, mode) == ("qwen3_b16", "full"):      # the metric names batch 1 AND batch 16
+                    roofline_b16 = stage_roofline(w2, name, mode, peak, peak_kind)
+                    roofline_b16["layer"] = {"us_per_layer": r2["us_per_layer"], "algorithmic_bytes": r2["algorithmic_bytes"],
+                                             "gbs": r2["gbs"], "frac_of_measured": r2["frac_of_measured"],
+                                             "distinct_experts": r2["distinct_experts"]}
                 w2.close()
                 extras.append(r2)
             except Exception as exc:   # an extra must never take the headline down
@@ -458,9 +556,9 @@ def main():
                 "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
                 "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic",
-                "config": {"workload": f"{args.workload} (H={shp.H} I={shp.I} E={shp.E} k={shp.k} S={shp.S} "
-                                       f"K={shp.K} r={shp.r}) T={shp.T} mode={args.mode}"
+                "config": {"workload": f"{args.workload} T={shp.T} mode={args.mode}"
                                        + (f" ablate={args.ablate}" if args.ablate else ""),
+                           "shape": f"H={shp.H} I={shp.I} E={shp.E} k={shp.k} S={shp.S} K={shp.K} r={shp.r}",
                            "distinct_layers": n_layers,
                            "l2": f"rotation over {n_layers} distinct layers touches "
                                  f"{n_layers * wl.mean_bytes / 1e6:.0f} MB per pass, larger than the 126 MB L2",
@@ -470,7 +568,8 @@ def main():
                 "hbm_gbs": layer_gbs, "hbm_frac_of_measured": layer_gbs / peak,
                 "hbm_frac_of_nominal_8TBs": layer_gbs / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_layer": wl.mean_bytes, "distinct_experts_per_layer": wl.mean_active,
-                "gpu_launches": launches, "clocks": clocks.summary(), "roofline": roofline, "e2e": e2e,
+                "gpu_launches": launches, "clocks": clocks.summary(), "timing": timing, "roofline": roofline,
+                "roofline_b16": roofline_b16, "cold_l2": cold, "e2e": e2e,
                 "lookup_bound": lookup_bound, "cpu_baseline": cpu, "extras": extras}
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -195,8 +195,8 @@ const char* moe_vqlr_last_error(const moe_vqlr_handle* h);
 
 /* Measurement aid (no counterpart in the paper; its profiles come from the Neuron tools,
  * Section 5.1).  With profiling on, every decode call records a CUDA event on the call's
- * stream before and after each stage.  Stages, in order: router_z, route, gateup, zdown, down
- * (moe_vqlr_stage_count() of them, named by moe_vqlr_stage_name()).  The events sit between
+ * stream before and after each stage.  Stages, in order: router_z, route, gateup, zdown, down,
+ * combine (moe_vqlr_stage_count() of them, named by moe_vqlr_stage_name()).  The events sit between
  * the kernels, so a profiled call can run slightly slower than an unprofiled one. */
 int moe_vqlr_set_profiling(moe_vqlr_handle* h, int32_t on);
 
@@ -244,8 +244,11 @@ int moe_vqlr_probe_lookup_rate(int32_t codebook_size, int32_t replicated, double
  * paper: it exists for processes where a memory pool or the host application owns every
  * allocation, so moe_vqlr_create(), which allocates a workspace, is off limits).  Computes
  *   logit[t][e] = <router_w[e], x[t]> (+ router_bias[e]),  the k best experts per token (ties:
- *   lower id) and their affinities, exactly as moe_vqlr_decode_layer does,
- * and writes topk_id[T][k] (int32) and topk_w[T][k] (fp32).  All pointers are DEVICE pointers;
+ *   lower id) and their affinities -- the same definition as in moe_vqlr_decode_layer, with a
+ *   summation order of its own (logits agree to fp32 rounding, so ids can differ where two
+ *   logits are closer than that) --
+ * and writes topk_id[T][k] (int32) and topk_w[T][k] (fp32).  Logits must be finite: with fewer
+ * than k finite logits for a token the remaining slots repeat low expert ids (in range, unflagged).  All pointers are DEVICE pointers;
  * x [T][H] bf16 and router_w [E][H] bf16 must be 16-byte aligned, H a multiple of 8;
  * router_bias [E] fp32 may be NULL.  Asynchronous on cuda_stream.
  *

@@ -40,6 +40,26 @@ def test_mixtral_full_size_b1_sampled_rows(mode):
     _sampled_check(shp, rows)
 
 
+@pytest.mark.parametrize("name,mode", [("mixtral_b4", "full"), ("mixtral_b4", "paper"),
+                                       ("mixtral_b16", "full"), ("mixtral_b16", "paper")])
+def test_mixtral_full_size_batches_sampled_rows(name, mode):
+    # the named batch sizes at the named shape (I = 14336: 56 slices of the down contraction); the
+    # oracle computes the sampled output rows of every (token, expert) pair
+    shp = synth.shape(name, mode=mode)
+    rows = sorted(set(np.random.default_rng(3).integers(0, shp.H, 48).tolist()) | {0, shp.H - 1})
+    _sampled_check(shp, rows)
+
+
+@pytest.mark.parametrize("name,mode", [("qwen3", "paper"), ("qwen3", "dense"), ("qwen3_b16", "paper"),
+                                       ("dsv2lite", "paper"), ("dsv2lite_b8", "paper"),
+                                       ("dsv2lite_deployed", "paper"), ("olmoe_deployed_b16", "paper")])
+def test_named_configurations_at_their_own_expert_count(name, mode):
+    # every output element against the oracle, with the models' E (128 / 64), bf16 down projection
+    shp = synth.shape(name, mode=mode)
+    rows = list(range(shp.H))
+    _sampled_check(shp, rows)
+
+
 def test_more_slices_than_warps_b16():
     # I = 3584 -> 14 slices of the down contraction for 12 warps; every expert active at T = 16
     shp = synth.shape("mixtral_b16", I=3584)
