@@ -80,8 +80,7 @@ enum {
                                          of the chain of five
                                          kernels.  Same results; measured slower than the
                                          chain on B200, so off by default.  Ignored where the
-                                         configuration cannot use it.  The environment
-                                         variable MOE_VQLR_COOP=1 at create() sets it too. */
+                                         configuration cannot use it. */
   MOE_VQLR_FLAG_ACT_GELU_TANH = 4u,   /* the expert activation phi of Section 2.1 (it depends
                                          on the model): p = phi(gate) * up with
                                          phi(g) = 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3)))
@@ -96,6 +95,24 @@ enum {
   MOE_VQLR_FLAG_ABLATE_PER_EXPERT_LAUNCH = 16u, /* gate/up and down run as one kernel launch per
                                          work group (expert) instead of one launch over all
                                          activated experts; implies the chain of kernels */
+  /* Path selection, for tests and A/B measurements.  Which kernels a call runs never changes its
+   * results beyond the summation order; without these flags create() picks the fastest path the
+   * configuration allows. */
+  MOE_VQLR_FLAG_NO_FUSED = 64u,          /* never run a call as router -> one fused expert kernel ->
+                                         weighted sum (the default for calls whose work items fill
+                                         at most one wave of blocks): always the chain of kernels */
+  MOE_VQLR_FLAG_FORCE_FUSED = 128u,      /* ... or run every call that fits its shared memory that way */
+  MOE_VQLR_FLAG_GENERIC_KERNELS = 256u,  /* only the generic CUDA-core kernels (one warp per output
+                                         row), which otherwise serve the shapes the tensor-core
+                                         kernels do not cover */
+  MOE_VQLR_FLAG_PROJECTION_CODE_BOOK = 512u, /* calls with two or more tokens evaluate the VQ term of
+                                         gate / up through per-token projection code books
+                                         T[b][k] = <x_b, codebook[k]> (Section 4.2; needs K <= 256 and
+                                         vq_dim 8; measured slower than the reconstructing tensor-core
+                                         kernel on B200, hence opt-in) */
+  MOE_VQLR_FLAG_PHASE_CLOCKS = 1024u,    /* the tensor-core kernels store clock readings at their phase
+                                         boundaries for moe_vqlr_phase_clocks (moe_vqlr_bench.h); only
+                                         in a library built with -DMOE_VQLR_TRACE */
   MOE_VQLR_FLAG_TEST_BARRIER_TIMEOUT = 32u /* test switch, only with MOE_VQLR_FLAG_PERSISTENT: the
                                          persistent kernel's grid barrier waits for one arrival
                                          more than will ever come and gives up after 2000 polls
@@ -144,13 +161,10 @@ typedef struct {
  * The weights stay where they are (borrowed); the one exception is a copy of the DOWN index map
  * in a slice-major order (same values, at most 1/3 larger), made once here inside the workspace
  * when the configuration can run its single-token calls as router -> one fused expert kernel ->
- * weighted sum (Section 4's fused gate/up -> activation -> down pipeline; see
- * moe_vqlr_workspace_bytes).  Which kernels a call runs (that path, the chain of five kernels, or
- * the generic chain for shapes the tensor-core kernels do not cover) never changes its results
- * beyond the summation order; MOE_VQLR_FUSED=0 in the environment at create() keeps the handle
- * off the fused path, and MOE_VQLR_PCB=1 makes calls with two or more tokens evaluate the VQ term of
- * gate/up through per-token projection code books T[b][k] = <x_b, codebook[k]> (Section 4.2; K <=
- * 256, vq_dim 8; measured slower than the reconstructing tensor-core kernel on B200, hence opt-in). */
+ * weighted sum (Section 4's fused gate/up -> activation -> down pipeline).  Which kernels a call
+ * runs (that path, the chain of five kernels, or the generic chain for shapes the tensor-core
+ * kernels do not cover) never changes its results beyond the summation order; the path-selection
+ * flags above override the choice.  create() reads no environment variable. */
 int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out);
 
 /* Runs the layer for T tokens.  x: [T][H] bf16, device.  out: [T][H] bf16, device, written with
@@ -192,53 +206,6 @@ int moe_vqlr_destroy(moe_vqlr_handle* h);
 /* Text of the last error on this handle ("" if none); with NULL, of the last failed create()
  * on this thread.  The string is owned by the library. */
 const char* moe_vqlr_last_error(const moe_vqlr_handle* h);
-
-/* Measurement aid (no counterpart in the paper; its profiles come from the Neuron tools,
- * Section 5.1).  With profiling on, every decode call records a CUDA event on the call's
- * stream before and after each stage.  Stages, in order: router_z, route, gateup, zdown, down,
- * combine (moe_vqlr_stage_count() of them, named by moe_vqlr_stage_name()).  The events sit between
- * the kernels, so a profiled call can run slightly slower than an unprofiled one. */
-int moe_vqlr_set_profiling(moe_vqlr_handle* h, int32_t on);
-
-/* Waits for the last profiled call on this handle and writes the device time of each stage in
- * milliseconds to ms_out[0..stage_count) (0 for a stage the configuration does not run).
- * cap = capacity of ms_out, at least moe_vqlr_stage_count().  INVALID_ARG when the last call
- * was not profiled. */
-int moe_vqlr_last_stage_times(moe_vqlr_handle* h, float* ms_out, int32_t cap);
-
-int moe_vqlr_stage_count(void);
-const char* moe_vqlr_stage_name(int32_t i);
-
-/* Measurement aid (no counterpart in the paper): enqueues the kernel of ONE stage of the layer
- * on cuda_stream, with the same arguments as moe_vqlr_decode_layer, reading whatever the
- * previous stages of an earlier full call on this handle (same x, same T) left in the
- * workspace.  Lets a benchmark time a single kernel back to back, e.g. inside a captured graph.
- * A stage the configuration does not have enqueues nothing and returns MOE_VQLR_OK.  Stages
- * always run as the separate kernels of the chain, also on a handle created with
- * MOE_VQLR_FLAG_PERSISTENT. */
-int moe_vqlr_run_stage(moe_vqlr_handle* h, int32_t stage, const void* x, int32_t T, void* out,
-                       void* cuda_stream);
-
-/* Tracing aid (no counterpart in the paper).  When the environment variable
- * MOE_VQLR_PHASE_CLOCKS=1 is set at create() and the library was built with -DMOE_VQLR_TRACE,
- * the tensor-core kernels store SM clock readings at their phase boundaries: [kernel 4][block][warp 16][stamp 16] int64.  With out == NULL
- * returns the number of values; otherwise synchronously copies them to the HOST buffer out
- * (cap = its capacity in values) and returns the count, -1 on error, 0 when tracing is off. */
-int64_t moe_vqlr_phase_clocks(moe_vqlr_handle* h, int64_t* out, int64_t cap);
-
-/* Number of kernel launches this handle has enqueued since create(). */
-int64_t moe_vqlr_launch_count(const moe_vqlr_handle* h);
-
-/* Device workspace the handle owns, in bytes. */
-int64_t moe_vqlr_workspace_bytes(const moe_vqlr_handle* h);
-
-/* Measurement aid (no counterpart in the paper): runs a short probe kernel on the current device
- * and returns how many random 16-byte shared-memory reads per clock one SM sustains from a
- * code book of codebook_size entries (replicated != 0: the eightfold bank-replicated layout used
- * for small code books).  This is the rate that bounds the compressed projections.  Synchronous;
- * allocates and frees a few KB.  Returns OK, INVALID_ARG, UNSUPPORTED (book too large for shared
- * memory), OOM or CUDA. */
-int moe_vqlr_probe_lookup_rate(int32_t codebook_size, int32_t replicated, double* lookups_per_clk_per_sm);
 
 /* Routing step only, for callers that must not allocate device memory (no counterpart in the
  * paper: it exists for processes where a memory pool or the host application owns every

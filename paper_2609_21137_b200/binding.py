@@ -1,4 +1,4 @@
-"""Thin ctypes binding of the C ABI in ``include/moe_vqlr.h``: argument marshalling only.
+"""Thin ctypes binding of the C ABI in ``include/moe_vqlr.h`` and ``include/moe_vqlr_bench.h``: argument marshalling only.
 
 Every step of the layer runs in the CUDA library; there is no Python or CPU fallback.  Importing
 this module loads ``csrc/libmoe_vqlr.so`` and raises if it is missing (build it with
@@ -23,6 +23,11 @@ FLAG_ACT_GELU_TANH = 4
 FLAG_ABLATE_Z_PER_EXPERT = 8
 FLAG_ABLATE_PER_EXPERT_LAUNCH = 16
 FLAG_TEST_BARRIER_TIMEOUT = 32
+FLAG_NO_FUSED = 64
+FLAG_FORCE_FUSED = 128
+FLAG_GENERIC_KERNELS = 256
+FLAG_PROJECTION_CODE_BOOK = 512
+FLAG_PHASE_CLOCKS = 1024
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_last_status", "moe_vqlr_launch_count",
@@ -257,7 +262,7 @@ class MoeVqlrLayer:
 
     def phase_clocks(self):
         """Phase stamps of the last call as an int64 array [4][blocks][16][16], or None when the
-        handle was not created with MOE_VQLR_PHASE_CLOCKS=1."""
+        handle was not created with FLAG_PHASE_CLOCKS (or the library was built without tracing)."""
         n = int(_lib.moe_vqlr_phase_clocks(self._h, None, 0))
         if n <= 0:
             return None

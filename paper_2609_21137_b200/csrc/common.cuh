@@ -1,6 +1,7 @@
 // Shared definitions of the CUDA kernels: parameter block, bf16 helpers, warp reductions.
 #pragma once
 #include "moe_vqlr.h"
+#include "moe_vqlr_bench.h"
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>

@@ -18,8 +18,6 @@
 #include "fused_kernel.cuh"
 #include "pcb_kernel.cuh"
 
-#include <cstdlib>
-
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -565,8 +563,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     }
     h->plan_dn.chunk = h->plan_dn.tiles;
     {
-      const char* coop_env = getenv("MOE_VQLR_COOP");      // the persistent kernel walks the groups as parts of their own
-      const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) || (coop_env && coop_env[0] == '1');
+      const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) != 0;      // the persistent kernel walks the groups as parts of their own
       h->lrf = gu_vq && !want_coop && h->plan_gu.n_lr >= h->plan_gu.n_slices;
       h->lrf2 = h->lrf && h->plan_gu.n_lr > h->plan_gu.n_slices;
     }
@@ -581,15 +578,11 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     h->plan_gu.x_smem = 1;
     h->plan_gu.depth = 2;
     if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total > limit) h->plan_gu.x_smem = 0;
-    int gu_max_depth = kMaxDepth;
-    if (const char* dv = getenv("MOE_VQLR_GU_DEPTH")) gu_max_depth = atoi(dv);
-    for (int d = gu_max_depth; d >= 2; --d) {
+    for (int d = kMaxDepth; d >= 2; --d) {
       h->plan_gu.depth = d;
       if (gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total <= limit) break;
     }
-    int dn_max_depth = kMaxDepth;
-    if (const char* dv = getenv("MOE_VQLR_DN_DEPTH")) dn_max_depth = atoi(dv);
-    for (int d = dn_max_depth; d >= 2; --d) {
+    for (int d = kMaxDepth; d >= 2; --d) {
       h->plan_dn.depth = d;
       if (dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total <= limit) break;
     }
@@ -598,8 +591,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
     const size_t smem_gu = gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps, E, k, S).total;
     h->smem_fast_dn = dn_layout(K, !h->dn_dense, h->plan_dn, kDownThreads / 32, maxT * (k + S)).total;
     if (smem_gu > limit || h->smem_fast_dn > limit || (size_t)I * sizeof(float) > limit) ok = false;
-    const char* force = getenv("MOE_VQLR_FORCE_GENERIC");
-    if (force && force[0] == '1') ok = false;
+    if (cfg->flags & MOE_VQLR_FLAG_GENERIC_KERNELS) ok = false;
     h->fast = ok;
     h->d4 = ok && d4;
     h->idx_tc = h->d4 ? 2 : h->idx_bytes;
@@ -633,11 +625,11 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   h->pcb_Q = 0;
   h->smem_lr = 0;
   {
-    const char* penv = getenv("MOE_VQLR_PCB");            // 1: from two tokens on; otherwise off (measured slower than the tensor-core kernel)
+    const bool want_pcb = (cfg->flags & MOE_VQLR_FLAG_PROJECTION_CODE_BOOK) != 0;   // from two tokens on; off by default (measured slower than the tensor-core kernel)
     const bool gu_vq2 = P.gate.kind == MOE_VQLR_PROJ_VQLR && P.up.kind == MOE_VQLR_PROJ_VQLR;
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
     if (h->fast && gu_vq2 && !h->d4 && cfg->vq_dim == kD && h->idx_bytes == 1 && H % 16 == 0 && I % kPcbRows == 0 &&
-        pcb_smem_bytes(K) <= limit && penv && penv[0] == '1') {
+        pcb_smem_bytes(K) <= limit && want_pcb) {
       StagePlan pl = h->plan_gu;
       pl.x_smem = 0; pl.repl = 0;
       h->smem_lr = gu_layout(K, 0, maxT, H, r, pl, kFastThreads / 32, E, k, S).total;
@@ -658,10 +650,9 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   h->dn_restage = 0;
   h->smem_coop = 0;
   {
-    const char* coop_env = getenv("MOE_VQLR_COOP");
     int coop_attr = 0;
     cudaDeviceGetAttribute(&coop_attr, cudaDevAttrCooperativeLaunch, h->device);
-    const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) || (coop_env && coop_env[0] == '1');
+    const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) != 0;
     if (h->fast && !h->d4 && !h->lrf && !h->gu_dense && coop_attr && want_coop) {
       const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
       const int warps = kCoopThreads / 32;
@@ -702,9 +693,9 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   h->idx_dp = nullptr;
   size_t idx_dp_bytes = 0;
   {
-    const char* fenv = getenv("MOE_VQLR_FUSED");
+    const bool no_fused = (cfg->flags & MOE_VQLR_FLAG_NO_FUSED) != 0, force_fused = (cfg->flags & MOE_VQLR_FLAG_FORCE_FUSED) != 0;
     const bool book_ok = h->dn_dense || P.down.codebook == P.gate.codebook || (h->n_books == 2 && P.down.codebook == P.up.codebook);
-    if (h->fast && !h->gu_dense && book_ok && H % 16 == 0 && !(fenv && fenv[0] == '0')) {
+    if (h->fast && !h->gu_dense && book_ok && H % 16 == 0 && !no_fused) {
       const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
       const int tiles = I / 8;
       int target = h->sm_count / (k + S);            // slices per expert that fill the GPU at one token
@@ -737,7 +728,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
           }
       }
       // many thin slices would turn the partial y into the dominant traffic: leave those shapes to the chain
-      const bool forced = fenv && fenv[0] == '1';
+      const bool forced = force_fused;
       h->fused_forced = forced;      // tests: also where the items would not fill the GPU
       if (found && fp.n_sl <= 32 && (forced || (k + S) * fp.n_sl * 2 >= h->sm_count)) {
         fp.d_nsl = make_fastdiv((unsigned int)fp.n_sl);
@@ -799,8 +790,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   }
 
   // workspace
-  const char* clk_env = getenv("MOE_VQLR_PHASE_CLOCKS");
-  const bool want_clk = clk_env && clk_env[0] == '1';
+  const bool want_clk = (cfg->flags & MOE_VQLR_FLAG_PHASE_CLOCKS) != 0;
   const size_t n_pos = (size_t)maxT * (k + S);
   unsigned int* idx_max = nullptr;      // scratch of the index validation
   auto plan = [&](char* base) {

@@ -1,7 +1,7 @@
 // moe_vqlr_probe_lookup_rate: measures how many random 16-byte shared-memory reads per clock one
 // SM sustains from a K-entry code book (the unit of work the compressed projections are made
 // of).  Used by the benchmark to state the lookup-rate bound next to the HBM roofline.
-#include "moe_vqlr.h"
+#include "moe_vqlr_bench.h"
 
 #include <cuda_runtime.h>
 

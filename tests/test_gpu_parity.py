@@ -117,7 +117,7 @@ def test_repeatable_bitwise():
                                  synth.shape("tiny", T=5, act="gelu_tanh", mode="paper"),
                                  synth.shape("qwen3", E=16, T=3, act="gelu_tanh")],
                          ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
-def test_gelu_expert_activation(shp, path, monkeypatch):
+def test_gelu_expert_activation(shp, path):
     """MOE_VQLR_FLAG_ACT_GELU_TANH on every kernel path (the generic kernels, the chain, the fused
     expert kernel, the persistent kernel): p = gelu_tanh(gate) * up as in the oracle; a path that
     ignored the flag would miss the tolerance (SiLU and GELU differ by 15 % at gate = 1)."""
@@ -125,16 +125,9 @@ def test_gelu_expert_activation(shp, path, monkeypatch):
     layer, res, _ = make_checked_layer(shp, 0)
     silu = oracle.OracleLayer.from_synth(layer, act="silu").decode_layer(layer.x)
     assert np.max(np.abs(silu.out - res.out)) > 0.05 * np.max(np.abs(res.out))
-    kw = {}
-    if path == "generic":
-        monkeypatch.setenv("MOE_VQLR_FORCE_GENERIC", "1")
-    elif path == "fused":
-        monkeypatch.setenv("MOE_VQLR_FUSED", "1")
-    elif path == "chain":
-        monkeypatch.setenv("MOE_VQLR_FUSED", "0")
-    elif path == "persistent":
-        kw["flags"] = binding.FLAG_PERSISTENT
-    mod, (out, dbg) = run_gpu(layer, **kw)
+    flags = {"default": 0, "generic": binding.FLAG_GENERIC_KERNELS, "fused": binding.FLAG_FORCE_FUSED,
+             "chain": binding.FLAG_NO_FUSED, "persistent": binding.FLAG_PERSISTENT}[path]
+    mod, (out, dbg) = run_gpu(layer, flags=flags)
     assert_routing(dbg, res)
     assert_output(bf16_tensor_to_f64(out), res.out, what=f"{shp.name} gelu {path}")
     mod.close()

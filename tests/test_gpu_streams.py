@@ -1,7 +1,6 @@
 """The same layer through the other launch routes: a side stream (kernels chained by
 programmatic dependent launch), a captured CUDA graph, and the generic kernels forced on a
 shape the tensor-core kernels would normally take."""
-import os
 
 import numpy as np
 import pytest
@@ -70,11 +69,7 @@ def test_graph_capture_replay():
 def test_generic_kernels_forced(shp):
     from paper_2609_21137_b200 import binding
     layer, res, _ = make_checked_layer(shp, 0)
-    os.environ["MOE_VQLR_FORCE_GENERIC"] = "1"
-    try:
-        mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
-    finally:
-        del os.environ["MOE_VQLR_FORCE_GENERIC"]
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_GENERIC_KERNELS)
     x = binding.bits_to_device(layer.x, "cuda")
     out, dbg = mod.decode(x, debug=True)
     torch.cuda.synchronize()
@@ -116,11 +111,7 @@ def test_fused_expert_kernel_forced(shp):
     items would not fill the GPU: three launches per call, the chain's results."""
     from paper_2609_21137_b200 import binding
     layer, res, _ = make_checked_layer(shp, 0)
-    os.environ["MOE_VQLR_FUSED"] = "1"
-    try:
-        mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
-    finally:
-        del os.environ["MOE_VQLR_FUSED"]
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_FORCE_FUSED)
     x = binding.bits_to_device(layer.x, "cuda")
     for _ in range(2):
         before = mod.launch_count
@@ -138,22 +129,19 @@ def test_fused_single_token_ties_and_no_renorm():
     id ascending) when two router rows are identical, whichever side of the cut the pair falls on."""
     from paper_2609_21137_b200 import binding
     shp = synth.shape("tiny", T=1, E=8, k=3)
-    os.environ["MOE_VQLR_FUSED"] = "1"
-    try:
-        for seed in range(8):
-            for renorm in (True, False):
-                layer, res, _ = make_checked_layer(shp, seed=seed, tie=(6, 2), renorm_topk=renorm)
-                mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", renorm_topk=renorm)
-                x = binding.bits_to_device(layer.x, "cuda")
-                before = mod.launch_count
-                out, dbg = mod.decode(x, debug=True)
-                torch.cuda.synchronize()
-                assert mod.launch_count - before == 3
-                assert_routing(dbg, res)
-                assert_output(bf16_tensor_to_f64(out), res.out)
-                mod.close()
-    finally:
-        del os.environ["MOE_VQLR_FUSED"]
+    for seed in range(8):
+        for renorm in (True, False):
+            layer, res, _ = make_checked_layer(shp, seed=seed, tie=(6, 2), renorm_topk=renorm)
+            mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", renorm_topk=renorm,
+                                                  flags=binding.FLAG_FORCE_FUSED)
+            x = binding.bits_to_device(layer.x, "cuda")
+            before = mod.launch_count
+            out, dbg = mod.decode(x, debug=True)
+            torch.cuda.synchronize()
+            assert mod.launch_count - before == 3
+            assert_routing(dbg, res)
+            assert_output(bf16_tensor_to_f64(out), res.out)
+            mod.close()
 
 
 @pytest.mark.parametrize("shp", [
@@ -166,11 +154,7 @@ def test_fused_odd_expert_counts(shp):
     counts that do not fill its vector loads or its warps, and the forced multi-token path with a bias."""
     from paper_2609_21137_b200 import binding
     layer, res, _ = make_checked_layer(shp, 0)
-    os.environ["MOE_VQLR_FUSED"] = "1"
-    try:
-        mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
-    finally:
-        del os.environ["MOE_VQLR_FUSED"]
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_FORCE_FUSED)
     x = binding.bits_to_device(layer.x, "cuda")
     before = mod.launch_count
     out, dbg = mod.decode(x, debug=True)
@@ -260,15 +244,14 @@ def test_ablation_switches_keep_results(shp):
                                  synth.LayerShape("r0_books", H=1024, I=64, E=8, k=3, d=8, K=64, r=0, T=4,
                                                   per_projection_codebook=True)],
                          ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
-def test_projection_code_book_path(shp, monkeypatch):
-    """MOE_VQLR_PCB=1: gate/up through per-token tables T[b][k] = <x_b, codebook[k]> (Section 4.2)
+def test_projection_code_book_path(shp):
+    """MOE_VQLR_FLAG_PROJECTION_CODE_BOOK: gate/up through per-token tables T[b][k] = <x_b, codebook[k]> (Section 4.2)
     with the low-rank term in a kernel of its own: six launches per call, the oracle's results; one
     and several table pieces, a ragged piece, small code books, rank 0, separate books."""
     from paper_2609_21137_b200 import binding
-    monkeypatch.setenv("MOE_VQLR_PCB", "1")
-    monkeypatch.setenv("MOE_VQLR_FUSED", "0")
     layer, res, _ = make_checked_layer(shp, 0)
-    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda",
+                                          flags=binding.FLAG_PROJECTION_CODE_BOOK | binding.FLAG_NO_FUSED)
     x = binding.bits_to_device(layer.x, "cuda")
     for _ in range(2):
         before = mod.launch_count
@@ -344,15 +327,14 @@ def test_bounded_wait_that_runs_out_is_reported_and_the_handle_recovers():
 
 
 @pytest.mark.parametrize("path", ["default", "generic"])
-def test_non_finite_logits_are_reported(path, monkeypatch):
+def test_non_finite_logits_are_reported(path):
     """A NaN in the tokens makes every router logit NaN: the ids stay in range and the status word
     reports MOE_VQLR_ERR_INVALID_ARG."""
     from paper_2609_21137_b200 import binding
-    if path == "generic":
-        monkeypatch.setenv("MOE_VQLR_FORCE_GENERIC", "1")
     shp = synth.shape("tiny", T=2)
     layer, _, _ = make_checked_layer(shp, 0)
-    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda",
+                                          flags=binding.FLAG_GENERIC_KERNELS if path == "generic" else 0)
     xb = layer.x.copy()
     xb[1, 3] = 0x7FC0                                      # bf16 NaN in token 1
     x = binding.bits_to_device(xb, "cuda")
