@@ -40,7 +40,7 @@ class _Layer(C.Structure):
                 ("router_bias", C.c_void_p), ("gate", _Proj), ("up", _Proj), ("down", _Proj)]
 
 
-ACTIVATIONS = {"silu": 0, "gelu_tanh": 1}     # ORACLE_ACT_* of the C file
+ACTIVATIONS = {"silu": 0, "gelu_tanh": 1, "relu2": 2}     # ORACLE_ACT_* of the C file ("relu2": up-only experts)
 
 _lib = None
 
@@ -103,12 +103,14 @@ class OracleLayer:
 
     def _proj(self, p) -> _Proj:
         P = _Proj()
+        if p is None:              # up-only experts have no gate projection
+            return P
         P.kind = int(p.kind)
         idx = None
         if p.idx is not None:
             idx = np.ascontiguousarray(p.idx)
             assert idx.dtype in (np.uint8, np.uint16)
-            P.idx_bytes = idx.dtype.itemsize
+            P.idx_bytes = 12 if getattr(p, "idx_bits", 0) == 12 else idx.dtype.itemsize
         else:
             P.idx_bytes = 1
         arrs = dict(codebook=_c(p.codebook, np.uint16), idx=idx, basis=_c(p.basis, np.uint16),
@@ -185,6 +187,16 @@ def activation(v, act: str = "silu") -> np.ndarray:
     a = np.atleast_1d(np.asarray(v, dtype=np.float64))
     f = lib().oracle_activation
     return np.array([f(float(t), ACTIVATIONS[act]) for t in a.ravel()]).reshape(a.shape)
+
+
+def read_index(idx: np.ndarray, idx_bytes: int, pos: int) -> int:
+    """Index number ``pos`` of a flat index map stored with 1 or 2 bytes per index, or (12) as
+    twelve-bit indices packed two to three bytes."""
+    a = np.ascontiguousarray(idx)
+    f = lib().oracle_read_index
+    f.restype = C.c_uint32
+    f.argtypes = [C.c_void_p, C.c_int, C.c_size_t]
+    return int(f(a.ctypes.data_as(C.c_void_p), idx_bytes, pos))
 
 
 def topk_affinity(logits: np.ndarray, k: int, renorm: bool = True):

@@ -31,11 +31,12 @@
 #endif
 
 enum { ORACLE_PROJ_VQLR = 0, ORACLE_PROJ_DENSE = 1 };
-enum { ORACLE_ACT_SILU = 0, ORACLE_ACT_GELU_TANH = 1 };
+enum { ORACLE_ACT_SILU = 0, ORACLE_ACT_GELU_TANH = 1,
+       ORACLE_ACT_RELU2_UP_ONLY = 2 /* no gate projection: p = max(W_up x, 0)^2 (Section 5.7) */ };
 
 typedef struct {
   int32_t kind;
-  int32_t idx_bytes;          /* 1 or 2 */
+  int32_t idx_bytes;          /* 1 or 2; 12: indices of 12 bits packed two to three bytes */
   const uint16_t* codebook;   /* [K][d] bf16 */
   const void* idx;            /* [E+S][out][in/d] */
   const uint16_t* basis;      /* [r][in] bf16 or NULL */
@@ -139,9 +140,21 @@ void oracle_group_by_expert(const int32_t* ids, int T, int k, int E, int32_t* co
   offsets[E] = n;
 }
 
+/* Index number `pos` of a map.  The deployed index width b_J(K) grows only when K crosses an
+ * encoding boundary (Appendix "Exact engine-work counts"): one byte up to K = 256, two bytes
+ * beyond, or -- the packed encoding for 256 < K <= 4096 -- twelve bits, two indices to three
+ * bytes, little end first: index 2q sits in byte 3q and the low half of byte 3q+1, index 2q+1 in
+ * the high half of byte 3q+1 and byte 3q+2. */
+uint32_t oracle_read_index(const void* idx, int idx_bytes, size_t pos) {
+  if (idx_bytes == 1) return (uint32_t)((const uint8_t*)idx)[pos];
+  if (idx_bytes == 2) return (uint32_t)((const uint16_t*)idx)[pos];
+  const uint8_t* b = (const uint8_t*)idx + (pos >> 1) * 3;
+  return (pos & 1) ? ((uint32_t)b[1] >> 4) | ((uint32_t)b[2] << 4)
+                   : (uint32_t)b[0] | (((uint32_t)b[1] & 0xfu) << 8);
+}
+
 static uint32_t read_index(const oracle_proj* P, size_t pos) {
-  return P->idx_bytes == 1 ? (uint32_t)((const uint8_t*)P->idx)[pos]
-                           : (uint32_t)((const uint16_t*)P->idx)[pos];
+  return oracle_read_index(P->idx, P->idx_bytes, pos);
 }
 
 /* Dense reconstruction of one projection of expert e (Eq. 1, transposed):
@@ -202,6 +215,12 @@ double oracle_activation(double v, int act) {
  * Wd has n_out rows (H, or fewer when rows are sampled). */
 void oracle_gated_expert(const double* Wg, const double* Wu, const double* Wd, const double* x,
                          int H, int I, int n_out, int act, double* g, double* u, double* p, double* y) {
+  if (act == ORACLE_ACT_RELU2_UP_ONLY) {      /* experts without a gate: p = relu(u)^2, Wg is not read */
+    oracle_matvec(Wu, x, I, H, u);
+    for (int i = 0; i < I; ++i) { g[i] = 0.0; p[i] = u[i] > 0.0 ? u[i] * u[i] : 0.0; }
+    oracle_matvec(Wd, p, n_out, I, y);
+    return;
+  }
   oracle_matvec(Wg, x, I, H, g);
   oracle_matvec(Wu, x, I, H, u);
   for (int i = 0; i < I; ++i) p[i] = oracle_activation(g[i], act) * u[i];
@@ -261,7 +280,7 @@ int oracle_decode_layer(const oracle_layer* L, const uint16_t* x, int T, double*
     const int shared = e >= E;
     const int n_pairs = shared ? T : counts[e];
     if (n_pairs == 0) continue;
-    rc |= oracle_reconstruct(&L->gate, e, I, H, L->d, L->K, L->r, Wg);
+    if (L->act != ORACLE_ACT_RELU2_UP_ONLY) rc |= oracle_reconstruct(&L->gate, e, I, H, L->d, L->K, L->r, Wg);
     rc |= oracle_reconstruct(&L->up, e, I, H, L->d, L->K, L->r, Wu);
     rc |= oracle_reconstruct(&L->down, e, H, I, L->d, L->K, L->r, Wd_full);
     for (int q = 0; q < n_out; ++q) {

@@ -43,7 +43,9 @@ class LayerShape:
     # "dense": all three dense bf16 (the uncompressed comparison layer)
     mode: str = "full"
     per_projection_codebook: bool = False   # False: one code book aliased by all projections
-    act: str = "silu"                       # expert activation phi: "silu" (SwiGLU) or "gelu_tanh" (GeGLU)
+    act: str = "silu"                       # expert activation phi: "silu" (SwiGLU), "gelu_tanh" (GeGLU) or
+                                            # "relu2": up-only experts, p = relu(up)^2, no gate projection
+    idx12: bool = False                     # 256 < K <= 4096: indices stored as 12 bits, two to three bytes
 
     @property
     def idx_dtype(self):
@@ -82,6 +84,11 @@ SHAPES: Dict[str, LayerShape] = {
     "qwen3_5bit": LayerShape("qwen3_5bit", H=2048, I=768, E=128, k=8, d=8, K=256, r=504, T=1,
                              mode="paper", per_projection_codebook=True),
     # the (4, 256, 256) point on the OLMoE shape: four-value code words (generic kernels)
+    # Nemotron-3-Nano-shaped layer at its deployed point (8, 256, 512): up-only ReLU^2 experts, bf16 down projection
+    "nemotron_deployed": LayerShape("nemotron_deployed", H=2688, I=1856, E=128, k=6, d=8, K=256, r=512, T=1,
+                                    mode="paper", per_projection_codebook=True, act="relu2"),
+    # the Qwen3-shaped layer with its K = 4096 indices packed to twelve bits
+    "qwen3_idx12": LayerShape("qwen3_idx12", H=2048, I=768, E=128, k=8, d=8, K=4096, r=64, T=1, idx12=True),
     "olmoe_deployed": LayerShape("olmoe_deployed", H=2048, I=1024, E=64, k=8, d=4, K=256, r=256, T=1,
                                  mode="paper", per_projection_codebook=True),
     "olmoe_deployed_b8": LayerShape("olmoe_deployed_b8", H=2048, I=1024, E=64, k=8, d=4, K=256, r=256, T=8,
@@ -124,7 +131,8 @@ class Projection:
     out_dim: int
     in_dim: int
     codebook: Optional[np.ndarray] = None   # [K][d] bf16 bits
-    idx: Optional[np.ndarray] = None        # [E+S][out][in/d] u8/u16
+    idx: Optional[np.ndarray] = None        # [E+S][out][in/d] u8/u16; idx_bits == 12: packed bytes [E+S][out][in/d*3/2]
+    idx_bits: int = 0                       # 12 for the packed twelve-bit encoding, else 8 * itemsize of idx
     basis: Optional[np.ndarray] = None      # [r][in] bf16 bits
     factor: Optional[np.ndarray] = None     # [E+S][out][r] bf16 bits
     dense: Optional[np.ndarray] = None      # [E+S][out][in] bf16 bits
@@ -147,6 +155,20 @@ def _normal_bf16(rng: np.random.Generator, size, std: float) -> np.ndarray:
     return f32_to_bf16_bits(rng.standard_normal(size, dtype=np.float32) * np.float32(std))
 
 
+def pack12(idx: np.ndarray) -> np.ndarray:
+    """Twelve-bit packing of an index array whose last dimension is even: indices 2q and 2q+1 of a
+    row go to bytes 3q .. 3q+2, little end first (low eight bits of the first; its high four bits
+    with the low four of the second; high eight bits of the second)."""
+    a = np.ascontiguousarray(idx, dtype=np.uint16)
+    assert a.shape[-1] % 2 == 0 and int(a.max(initial=0)) < 4096
+    lo, hi = a[..., 0::2], a[..., 1::2]
+    out = np.empty(a.shape[:-1] + (a.shape[-1] // 2, 3), np.uint8)
+    out[..., 0] = lo & 0xFF
+    out[..., 1] = (lo >> 8) | ((hi & 0xF) << 4)
+    out[..., 2] = hi >> 4
+    return out.reshape(a.shape[:-1] + (a.shape[-1] // 2 * 3,))
+
+
 def make_layer(shp: LayerShape, seed: int = 0) -> Layer:
     """Draw one layer.  Draw order is fixed (router, bias, tokens, code books, bases, indices,
     factors, dense matrices) so that a given (shape, seed) always yields the same bits."""
@@ -162,11 +184,14 @@ def make_layer(shp: LayerShape, seed: int = 0) -> Layer:
           "down": shp.mode == "full"}
     if shp.mode not in ("full", "paper", "dense"):
         raise ValueError(f"unknown mode {shp.mode!r}")
+    names = ("up", "down") if shp.act == "relu2" else ("gate", "up", "down")     # up-only experts: nothing is drawn for a gate
+    if shp.idx12 and not (256 < K <= 4096 and d == 8):
+        raise ValueError("idx12 needs 256 < K <= 4096 and d == 8")
 
     # code books: one per layer (aliased) unless per_projection_codebook
     books = {}
     shared_book = None
-    for p in ("gate", "up", "down"):
+    for p in names:
         if not vq[p]:
             continue
         if shp.per_projection_codebook or shared_book is None:
@@ -178,39 +203,40 @@ def make_layer(shp: LayerShape, seed: int = 0) -> Layer:
         books[p] = book
     # shared bases, std in^-1/2 so that z = B x has about unit variance
     bases = {}
-    for p in ("gate", "up", "down"):
+    for p in names:
         if vq[p] and r > 0:
             out_dim, in_dim = dims[p]
             bases[p] = _normal_bf16(rng, (r, in_dim), in_dim ** -0.5)
     # private index maps, iid uniform on [0, K)
     idxs = {}
-    for p in ("gate", "up", "down"):
+    for p in names:
         if vq[p]:
             out_dim, in_dim = dims[p]
             idxs[p] = rng.integers(0, K, size=(n_exp, out_dim, in_dim // d),
                                    dtype=shp.idx_dtype)
     # private coefficients
     factors = {}
-    for p in ("gate", "up", "down"):
+    for p in names:
         if vq[p] and r > 0:
             out_dim, in_dim = dims[p]
             factors[p] = _normal_bf16(rng, (n_exp, out_dim, r), 0.01)
     # dense projections
     denses = {}
-    for p in ("gate", "up", "down"):
+    for p in names:
         if not vq[p]:
             out_dim, in_dim = dims[p]
             denses[p] = _normal_bf16(rng, (n_exp, out_dim, in_dim), 0.02)
 
     projs = {}
-    for p in ("gate", "up", "down"):
+    for p in names:
         out_dim, in_dim = dims[p]
         if vq[p]:
-            projs[p] = Projection(PROJ_VQLR, out_dim, in_dim, codebook=books[p], idx=idxs[p],
+            projs[p] = Projection(PROJ_VQLR, out_dim, in_dim, codebook=books[p],
+                                  idx=pack12(idxs[p]) if shp.idx12 else idxs[p], idx_bits=12 if shp.idx12 else 0,
                                   basis=bases.get(p), factor=factors.get(p))
         else:
             projs[p] = Projection(PROJ_DENSE_BF16, out_dim, in_dim, dense=denses[p])
-    return Layer(shape=shp, router_w=router_w, router_bias=bias, x=x, gate=projs["gate"],
+    return Layer(shape=shp, router_w=router_w, router_bias=bias, x=x, gate=projs.get("gate"),
                  up=projs["up"], down=projs["down"], seed=seed)
 
 

@@ -412,3 +412,93 @@ def test_generator_is_deterministic_and_bf16_exact():
     bits = synth.f32_to_bf16_bits(v)
     ref = torch.from_numpy(v).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(bits, ref)
+
+
+# ------------------------------------------------------------------------------------------
+# up-only ReLU^2 experts (Section 5.7: the Nemotron-shaped layer) and a padded hidden dimension
+# ------------------------------------------------------------------------------------------
+def test_single_up_only_expert_is_plain_relu2_mlp():
+    """E = 1, k = 1, no gate projection: the layer is x -> W_down relu(W_up x)^2, computed here by
+    torch in fp64 from the oracle's own reconstruction of the two matrices."""
+    shp = small_shape(E=1, k=1, T=3, r=3, act="relu2")
+    layer = synth.make_layer(shp, 9)
+    assert layer.gate is None
+    orc = oracle.OracleLayer.from_synth(layer)
+    res = orc.decode_layer(layer.x)
+    W = {}
+    for p in ("up", "down"):                       # Eq. 1 written out with numpy, not the oracle's routine
+        P = getattr(layer, p)
+        W[p] = torch.from_numpy(f64(P.codebook)[P.idx[0].astype(int)].reshape(P.out_dim, P.in_dim)
+                                + f64(P.factor[0]) @ f64(P.basis))
+    Wu, Wd = W["up"], W["down"]
+    xt = torch.from_numpy(f64(layer.x))
+    ref = (torch.relu(xt @ Wu.T) ** 2) @ Wd.T
+    np.testing.assert_allclose(res.out, ref.numpy(), rtol=1e-12, atol=1e-14)
+    # p >= 0 everywhere, so flipping the sign of the tokens changes the result unless u == 0
+    neg = layer.x ^ np.uint16(0x8000)
+    res2 = orc.decode_layer(neg)
+    ref2 = (torch.relu(-xt @ Wu.T) ** 2) @ Wd.T
+    np.testing.assert_allclose(res2.out, ref2.numpy(), rtol=1e-12, atol=1e-14)
+    assert np.max(np.abs(res2.out - res.out)) > 1e-6
+
+
+def test_up_only_differs_from_a_gated_expert_and_ignores_a_gate():
+    shp = small_shape(T=2, act="relu2")
+    up_only = synth.make_layer(shp, 4)
+    res = oracle.OracleLayer.from_synth(up_only).decode_layer(up_only.x)
+    # the same layer with SOME gate attached and the up-only activation: the gate must not be read
+    gated = synth.make_layer(small_shape(T=2), 5)
+    mixed = synth.Layer(shape=shp, router_w=up_only.router_w, router_bias=None, x=up_only.x, gate=gated.gate,
+                        up=up_only.up, down=up_only.down)
+    res_mixed = oracle.OracleLayer.from_synth(mixed, act="relu2").decode_layer(up_only.x)
+    np.testing.assert_array_equal(res_mixed.out, res.out)
+    res_silu = oracle.OracleLayer.from_synth(mixed, act="silu").decode_layer(up_only.x)
+    assert np.max(np.abs(res_silu.out - res.out)) > 1e-3 * np.max(np.abs(res.out))
+
+
+def test_padding_the_hidden_dimension_with_zero_activations_changes_nothing():
+    """A hidden size that is not a multiple of the block length is padded (Section 5.7): the
+    padded tokens carry zeros there, so whatever the padded weight columns hold -- here random
+    code words and a random low-rank part -- the output rows of the true hidden size equal a dense
+    evaluation on the unpadded matrices."""
+    H_true, H_pad = 44, 48
+    shp = small_shape(H=H_pad, E=1, k=1, T=2, act="relu2")
+    layer = synth.make_layer(shp, 11)
+    x = layer.x.copy()
+    x[:, H_true:] = 0                              # bf16 +0
+    orc = oracle.OracleLayer.from_synth(layer)
+    res = orc.decode_layer(x)
+    Wu = torch.from_numpy(orc.reconstruct("up", 0))[:, :H_true]           # I x H_true
+    Wd = torch.from_numpy(orc.reconstruct("down", 0))[:H_true]            # H_true x I
+    xt = torch.from_numpy(f64(x))[:, :H_true]
+    ref = (torch.relu(xt @ Wu.T) ** 2) @ Wd.T
+    np.testing.assert_allclose(res.out[:, :H_true], ref.numpy(), rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------------------------------------------
+# twelve-bit packed indices (Appendix "Exact engine-work counts": the index width b_J(K))
+# ------------------------------------------------------------------------------------------
+def test_packed_twelve_bit_indices_round_trip_and_equal_the_uint16_layer():
+    rng = np.random.default_rng(0)
+    idx = rng.integers(0, 4096, size=(3, 5, 16), dtype=np.uint16)
+    idx[0, 0, :4] = [0, 4095, 0x0F0, 0xA05]        # extremes and both nibble positions
+    packed = synth.pack12(idx)
+    assert packed.dtype == np.uint8 and packed.shape == (3, 5, 24)
+    # bytes of the first pair by hand: 0x000, 0xFFF -> 00 F0 FF
+    assert packed[0, 0, :3].tolist() == [0x00, 0xF0, 0xFF]
+    flat = idx.reshape(-1)
+    for pos in list(range(40)) + [flat.size - 1]:
+        assert oracle.read_index(packed, 12, pos) == int(flat[pos])
+    # storage: twelve bits per index is three quarters of the uint16 map
+    assert packed.nbytes * 4 == idx.nbytes * 3
+    assert abs(oracle.storage_bits_per_weight(8, 4096, 0, 2048, 768, 128, b_J=12)
+               - (12 / 8 + 16 * 4096 * 8 / (128 * 2048 * 768))) < 1e-12
+    # the layer: same draws, indices packed -> bit-identical oracle output, on every projection
+    a = synth.make_layer(small_shape(K=700, T=2, I=32), 3)           # rows of 6 (gate, up) and 4 (down) indices
+    b = synth.make_layer(small_shape(K=700, T=2, I=32, idx12=True), 3)
+    assert b.gate.idx.dtype == np.uint8 and b.gate.idx_bits == 12
+    ra = oracle.OracleLayer.from_synth(a).decode_layer(a.x)
+    rb = oracle.OracleLayer.from_synth(b).decode_layer(b.x)
+    np.testing.assert_array_equal(ra.out, rb.out)
+    np.testing.assert_array_equal(oracle.OracleLayer.from_synth(b).reconstruct("down", 2),
+                                  oracle.OracleLayer.from_synth(a).reconstruct("down", 2))
