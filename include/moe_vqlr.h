@@ -17,7 +17,8 @@
  *     factor_P[e] * z with z = basis_P * input computed once per token and shared by all
  *     experts (Section 3.2, "z = D^T h"); or W_P,e = dense_P[e] for a projection kept in bf16
  *     (Section 3.1 keeps the down projection uncompressed)
- *   p = phi(W_gate,e x) * (W_up,e x);    y = W_down,e p      (phi = SiLU: SwiGLU expert; or GELU)
+ *   p = phi(W_gate,e x) * (W_up,e x);    y = W_down,e p      (phi = SiLU: SwiGLU expert; or GELU;
+ *                                                            or, without a gate, p = relu(W_up,e x)^2)
  *   out[t] = sum_s a[t][s] * y[t][s]  +  sum over the always-on shared experts of y (weight 1)
  *
  * Symbols: H hidden size, I expert intermediate size, E routed experts, k experts per token,
@@ -86,6 +87,12 @@ enum {
                                          phi(g) = 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3)))
                                          (the GELU form of GeGLU experts, e.g. the Gemma shape)
                                          instead of the default phi = SiLU (SwiGLU experts) */
+  MOE_VQLR_FLAG_ACT_RELU2_UP_ONLY = 4096u, /* experts WITHOUT a gate projection (Section 5.7: the
+                                         Nemotron-shaped layer): p = max(W_up x, 0)^2, y = W_down p.
+                                         The `gate` member of the configuration is ignored.  A hidden
+                                         or intermediate size that is not a multiple of the block
+                                         length is padded by the caller: zero activations in the
+                                         padding make its weights irrelevant */
   /* The next two switches turn OFF one mechanism each, to measure what it buys (the attribution
    * of Section 5.4, part A of its table).  Results are unchanged.  They act on the tensor-core
    * paths; the generic kernels and the persistent kernel ignore them. */

@@ -57,23 +57,26 @@ def projection_private_bytes(kind_vq: bool, out_dim: int, in_dim: int, d: int, K
 
 
 def layer_bytes(*, H: int, I: int, E: int, d: int, K: int, r: int, T: int, mode: str,
-                n_active: int, n_codebooks: int = 1, gate_up_share_basis: bool = False) -> LayerBytes:
+                n_active: int, n_codebooks: int = 1, gate_up_share_basis: bool = False,
+                up_only: bool = False) -> LayerBytes:
     """mode: "full" (gate/up/down VQ+LR), "paper" (down dense bf16), "dense" (all dense bf16).
-    n_active counts distinct activated experts including always-on shared experts."""
+    n_active counts distinct activated experts including always-on shared experts.
+    up_only: experts without a gate projection (one projection onto the intermediate size)."""
+    n_gu = 1 if up_only else 2
     vq_gu = mode in ("full", "paper")
     vq_d = mode == "full"
     shared = 0
     if vq_gu or vq_d:
         shared += n_codebooks * 2 * K * d
     if vq_gu and r > 0:
-        shared += (1 if gate_up_share_basis else 2) * 2 * r * H
+        shared += (1 if gate_up_share_basis or up_only else 2) * 2 * r * H
     if vq_d and r > 0:
         shared += 2 * r * I
     return LayerBytes(router=2 * E * H, shared=shared,
-                      per_expert_gateup=2 * projection_private_bytes(vq_gu, I, H, d, K, r),
+                      per_expert_gateup=n_gu * projection_private_bytes(vq_gu, I, H, d, K, r),
                       per_expert_down=projection_private_bytes(vq_d, H, I, d, K, r),
                       tokens_io=2 * 2 * T * H, n_active=n_active,
-                      lookups_per_expert_gateup=2 * I * (H // d) if vq_gu else 0,
+                      lookups_per_expert_gateup=n_gu * I * (H // d) if vq_gu else 0,
                       lookups_per_expert_down=H * (I // d) if vq_d else 0)
 
 

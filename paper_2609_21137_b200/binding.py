@@ -28,6 +28,7 @@ FLAG_FORCE_FUSED = 128
 FLAG_GENERIC_KERNELS = 256
 FLAG_PROJECTION_CODE_BOOK = 512
 FLAG_PHASE_CLOCKS = 1024
+FLAG_ACT_RELU2_UP_ONLY = 4096
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_last_status", "moe_vqlr_launch_count",
@@ -163,7 +164,7 @@ class MoeVqlrLayer:
     """
 
     def __init__(self, *, H, I, E, k, S=0, d=8, K=0, r=0, max_tokens=16, router_w, router_bias=None,
-                 gate, up, down, renorm_topk=True, flags=0, act="silu"):
+                 gate=None, up, down, renorm_topk=True, flags=0, act="silu"):
         self.H, self.I, self.E, self.k, self.S, self.K, self.r = H, I, E, k, S, K, r
         self.max_tokens = max_tokens
         self._keep = [router_w, router_bias, gate, up, down]
@@ -172,12 +173,14 @@ class MoeVqlrLayer:
         cfg.hidden, cfg.inter, cfg.n_experts, cfg.top_k, cfg.n_shared = H, I, E, k, S
         cfg.vq_dim, cfg.codebook_size, cfg.rank, cfg.max_tokens = d, K, r, max_tokens
         cfg.renorm_topk = 1 if renorm_topk else 0
-        if act not in ("silu", "gelu_tanh"):
+        if act not in ("silu", "gelu_tanh", "relu2"):
             raise ValueError(f"unknown expert activation {act!r}")
-        cfg.flags = flags | (FLAG_ACT_GELU_TANH if act == "gelu_tanh" else 0)
+        cfg.flags = flags | {"silu": 0, "gelu_tanh": FLAG_ACT_GELU_TANH, "relu2": FLAG_ACT_RELU2_UP_ONLY}[act]
         cfg.router_w = router_w.data_ptr()
         cfg.router_bias = None if router_bias is None else router_bias.data_ptr()
         for name, p in (("gate", gate), ("up", up), ("down", down)):
+            if p is None:              # up-only experts ("relu2") have no gate projection
+                continue
             P = getattr(cfg, name)
             dense = p.get("dense")
             P.kind = PROJ_DENSE_BF16 if dense is not None else PROJ_VQLR
@@ -206,6 +209,8 @@ class MoeVqlrLayer:
             return cache[id(a)]
 
         def proj(p):
+            if p is None:
+                return None
             return dict(codebook=up(p.codebook), idx=up(p.idx), basis=up(p.basis),
                         factor=up(p.factor), dense=up(p.dense))
 

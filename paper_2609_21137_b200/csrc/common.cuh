@@ -31,7 +31,8 @@ struct ProjDev {
 
 struct Params {
   int H, I, E, k, S, K, r, renorm;
-  int act;                 // expert activation: 0 = SiLU, 1 = GELU (tanh form)
+  int act;                 // expert activation: 0 = SiLU, 1 = GELU (tanh form), 2 = up-only experts, p = relu(u)^2
+                           // (the gate projection then aliases up: kernels that know skip its work, the rest repeat it)
   int d;                   // VQ block length: 8 (one code word = 16 bytes) or 4 (8 bytes)
   int z_repeat;            // 1; ablation: every basis projection is computed this many times (once per selected expert)
   int n_zrows;             // rows of the stacked basis projection: (distinct gate/up bases) * r
@@ -76,6 +77,10 @@ struct Params {
 // The model-specific expert activation phi applied to the gate output (Section 2.1):
 // p = phi(g) * u.  act is uniform over the launch.
 __device__ __forceinline__ float gated_act(float g, float u, int act) {
+  if (act == 2) {                       // up-only experts (Section 5.7): the gate value is not used
+    const float v = fmaxf(u, 0.f);
+    return v * v;
+  }
   if (act == 1) {
     const float t = tanhf(0.7978845608028654f * (g + 0.044715f * g * g * g));
     return 0.5f * g * (1.f + t) * u;

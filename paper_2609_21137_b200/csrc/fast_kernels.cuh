@@ -1019,16 +1019,17 @@ __device__ __forceinline__ void gu_issue(const Params& P, const StagePlan& pl, c
     const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
     const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx);
     const size_t row = (size_t)m.R.grp_e[w.pf.grp] * P.I + w.pf.jt * 8 + g;
+    const bool up_only = P.act == 2;       // experts without a gate: its bytes are not requested
     if (w.pf.part < pl.n_slices) {
       const int b = w.pf.part * 32 + 8 * c;
       if (b < nb) {
-        cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_g + row * nb + b);
+        if (!up_only) cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_g + row * nb + b);
         cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 1) * 32, idx_u + row * nb + b);
       }
     } else {
       const int rho = (w.pf.part - pl.n_slices) * 32 + 8 * c;
       if (rho < P.r) {
-        cp_async16(ring + (w.pf_slot * 2 + 0) * 32, P.gate.factor + row * P.r + rho);
+        if (!up_only) cp_async16(ring + (w.pf_slot * 2 + 0) * 32, P.gate.factor + row * P.r + rho);
         cp_async16(ring + (w.pf_slot * 2 + 1) * 32, P.up.factor + row * P.r + rho);
       }
     }
@@ -1078,6 +1079,7 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
 
   uint4 fx[8];                       // activation fragments of the current (group, part)
   int frag_grp = -1, frag_part = -1;
+  const bool up_only = P.act == 2;   // experts without a gate projection: only the up products are formed
 
   for (int i = 0; i < n_my; ++i) {
     if (i + D - 1 < n_my) issue();
@@ -1102,11 +1104,11 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
       lr_row = (size_t)R.grp_e[grp] * P.I + jt * 8 + g;
       const int rho = part * 32 + 8 * c, rho2 = rho + pl.n_slices * 32;
       if (rho < P.r) {
-        lf_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho));
+        if (!up_only) lf_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho));
         lf_u = __ldg(reinterpret_cast<const uint4*>(P.up.factor + lr_row * P.r + rho));
       }
       if (LRF == 2 && part + pl.n_slices < pl.n_lr && rho2 < P.r) {
-        lf2_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho2));
+        if (!up_only) lf2_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho2));
         lf2_u = __ldg(reinterpret_cast<const uint4*>(P.up.factor + lr_row * P.r + rho2));
       }
     }
@@ -1128,23 +1130,37 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int b = b0 + 4 * j;
-          vg[j] = b < nb ? __ldg(wg + b) : make_uint4(0, 0, 0, 0);
+          vg[j] = (b < nb && !up_only) ? __ldg(wg + b) : make_uint4(0, 0, 0, 0);
           vu[j] = b < nb ? __ldg(wu + b) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { mma_block(acc_g[j & 1], fx[j], vg[j]); mma_block(acc_u[j & 1], fx[j], vu[j]); }
+        for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], vu[j]);
+        if (!up_only)
+#pragma unroll
+          for (int j = 0; j < 8; ++j) mma_block(acc_g[j & 1], fx[j], vg[j]);
       } else {
         // mma.sync needs the whole warp: lanes whose block group lies beyond the row run it
         // with index 0 and zero activation fragments
         uint4 raw_g = {0, 0, 0, 0}, raw_u = {0, 0, 0, 0};
         if (b0 < nb) {
-          raw_g = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32);
+          if (!up_only) raw_g = ring_idx8<IdxT>(ring + (slot * 2 + 0) * 32);
           raw_u = ring_idx8<IdxT>(ring + (slot * 2 + 1) * 32);
         }
         uint32_t ig[8], iu[8];
         unpack_idx8<IdxT>(raw_g, ig);
         unpack_idx8<IdxT>(raw_u, iu);
-        if (D4) {
+        if (up_only) {                 // one projection: half the code-word reads and mma's
+          if (D4) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], lookup_d4(s_cb_u, iu[j], lane));
+          } else if (pl.repl) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], s_cb_u[(iu[j] << 3) | (lane & 7)]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], s_cb_u[iu[j]]);
+          }
+        } else if (D4) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             mma_block(acc_g[j & 1], fx[j], lookup_d4(s_cb_g, ig[j], lane));
@@ -1170,7 +1186,7 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
       uint4 fg = {0, 0, 0, 0}, fu = {0, 0, 0, 0};
       uint4 zgh = {0, 0, 0, 0}, zgl = {0, 0, 0, 0}, zuh = {0, 0, 0, 0}, zul = {0, 0, 0, 0};
       if (rho0 < P.r) {
-        fg = ring[(slot * 2 + 0) * 32];
+        if (!up_only) fg = ring[(slot * 2 + 0) * 32];
         fu = ring[(slot * 2 + 1) * 32];
         if (tok >= 0) {
           const int ig2 = (tok * 2 + P.gate.zslot) * rb + (rho0 >> 3), iu2 = (tok * 2 + P.up.zslot) * rb + (rho0 >> 3);
@@ -1190,7 +1206,7 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
         } else if (lg != part) {            // further groups of this slice (ranks beyond 64 * n_slices)
           lf_g = lf_u = make_uint4(0, 0, 0, 0);
           if (rho < P.r) {
-            lf_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho));
+            if (!up_only) lf_g = __ldg(reinterpret_cast<const uint4*>(P.gate.factor + lr_row * P.r + rho));
             lf_u = __ldg(reinterpret_cast<const uint4*>(P.up.factor + lr_row * P.r + rho));
           }
         }

@@ -164,6 +164,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     if (u.i == it.ns) { u.part = it.lp; u.tile = it.lt; }
     else if (++u.tile == it.tiles) { u.tile = 0; ++u.part; }
   };
+  const bool up_only = P.act == 2;     // experts without a gate: its bytes are not requested, its products not formed
   int g_rq = 0, g_use = 0;             // gate/up ring: next slot to request into, next to consume
   bool requests_on = true;             // off: the request code runs (and warms the instruction cache) without asking for bytes
   auto gu_request = [&](const Item& it, UnitCur& rq) {                    // requests come in the order of use
@@ -175,13 +176,13 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     if (part < pg.n_slices) {
       const int b = part * 32 + 8 * c;
       if (b < nb && requests_on) {
-        cp_async_idx8<IdxT>(slot, idx_g + row * nb + b);
+        if (!up_only) cp_async_idx8<IdxT>(slot, idx_g + row * nb + b);
         cp_async_idx8<IdxT>(slot + 32, idx_u + row * nb + b);
       }
     } else {
       const int rho = (part - pg.n_slices) * 32 + 8 * c;
       if (rho < P.r && requests_on) {
-        cp_async16(slot, P.gate.factor + row * P.r + rho);
+        if (!up_only) cp_async16(slot, P.gate.factor + row * P.r + rho);
         cp_async16(slot + 32, P.up.factor + row * P.r + rho);
       }
     }
@@ -288,28 +289,28 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
           // mma.sync needs the whole warp: lanes whose block group lies beyond the row run it
           // with index 0 and zero activation fragments
           uint4 raw_g = {0, 0, 0, 0}, raw_u = {0, 0, 0, 0};
-          if (b0 < nb) { raw_g = ring_idx8<IdxT>(slot); raw_u = ring_idx8<IdxT>(slot + 32); }
+          if (b0 < nb) { if (!up_only) raw_g = ring_idx8<IdxT>(slot); raw_u = ring_idx8<IdxT>(slot + 32); }
           uint32_t ig[8], iu[8];
           unpack_idx8<IdxT>(raw_g, ig);
           unpack_idx8<IdxT>(raw_u, iu);
           if (D4) {                   // four-value code words: two 8-byte reads per block
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              mma_block(acc_g[j & 1], fx[j], lookup_d4(m.cb_g, ig[j], lane));
-              mma_block(acc_u[j & 1], fx[j], lookup_d4(m.cb_u, iu[j], lane));
-            }
+            for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], lookup_d4(m.cb_u, iu[j], lane));
+            if (!up_only)
+#pragma unroll
+              for (int j = 0; j < 8; ++j) mma_block(acc_g[j & 1], fx[j], lookup_d4(m.cb_g, ig[j], lane));
           } else if (pg.repl) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              mma_block(acc_g[j & 1], fx[j], m.cb_g[(ig[j] << 3) | (lane & 7)]);
-              mma_block(acc_u[j & 1], fx[j], m.cb_u[(iu[j] << 3) | (lane & 7)]);
-            }
+            for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], m.cb_u[(iu[j] << 3) | (lane & 7)]);
+            if (!up_only)
+#pragma unroll
+              for (int j = 0; j < 8; ++j) mma_block(acc_g[j & 1], fx[j], m.cb_g[(ig[j] << 3) | (lane & 7)]);
           } else {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              mma_block(acc_g[j & 1], fx[j], m.cb_g[ig[j]]);
-              mma_block(acc_u[j & 1], fx[j], m.cb_u[iu[j]]);
-            }
+            for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], m.cb_u[iu[j]]);
+            if (!up_only)
+#pragma unroll
+              for (int j = 0; j < 8; ++j) mma_block(acc_g[j & 1], fx[j], m.cb_g[ig[j]]);
           }
         } else {
           // low-rank unit: B = 8 ranks of this lane's factor row, A = the matching z values (hi, lo)
@@ -317,7 +318,7 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
           uint4 fg = {0, 0, 0, 0}, fu = {0, 0, 0, 0};
           uint4 zgh = {0, 0, 0, 0}, zgl = {0, 0, 0, 0}, zuh = {0, 0, 0, 0}, zul = {0, 0, 0, 0};
           if (rho0 < P.r) {
-            fg = slot[0];
+            if (!up_only) fg = slot[0];
             fu = slot[32];
             if (tok >= 0) {
               const int ig2 = (tok * 2 + P.gate.zslot) * rb + (rho0 >> 3), iu2 = (tok * 2 + P.up.zslot) * rb + (rho0 >> 3);

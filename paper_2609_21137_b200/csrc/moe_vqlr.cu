@@ -448,9 +448,14 @@ int take_status(moe_vqlr_handle* h) {
 
 extern "C" {
 
-int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
+int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
   if (out) *out = nullptr;
-  if (!cfg || !out) return fail(nullptr, MOE_VQLR_ERR_INVALID_ARG, "cfg/out is null");
+  if (!cfg_in || !out) return fail(nullptr, MOE_VQLR_ERR_INVALID_ARG, "cfg/out is null");
+  // Up-only experts have no gate projection: internally it aliases the up projection, so that every
+  // pointer stays valid; the tensor-core kernels skip its bytes and its arithmetic.
+  moe_vqlr_config cfg_local = *cfg_in;
+  if (cfg_local.flags & MOE_VQLR_FLAG_ACT_RELU2_UP_ONLY) cfg_local.gate = cfg_local.up;
+  const moe_vqlr_config* cfg = &cfg_local;
   const int H = cfg->hidden, I = cfg->inter, E = cfg->n_experts, k = cfg->top_k, S = cfg->n_shared;
   const int K = cfg->codebook_size, r = cfg->rank, maxT = cfg->max_tokens;
   if (H <= 0 || I <= 0 || E <= 0 || k <= 0 || S < 0 || r < 0 || maxT <= 0)
@@ -497,7 +502,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg, moe_vqlr_handle** out) {
   memset(&P, 0, sizeof P);
   P.H = H; P.I = I; P.E = E; P.k = k; P.S = S; P.K = any_vq ? K : 0; P.r = r;
   P.renorm = cfg->renorm_topk ? 1 : 0;
-  P.act = (cfg->flags & MOE_VQLR_FLAG_ACT_GELU_TANH) ? 1 : 0;
+  P.act = (cfg->flags & MOE_VQLR_FLAG_ACT_RELU2_UP_ONLY) ? 2 : (cfg->flags & MOE_VQLR_FLAG_ACT_GELU_TANH) ? 1 : 0;
   P.d = cfg->vq_dim;
   P.z_repeat = (cfg->flags & MOE_VQLR_FLAG_ABLATE_Z_PER_EXPERT) ? cfg->top_k + cfg->n_shared : 1;
   h->per_expert_launch = (cfg->flags & MOE_VQLR_FLAG_ABLATE_PER_EXPERT_LAUNCH) != 0;

@@ -38,7 +38,7 @@ def make_device_layer(shp: LayerShape, seed: int, device="cuda") -> dict:
           "down": shp.mode == "full"}
     shared_book = None
     projs = {}
-    for p in ("gate", "up", "down"):
+    for p in (("up", "down") if shp.act == "relu2" else ("gate", "up", "down")):     # up-only experts: no gate
         out_dim, in_dim = dims[p]
         if vq[p]:
             if shp.per_projection_codebook or shared_book is None:
@@ -54,5 +54,5 @@ def make_device_layer(shp: LayerShape, seed: int, device="cuda") -> dict:
         else:
             projs[p] = dict(dense=_normal_bf16(gen, (n_exp, out_dim, in_dim), 0.02, device))
     return dict(H=H, I=I, E=E, k=shp.k, S=S, d=d, K=K if any(vq.values()) else 0, r=r,
-                max_tokens=max(T, 1), router_w=router_w, router_bias=bias, gate=projs["gate"],
+                max_tokens=max(T, 1), router_w=router_w, router_bias=bias, gate=projs.get("gate"),
                 up=projs["up"], down=projs["down"], act=shp.act, x=x)

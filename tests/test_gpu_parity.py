@@ -157,3 +157,42 @@ def test_long_intermediate_many_pairs():
     # I > 4096 and many (token, expert) pairs: z_d comes from the kernel that takes four ranks per warp
     shp = synth.LayerShape("longI_b16", H=256, I=4608, E=6, k=3, d=8, K=256, r=128, T=16, router_bias=True)
     _full_check(shp)
+
+
+@pytest.mark.parametrize("path", ["default", "generic", "fused", "chain", "persistent"])
+@pytest.mark.parametrize("shp", [synth.shape("tiny", T=1, act="relu2"),
+                                 synth.shape("tiny", T=5, act="relu2", mode="paper"),
+                                 synth.shape("qwen3", E=16, T=3, act="relu2"),
+                                 synth.shape("dsv2lite", E=16, T=1, act="relu2")],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}")
+def test_up_only_relu2_experts(shp, path):
+    """MOE_VQLR_FLAG_ACT_RELU2_UP_ONLY on every kernel path: experts without a gate projection,
+    p = relu(W_up x)^2 (Section 5.7).  The tensor-core kernels skip the gate's bytes and products, the
+    other paths repeat the up projection in its place; all must match the oracle, which never
+    reads a gate."""
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    assert layer.gate is None
+    flags = {"default": 0, "generic": binding.FLAG_GENERIC_KERNELS, "fused": binding.FLAG_FORCE_FUSED,
+             "chain": binding.FLAG_NO_FUSED, "persistent": binding.FLAG_PERSISTENT}[path]
+    mod, (out, dbg) = run_gpu(layer, flags=flags)
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out, what=f"{shp.name} relu2 {path}")
+    mod.close()
+
+
+def test_nemotron_shaped_layer_and_a_padded_hidden_size():
+    """The Nemotron-3-Nano-shaped layer at its deployed point (8, 256, 512): H = 2688, I = 1856,
+    up-only ReLU^2 experts, bf16 down projection (fewer experts than the model to keep the oracle
+    quick); and a hidden size that is not a multiple of the block length, padded by the caller with
+    zero activations (the last four values of every token), as the paper's kernel does."""
+    _full_check(synth.shape("nemotron_deployed", E=24))
+    _full_check(synth.shape("nemotron_deployed", E=24, T=6))
+    shp = synth.shape("nemotron_deployed", E=24, T=2, H=2688 + 64)       # "true" hidden size 2748, padded to 2752
+    layer, _, _ = make_checked_layer(shp, 0)
+    layer.x[:, 2748:] = 0
+    res = oracle.OracleLayer.from_synth(layer).decode_layer(layer.x)
+    mod, (out, dbg) = run_gpu(layer)
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out, what="padded hidden size")
+    mod.close()
