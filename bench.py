@@ -201,7 +201,7 @@ class Workload:
         self.name, self.mode, self.device = name, mode, device
         shp = self.shp
         probe = accounting.layer_bytes(H=shp.H, I=shp.I, E=shp.E, d=shp.d, K=shp.K, r=shp.r, T=shp.T,
-                                       mode=mode, n_active=shp.k + shp.S, up_only=shp.act == "relu2")
+                                       mode=mode, n_active=shp.k + shp.S, up_only=shp.act == "relu2", idx12=shp.idx12)
         if n_layers <= 0:       # enough distinct layers that one rotation touches > 2.5x L2
             n_layers = max(4, min(64, -(-int(2.5 * L2_BYTES) // max(probe.total, 1))))
         self.layers, self.xs, self.outs = [], [], []
@@ -219,7 +219,7 @@ class Workload:
             n_act = int((dbg["counts"] > 0).sum().item()) + shp.S
             self.bytes.append(accounting.layer_bytes(H=shp.H, I=shp.I, E=shp.E, d=shp.d, K=shp.K, r=shp.r,
                                                      T=shp.T, mode=mode, n_active=n_act,
-                                                     up_only=shp.act == "relu2"))
+                                                     up_only=shp.act == "relu2", idx12=shp.idx12))
         torch.cuda.synchronize(device)
         self.mean_bytes = sum(b.total for b in self.bytes) / len(self.bytes)
         self.mean_active = sum(b.n_active for b in self.bytes) / len(self.bytes)

@@ -62,8 +62,9 @@ typedef struct {
   int32_t kind;         /* moe_vqlr_proj_kind                                                  */
   int32_t reserved;
   const void* codebook; /* [K][d] bf16                                     (VQLR)             */
-  const void* idx;      /* [E+S][out][in/d], uint8 when K <= 256 else uint16 (VQLR); blocks run
-                           along the contraction dimension `in`                               */
+  const void* idx;      /* [E+S][out][in/d], uint8 when K <= 256 else uint16 (or packed to twelve
+                           bits, MOE_VQLR_FLAG_IDX12) (VQLR); blocks run along the contraction
+                           dimension `in`                                                     */
   const void* basis;    /* [rank][in] bf16 = D^T, shared by all experts   (VQLR, rank > 0)    */
   const void* factor;   /* [E+S][out][rank] bf16 = C_e^T, expert-private  (VQLR, rank > 0)    */
   const void* dense;    /* [E+S][out][in] bf16                            (DENSE_BF16)        */
@@ -93,6 +94,14 @@ enum {
                                          or intermediate size that is not a multiple of the block
                                          length is padded by the caller: zero activations in the
                                          padding make its weights irrelevant */
+  MOE_VQLR_FLAG_IDX12 = 8192u,          /* the index maps hold TWELVE-bit indices, two to three bytes,
+                                         little end first (index 2q: byte 3q and the low half of byte
+                                         3q+1; index 2q+1: the high half of byte 3q+1 and byte 3q+2):
+                                         the index width between one and two bytes for 256 < K <= 4096
+                                         (Appendix "Exact engine-work counts": b_J(K) changes at the
+                                         encoding boundaries of K), a quarter fewer index bytes than
+                                         uint16.  Needs vq_dim 8 and H, I multiples of 16; maps stay
+                                         [E+S][out][in/8] indices, i.e. (in/8)*3/2 bytes per row */
   /* The next two switches turn OFF one mechanism each, to measure what it buys (the attribution
    * of Section 5.4, part A of its table).  Results are unchanged.  They act on the tensor-core
    * paths; the generic kernels and the persistent kernel ignore them. */

@@ -46,19 +46,21 @@ class LayerBytes:
         return self.n_active * (self.lookups_per_expert_gateup + self.lookups_per_expert_down)
 
 
-def index_bits(K: int) -> int:
-    return 8 if K <= 256 else 16
+def index_bits(K: int, idx12: bool = False) -> int:
+    """Deployed index width b_J(K): one byte up to K = 256, two bytes beyond, or twelve bits packed."""
+    return 8 if K <= 256 else (12 if idx12 else 16)
 
 
-def projection_private_bytes(kind_vq: bool, out_dim: int, in_dim: int, d: int, K: int, r: int) -> int:
+def projection_private_bytes(kind_vq: bool, out_dim: int, in_dim: int, d: int, K: int, r: int,
+                             idx12: bool = False) -> int:
     if kind_vq:
-        return out_dim * (in_dim // d) * index_bits(K) // 8 + 2 * out_dim * r
+        return out_dim * (in_dim // d) * index_bits(K, idx12) // 8 + 2 * out_dim * r
     return 2 * out_dim * in_dim
 
 
 def layer_bytes(*, H: int, I: int, E: int, d: int, K: int, r: int, T: int, mode: str,
                 n_active: int, n_codebooks: int = 1, gate_up_share_basis: bool = False,
-                up_only: bool = False) -> LayerBytes:
+                up_only: bool = False, idx12: bool = False) -> LayerBytes:
     """mode: "full" (gate/up/down VQ+LR), "paper" (down dense bf16), "dense" (all dense bf16).
     n_active counts distinct activated experts including always-on shared experts.
     up_only: experts without a gate projection (one projection onto the intermediate size)."""
@@ -73,8 +75,8 @@ def layer_bytes(*, H: int, I: int, E: int, d: int, K: int, r: int, T: int, mode:
     if vq_d and r > 0:
         shared += 2 * r * I
     return LayerBytes(router=2 * E * H, shared=shared,
-                      per_expert_gateup=n_gu * projection_private_bytes(vq_gu, I, H, d, K, r),
-                      per_expert_down=projection_private_bytes(vq_d, H, I, d, K, r),
+                      per_expert_gateup=n_gu * projection_private_bytes(vq_gu, I, H, d, K, r, idx12),
+                      per_expert_down=projection_private_bytes(vq_d, H, I, d, K, r, idx12),
                       tokens_io=2 * 2 * T * H, n_active=n_active,
                       lookups_per_expert_gateup=n_gu * I * (H // d) if vq_gu else 0,
                       lookups_per_expert_down=H * (I // d) if vq_d else 0)

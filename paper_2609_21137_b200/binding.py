@@ -29,6 +29,7 @@ FLAG_GENERIC_KERNELS = 256
 FLAG_PROJECTION_CODE_BOOK = 512
 FLAG_PHASE_CLOCKS = 1024
 FLAG_ACT_RELU2_UP_ONLY = 4096
+FLAG_IDX12 = 8192
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_last_status", "moe_vqlr_launch_count",
@@ -164,7 +165,7 @@ class MoeVqlrLayer:
     """
 
     def __init__(self, *, H, I, E, k, S=0, d=8, K=0, r=0, max_tokens=16, router_w, router_bias=None,
-                 gate=None, up, down, renorm_topk=True, flags=0, act="silu"):
+                 gate=None, up, down, renorm_topk=True, flags=0, act="silu", idx12=False):
         self.H, self.I, self.E, self.k, self.S, self.K, self.r = H, I, E, k, S, K, r
         self.max_tokens = max_tokens
         self._keep = [router_w, router_bias, gate, up, down]
@@ -175,7 +176,8 @@ class MoeVqlrLayer:
         cfg.renorm_topk = 1 if renorm_topk else 0
         if act not in ("silu", "gelu_tanh", "relu2"):
             raise ValueError(f"unknown expert activation {act!r}")
-        cfg.flags = flags | {"silu": 0, "gelu_tanh": FLAG_ACT_GELU_TANH, "relu2": FLAG_ACT_RELU2_UP_ONLY}[act]
+        cfg.flags = flags | {"silu": 0, "gelu_tanh": FLAG_ACT_GELU_TANH, "relu2": FLAG_ACT_RELU2_UP_ONLY}[act] \
+            | (FLAG_IDX12 if idx12 else 0)
         cfg.router_w = router_w.data_ptr()
         cfg.router_bias = None if router_bias is None else router_bias.data_ptr()
         for name, p in (("gate", gate), ("up", up), ("down", down)):
@@ -217,7 +219,8 @@ class MoeVqlrLayer:
         return cls(H=s.H, I=s.I, E=s.E, k=s.k, S=s.S, d=s.d, K=s.K, r=s.r,
                    max_tokens=max_tokens or max(s.T, 1), router_w=up(layer.router_w),
                    router_bias=up(layer.router_bias), gate=proj(layer.gate), up=proj(layer.up),
-                   down=proj(layer.down), renorm_topk=renorm_topk, flags=flags, act=s.act)
+                   down=proj(layer.down), renorm_topk=renorm_topk,
+                   flags=flags | (FLAG_IDX12 if getattr(s, "idx12", False) else 0), act=s.act)
 
     # -----------------------------------------------------------------------------------
     def _check(self, rc):

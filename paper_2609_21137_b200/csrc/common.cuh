@@ -34,6 +34,7 @@ struct Params {
   int act;                 // expert activation: 0 = SiLU, 1 = GELU (tanh form), 2 = up-only experts, p = relu(u)^2
                            // (the gate projection then aliases up: kernels that know skip its work, the rest repeat it)
   int d;                   // VQ block length: 8 (one code word = 16 bytes) or 4 (8 bytes)
+  int idx12;               // index maps hold 12-bit indices, two to three bytes (256 < K <= 4096); the uint16 kernels run
   int z_repeat;            // 1; ablation: every basis projection is computed this many times (once per selected expert)
   int n_zrows;             // rows of the stacked basis projection: (distinct gate/up bases) * r
   const bf16* router_w;
@@ -126,6 +127,27 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
+}
+
+// Twelve-bit packed index maps (the index width between one and two bytes: the deployed width
+// changes only at an encoding boundary of K).  Indices 2q and 2q+1 of a map occupy bytes 3q..3q+2,
+// little end first, i.e. a run of eight indices is a 96-bit little-endian number of 12-bit fields.
+// Element `elem` (even) of a map that the kernels otherwise address as IdxT:
+template <typename IdxT>
+__device__ __forceinline__ const IdxT* idx_at(const IdxT* base, size_t elem, int idx12) {
+  return idx12 ? reinterpret_cast<const IdxT*>(reinterpret_cast<const unsigned char*>(base) + (elem >> 1) * 3) : base + elem;
+}
+__device__ __forceinline__ void unpack_idx12x8(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t (&id)[8]) {
+  id[0] = w0 & 0xfffu;          id[1] = (w0 >> 12) & 0xfffu;
+  id[2] = (w0 >> 24) | ((w1 & 0xfu) << 8);
+  id[3] = (w1 >> 4) & 0xfffu;   id[4] = (w1 >> 16) & 0xfffu;
+  id[5] = (w1 >> 28) | ((w2 & 0xffu) << 4);
+  id[6] = (w2 >> 8) & 0xfffu;   id[7] = w2 >> 20;
+}
+// One index of a packed map (element `elem` counted from `base`).
+__device__ __forceinline__ uint32_t read_idx12(const void* base, size_t elem) {
+  const unsigned char* b = static_cast<const unsigned char*>(base) + (elem >> 1) * 3;
+  return (elem & 1) ? ((uint32_t)b[1] >> 4) | ((uint32_t)b[2] << 4) : (uint32_t)b[0] | (((uint32_t)b[1] & 0xfu) << 8);
 }
 
 // Position of 16-byte block b of an activation row in shared memory.  Lane l of a warp walks

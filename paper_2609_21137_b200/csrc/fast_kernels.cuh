@@ -148,9 +148,31 @@ __device__ __forceinline__ void cp_async_wait_pending(int pending) {
     default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
   }
 }
+__device__ __forceinline__ void cp_async4(void* smem, const void* gptr) {
+  const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sa), "l"(gptr) : "memory");
+}
+// Eight indices of a row into a 16-byte ring slot: 16 bytes of uint16, 8 of uint8, or (idx12) the
+// 12 bytes of eight packed twelve-bit indices, which start on a 4-byte boundary only.
 template <typename IdxT>
-__device__ __forceinline__ void cp_async_idx8(uint4* smem, const IdxT* gptr) {
-  if (sizeof(IdxT) == 2) cp_async16(smem, gptr); else cp_async8(smem, gptr);
+__device__ __forceinline__ void cp_async_idx8(uint4* smem, const IdxT* gptr, int idx12 = 0) {
+  if (sizeof(IdxT) == 2) {
+    if (idx12) {
+      const char* g = reinterpret_cast<const char*>(gptr);
+      char* d = reinterpret_cast<char*>(smem);
+      cp_async4(d, g); cp_async4(d + 4, g + 4); cp_async4(d + 8, g + 8);
+    } else {
+      cp_async16(smem, gptr);
+    }
+  } else {
+    cp_async8(smem, gptr);
+  }
+}
+// The eight indices of a ring slot.
+template <typename IdxT>
+__device__ __forceinline__ void slot_idx8(const uint4& raw, int idx12, uint32_t (&id)[8]) {
+  if (sizeof(IdxT) == 2 && idx12) unpack_idx12x8(raw.x, raw.y, raw.z, id);
+  else unpack_idx8<IdxT>(raw, id);
 }
 template <typename IdxT>
 __device__ __forceinline__ uint4 ring_idx8(const uint4* smem) {
@@ -1023,8 +1045,8 @@ __device__ __forceinline__ void gu_issue(const Params& P, const StagePlan& pl, c
     if (w.pf.part < pl.n_slices) {
       const int b = w.pf.part * 32 + 8 * c;
       if (b < nb) {
-        if (!up_only) cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_g + row * nb + b);
-        cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 1) * 32, idx_u + row * nb + b);
+        if (!up_only) cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_at(idx_g, row * nb + b, P.idx12), P.idx12);
+        cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 1) * 32, idx_at(idx_u, row * nb + b, P.idx12), P.idx12);
       }
     } else {
       const int rho = (w.pf.part - pl.n_slices) * 32 + 8 * c;
@@ -1147,8 +1169,8 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
           raw_u = ring_idx8<IdxT>(ring + (slot * 2 + 1) * 32);
         }
         uint32_t ig[8], iu[8];
-        unpack_idx8<IdxT>(raw_g, ig);
-        unpack_idx8<IdxT>(raw_u, iu);
+        slot_idx8<IdxT>(raw_g, P.idx12, ig);
+        slot_idx8<IdxT>(raw_u, P.idx12, iu);
         if (up_only) {                 // one projection: half the code-word reads and mma's
           if (D4) {
 #pragma unroll
@@ -1524,7 +1546,7 @@ __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, c
     for (int sub = 0; sub < TPU; ++sub) {
       const size_t rs = row + 8 * sub;
       uint4* slot = ring + (size_t)(w.pf_slot * TPU + sub) * 2 * 32;
-      if (b < nb) cp_async_idx8<IdxT>(slot, idx_d + rs * nb + b);
+      if (b < nb) cp_async_idx8<IdxT>(slot, idx_at(idx_d, rs * nb + b, P.idx12), P.idx12);
       if (pf.part < pl.n_lr && rho < P.r) cp_async16(slot + 32, P.down.factor + rs * P.r + rho);
     }
   }
@@ -1611,7 +1633,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
       uint4 raw = {0, 0, 0, 0};
       if (b0 < nb) raw = ring_idx8<IdxT>(uslot);
       uint32_t id[8];
-      unpack_idx8<IdxT>(raw, id);
+      slot_idx8<IdxT>(raw, P.idx12, id);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const uint4 w = D4 ? lookup_d4(s_cb, id[j], lane) : s_cb[pl.repl ? ((id[j] << 3) | (lane & 7)) : id[j]];

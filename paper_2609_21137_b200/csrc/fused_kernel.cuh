@@ -67,7 +67,7 @@ __host__ __device__ inline FusedLayout fused_layout(int K, int n_books, int T, i
 // (0 beyond the slice).
 template <typename IdxT>
 __global__ void k_relay_down_idx(const IdxT* __restrict__ src, IdxT* __restrict__ dst, int n_exp, int H, int nbI,
-                                 int tps, int n_sl, int jd) {
+                                 int tps, int n_sl, int jd, int idx12) {
   const size_t total = (size_t)n_exp * n_sl * (H / 8) * 32 * jd;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const int j = (int)(i % jd);
@@ -79,7 +79,8 @@ __global__ void k_relay_down_idx(const IdxT* __restrict__ src, IdxT* __restrict_
     const int si = (int)(q % n_sl);
     const int e = (int)(q / n_sl);
     const int g = lane >> 2, c = lane & 3, b = 4 * j + c, blk = si * tps + b;
-    dst[i] = (b < tps && blk < nbI) ? src[((size_t)e * H + tile * 8 + g) * nbI + blk] : (IdxT)0;
+    const size_t at = ((size_t)e * H + tile * 8 + g) * nbI + blk;
+    dst[i] = (b < tps && blk < nbI) ? (idx12 ? (IdxT)read_idx12(src, at) : src[at]) : (IdxT)0;
   }
 }
 
@@ -176,8 +177,8 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     if (part < pg.n_slices) {
       const int b = part * 32 + 8 * c;
       if (b < nb && requests_on) {
-        if (!up_only) cp_async_idx8<IdxT>(slot, idx_g + row * nb + b);
-        cp_async_idx8<IdxT>(slot + 32, idx_u + row * nb + b);
+        if (!up_only) cp_async_idx8<IdxT>(slot, idx_at(idx_g, row * nb + b, P.idx12), P.idx12);
+        cp_async_idx8<IdxT>(slot + 32, idx_at(idx_u, row * nb + b, P.idx12), P.idx12);
       }
     } else {
       const int rho = (part - pg.n_slices) * 32 + 8 * c;
@@ -291,8 +292,8 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
           uint4 raw_g = {0, 0, 0, 0}, raw_u = {0, 0, 0, 0};
           if (b0 < nb) { if (!up_only) raw_g = ring_idx8<IdxT>(slot); raw_u = ring_idx8<IdxT>(slot + 32); }
           uint32_t ig[8], iu[8];
-          unpack_idx8<IdxT>(raw_g, ig);
-          unpack_idx8<IdxT>(raw_u, iu);
+          slot_idx8<IdxT>(raw_g, P.idx12, ig);
+          slot_idx8<IdxT>(raw_u, P.idx12, iu);
           if (D4) {                   // four-value code words: two 8-byte reads per block
 #pragma unroll
             for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], lookup_d4(m.cb_u, iu[j], lane));

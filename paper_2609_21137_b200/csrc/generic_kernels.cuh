@@ -204,9 +204,15 @@ __device__ __forceinline__ void load_idx8<uint8_t>(const uint8_t* p, uint32_t (&
 
 // The eight weights of 8-value block b of a row: one code word (d = 8) or two consecutive
 // 4-value code words (d = 4, Section 5.5's shorter vectors: the row then has two indices per block).
+// Eight indices of a packed twelve-bit row starting at element 8 c (a 4-byte boundary).
+__device__ __forceinline__ void load_idx12x8(const void* row, int c, uint32_t (&id)[8]) {
+  const uint32_t* w = reinterpret_cast<const uint32_t*>(static_cast<const unsigned char*>(row) + (size_t)c * 12);
+  unpack_idx12x8(__ldg(w), __ldg(w + 1), __ldg(w + 2), id);
+}
+
 template <typename IdxT>
-__device__ __forceinline__ uint4 row_block8(const IdxT* __restrict__ idx_row, int b, const uint4* __restrict__ s_cb, int d) {
-  if (d == 8) return s_cb[idx_row[b]];
+__device__ __forceinline__ uint4 row_block8(const IdxT* __restrict__ idx_row, int b, const uint4* __restrict__ s_cb, int d, int idx12 = 0) {
+  if (d == 8) return s_cb[idx12 ? read_idx12(idx_row, b) : idx_row[b]];
   const uint2* cb2 = reinterpret_cast<const uint2*>(s_cb);
   const uint2 lo = cb2[idx_row[2 * b]], hi = cb2[idx_row[2 * b + 1]];
   return make_uint4(lo.x, lo.y, hi.x, hi.y);
@@ -230,11 +236,11 @@ __device__ __forceinline__ void vq_row_bf16x(const IdxT* __restrict__ idx_row, i
                                              const uint4* __restrict__ s_cb,
                                              const uint4* __restrict__ s_x, int x_stride,
                                              const int (&tok)[kTokGroup], int nt,
-                                             float (&acc)[kTokGroup], int lane) {
+                                             float (&acc)[kTokGroup], int lane, int idx12 = 0) {
   if (d == 8 && (nb & 7) == 0) {
     for (int c = lane; c < (nb >> 3); c += 32) {
       uint32_t id[8];
-      load_idx8<IdxT>(idx_row + c * 8, id);
+      if (idx12) load_idx12x8(idx_row, c, id); else load_idx8<IdxT>(idx_row + c * 8, id);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         float wf[8];
@@ -252,7 +258,7 @@ __device__ __forceinline__ void vq_row_bf16x(const IdxT* __restrict__ idx_row, i
   } else {   // rows whose index run is not a multiple of eight blocks: one index at a time
     for (int b0 = lane; b0 < nb; b0 += 32) {
       float wf[8];
-      unpack8(row_block8<IdxT>(idx_row, b0, s_cb, d), wf);
+      unpack8(row_block8<IdxT>(idx_row, b0, s_cb, d, idx12), wf);
       const int b = swz(b0);
 #pragma unroll
       for (int tt = 0; tt < kTokGroup; ++tt)
@@ -339,16 +345,16 @@ k_gateup(const Params P, const bf16* __restrict__ x, int T, int two_books) {
       for (int tt = 0; tt < kTokGroup; ++tt) tok[tt] = tt < nt ? P.pair_token[off + q0 + tt] : 0;
       float g[kTokGroup] = {0.f, 0.f, 0.f, 0.f}, u[kTokGroup] = {0.f, 0.f, 0.f, 0.f};
       if (P.gate.kind == MOE_VQLR_PROJ_VQLR) {
-        vq_row_bf16x<IdxT>(static_cast<const IdxT*>(P.gate.idx) + row * (P.H / P.d), nbH, P.d, s_cb_g, s_x, xs,
-                           tok, nt, g, lane);
+        vq_row_bf16x<IdxT>(idx_at(static_cast<const IdxT*>(P.gate.idx), row * (P.H / P.d), P.idx12), nbH, P.d, s_cb_g, s_x, xs,
+                           tok, nt, g, lane, P.idx12);
         if (P.gate.zslot >= 0)
           lr_row(P.gate.factor + row * P.r, P.r, P.z + P.gate.zslot * P.r, 2 * P.r, tok, nt, g, lane);
       } else {
         dense_row_bf16x(P.gate.dense + row * P.H, nbH, s_x, xs, tok, nt, g, lane);
       }
       if (P.up.kind == MOE_VQLR_PROJ_VQLR) {
-        vq_row_bf16x<IdxT>(static_cast<const IdxT*>(P.up.idx) + row * (P.H / P.d), nbH, P.d, s_cb_u, s_x, xs,
-                           tok, nt, u, lane);
+        vq_row_bf16x<IdxT>(idx_at(static_cast<const IdxT*>(P.up.idx), row * (P.H / P.d), P.idx12), nbH, P.d, s_cb_u, s_x, xs,
+                           tok, nt, u, lane, P.idx12);
         if (P.up.zslot >= 0)
           lr_row(P.up.factor + row * P.r, P.r, P.z + P.up.zslot * P.r, 2 * P.r, tok, nt, u, lane);
       } else {
@@ -408,11 +414,11 @@ k_down(const Params P, bf16* __restrict__ out, int T) {
         const float* prow = P.p + (size_t)pos * P.I;
         float acc = 0.f;
         if (vq) {
-          const IdxT* idx_row = static_cast<const IdxT*>(P.down.idx) + row * (P.I / P.d);
+          const IdxT* idx_row = idx_at(static_cast<const IdxT*>(P.down.idx), row * (P.I / P.d), P.idx12);
           if (P.d == 8 && (nbI & 7) == 0) {
             for (int c = lane; c < (nbI >> 3); c += 32) {
               uint32_t id[8];
-              load_idx8<IdxT>(idx_row + c * 8, id);
+              if (P.idx12) load_idx12x8(idx_row, c, id); else load_idx8<IdxT>(idx_row + c * 8, id);
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 float wf[8];
@@ -426,7 +432,7 @@ k_down(const Params P, bf16* __restrict__ out, int T) {
           } else {
             for (int b = lane; b < nbI; b += 32) {
               float wf[8];
-              unpack8(row_block8<IdxT>(idx_row, b, s_cb, P.d), wf);
+              unpack8(row_block8<IdxT>(idx_row, b, s_cb, P.d, P.idx12), wf);
               const float4 p0 = *reinterpret_cast<const float4*>(prow + b * 8);
               const float4 p1 = *reinterpret_cast<const float4*>(prow + b * 8 + 4);
               const float pf[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
@@ -465,11 +471,11 @@ k_down(const Params P, bf16* __restrict__ out, int T) {
 
 // Largest index of an index map (create-time validation only).
 template <typename IdxT>
-__global__ void k_max_index(const IdxT* __restrict__ idx, size_t n, unsigned int* out) {
+__global__ void k_max_index(const IdxT* __restrict__ idx, size_t n, unsigned int* out, int idx12) {
   unsigned int m = 0;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
        i += (size_t)gridDim.x * blockDim.x)
-    m = max(m, (unsigned int)idx[i]);
+    m = max(m, idx12 ? read_idx12(idx, i) : (unsigned int)idx[i]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
   if ((threadIdx.x & 31) == 0) atomicMax(out, m);

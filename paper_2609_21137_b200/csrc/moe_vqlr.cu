@@ -470,6 +470,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
   const bool any_vq = cfg->gate.kind == MOE_VQLR_PROJ_VQLR || cfg->up.kind == MOE_VQLR_PROJ_VQLR ||
                       cfg->down.kind == MOE_VQLR_PROJ_VQLR;
   if (any_vq && (K <= 0 || K > 65536)) return fail(nullptr, MOE_VQLR_ERR_UNSUPPORTED, "codebook_size out of 1..65536");
+  if ((cfg->flags & MOE_VQLR_FLAG_IDX12) && any_vq && (K <= 256 || K > 4096 || cfg->vq_dim != kD || H % 16 || I % 16))
+    return fail(nullptr, MOE_VQLR_ERR_UNSUPPORTED, "12-bit indices need 256 < codebook_size <= 4096, vq_dim 8, hidden and inter multiples of 16");
   int rc;
   if ((rc = check_proj(cfg->gate, "gate", r)) || (rc = check_proj(cfg->up, "up", r)) ||
       (rc = check_proj(cfg->down, "down", r)))
@@ -504,6 +506,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
   P.renorm = cfg->renorm_topk ? 1 : 0;
   P.act = (cfg->flags & MOE_VQLR_FLAG_ACT_RELU2_UP_ONLY) ? 2 : (cfg->flags & MOE_VQLR_FLAG_ACT_GELU_TANH) ? 1 : 0;
   P.d = cfg->vq_dim;
+  P.idx12 = (any_vq && (cfg->flags & MOE_VQLR_FLAG_IDX12)) ? 1 : 0;
   P.z_repeat = (cfg->flags & MOE_VQLR_FLAG_ABLATE_Z_PER_EXPERT) ? cfg->top_k + cfg->n_shared : 1;
   h->per_expert_launch = (cfg->flags & MOE_VQLR_FLAG_ABLATE_PER_EXPERT_LAUNCH) != 0;
   P.router_w = static_cast<const bf16*>(cfg->router_w);
@@ -658,7 +661,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
     int coop_attr = 0;
     cudaDeviceGetAttribute(&coop_attr, cudaDevAttrCooperativeLaunch, h->device);
     const bool want_coop = (cfg->flags & MOE_VQLR_FLAG_PERSISTENT) != 0;
-    if (h->fast && !h->d4 && !h->lrf && !h->gu_dense && coop_attr && want_coop) {
+    if (h->fast && !h->d4 && !h->lrf && !h->gu_dense && !P.idx12 && coop_attr && want_coop) {
       const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
       const int warps = kCoopThreads / 32;
       h->plan_gu_coop = h->plan_gu;
@@ -870,9 +873,9 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
   if (h->fused && !h->dn_dense) {      // one-off: the down index map per slice
     const FusedPlan& fp = h->fplan;
     if (h->idx_tc == 1)
-      k_relay_down_idx<uint8_t><<<h->sm_count * 8, 256>>>(static_cast<const uint8_t*>(P.down.idx), static_cast<uint8_t*>(h->idx_dp), E + S, H, I / kD, fp.tps, fp.n_sl, fp.jd);
+      k_relay_down_idx<uint8_t><<<h->sm_count * 8, 256>>>(static_cast<const uint8_t*>(P.down.idx), static_cast<uint8_t*>(h->idx_dp), E + S, H, I / kD, fp.tps, fp.n_sl, fp.jd, 0);
     else
-      k_relay_down_idx<uint16_t><<<h->sm_count * 8, 256>>>(static_cast<const uint16_t*>(P.down.idx), static_cast<uint16_t*>(h->idx_dp), E + S, H, I / kD, fp.tps, fp.n_sl, fp.jd);
+      k_relay_down_idx<uint16_t><<<h->sm_count * 8, 256>>>(static_cast<const uint16_t*>(P.down.idx), static_cast<uint16_t*>(h->idx_dp), E + S, H, I / kD, fp.tps, fp.n_sl, fp.jd, P.idx12);
     ce = cudaDeviceSynchronize();
     if (ce != cudaSuccess) {
       rc = fail(nullptr, MOE_VQLR_ERR_CUDA, "re-laying the down index map: %s", cudaGetErrorString(ce));
@@ -889,8 +892,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
     for (int i = 0; i < 3; ++i) {
       if (projs[i]->kind != MOE_VQLR_PROJ_VQLR) continue;
       const size_t n = (size_t)(E + S) * H * I / cfg->vq_dim;
-      if (h->idx_bytes == 1) k_max_index<uint8_t><<<h->sm_count * 4, 256>>>(static_cast<const uint8_t*>(projs[i]->idx), n, d_max);
-      else k_max_index<uint16_t><<<h->sm_count * 4, 256>>>(static_cast<const uint16_t*>(projs[i]->idx), n, d_max);
+      if (h->idx_bytes == 1) k_max_index<uint8_t><<<h->sm_count * 4, 256>>>(static_cast<const uint8_t*>(projs[i]->idx), n, d_max, 0);
+      else k_max_index<uint16_t><<<h->sm_count * 4, 256>>>(static_cast<const uint16_t*>(projs[i]->idx), n, d_max, P.idx12);
     }
     unsigned int mx = 0;
     ce = cudaMemcpy(&mx, d_max, sizeof mx, cudaMemcpyDeviceToHost);

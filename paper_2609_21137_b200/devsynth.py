@@ -24,6 +24,15 @@ def _indices(gen, size, K, device):
     return torch.where(v >= 32768, v - 65536, v).to(torch.int16)
 
 
+def _pack12(idx16: torch.Tensor) -> torch.Tensor:
+    """Twelve-bit packing (two indices to three bytes, little end first) of an int16 index tensor
+    whose last dimension is even; same byte layout as ``synth.pack12``."""
+    v = idx16.to(torch.int32) & 0xFFFF
+    lo, hi = v[..., 0::2], v[..., 1::2]
+    out = torch.stack([lo & 0xFF, (lo >> 8) | ((hi & 0xF) << 4), hi >> 4], dim=-1).to(torch.uint8)
+    return out.reshape(*idx16.shape[:-1], idx16.shape[-1] // 2 * 3).contiguous()
+
+
 def make_device_layer(shp: LayerShape, seed: int, device="cuda") -> dict:
     """Returns keyword arguments for ``binding.MoeVqlrLayer`` plus ``x`` ([T][H] bf16)."""
     gen = torch.Generator(device=device)
@@ -47,12 +56,14 @@ def make_device_layer(shp: LayerShape, seed: int, device="cuda") -> dict:
                     shared_book = book
             else:
                 book = shared_book
+            idx = _indices(gen, (n_exp, out_dim, in_dim // d), K, device)
             projs[p] = dict(codebook=book,
-                            idx=_indices(gen, (n_exp, out_dim, in_dim // d), K, device),
+                            idx=_pack12(idx) if shp.idx12 else idx,
                             basis=_normal_bf16(gen, (r, in_dim), in_dim ** -0.5, device) if r > 0 else None,
                             factor=_normal_bf16(gen, (n_exp, out_dim, r), 0.01, device) if r > 0 else None)
         else:
             projs[p] = dict(dense=_normal_bf16(gen, (n_exp, out_dim, in_dim), 0.02, device))
     return dict(H=H, I=I, E=E, k=shp.k, S=S, d=d, K=K if any(vq.values()) else 0, r=r,
                 max_tokens=max(T, 1), router_w=router_w, router_bias=bias, gate=projs.get("gate"),
-                up=projs["up"], down=projs["down"], act=shp.act, x=x)
+                up=projs["up"], down=projs["down"], act=shp.act, x=x,
+                **({"idx12": True} if shp.idx12 else {}))

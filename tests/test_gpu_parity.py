@@ -196,3 +196,45 @@ def test_nemotron_shaped_layer_and_a_padded_hidden_size():
     assert_routing(dbg, res)
     assert_output(bf16_tensor_to_f64(out), res.out, what="padded hidden size")
     mod.close()
+
+
+@pytest.mark.parametrize("path", ["default", "generic", "fused", "chain"])
+@pytest.mark.parametrize("shp", [synth.shape("tiny", T=1, K=700, I=128, idx12=True),
+                                 synth.shape("tiny", T=5, K=4096, mode="paper", idx12=True),
+                                 synth.shape("qwen3", E=16, T=1, idx12=True),
+                                 synth.shape("qwen3", E=16, T=9, idx12=True, act="relu2")],
+                         ids=lambda s: f"{s.name}-{s.mode}-T{s.T}-K{s.K}")
+def test_twelve_bit_packed_indices(shp, path):
+    """MOE_VQLR_FLAG_IDX12: the index maps of all compressed projections packed to twelve bits.  The
+    oracle reads the same packed bytes (and is pinned to give the uint16 layer's result bit for bit)."""
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    assert layer.up.idx.dtype == np.uint8 and layer.up.idx.shape[-1] == (shp.H // 8) * 3 // 2
+    flags = {"default": 0, "generic": binding.FLAG_GENERIC_KERNELS, "fused": binding.FLAG_FORCE_FUSED,
+             "chain": binding.FLAG_NO_FUSED}[path]
+    mod, (out, dbg) = run_gpu(layer, flags=flags)
+    assert_routing(dbg, res)
+    assert_output(bf16_tensor_to_f64(out), res.out, what=f"{shp.name} idx12 {path}")
+    mod.close()
+
+
+def test_twelve_bit_indices_limits_and_validation():
+    from paper_2609_21137_b200 import binding
+    # K = 256 has one-byte indices: the packed encoding is refused
+    layer = synth.make_layer(synth.shape("tiny", K=700, I=128, idx12=True), 0)
+    with pytest.raises(binding.MoeVqlrError) as err:
+        binding.MoeVqlrLayer.from_synth(synth.Layer(shape=synth.shape("tiny", K=256, I=128, idx12=True), router_w=layer.router_w,
+                                                    router_bias=None, x=layer.x, gate=layer.gate, up=layer.up, down=layer.down))
+    assert err.value.status == binding.ERR_UNSUPPORTED
+    # index validation unpacks the twelve-bit fields: 701 >= K = 700 is found
+    packed = layer.up.idx
+    bad = packed.copy()
+    i0 = (700 + 1) & 0xFFF
+    bad[1, 2, 0] = i0 & 0xFF
+    bad[1, 2, 1] = (bad[1, 2, 1] & 0xF0) | (i0 >> 8)
+    layer.up.idx = bad
+    with pytest.raises(binding.MoeVqlrError) as err:
+        binding.MoeVqlrLayer.from_synth(layer, flags=binding.FLAG_VALIDATE_INDICES)
+    assert err.value.status == binding.ERR_BAD_INDEX
+    layer.up.idx = packed
+    binding.MoeVqlrLayer.from_synth(layer, flags=binding.FLAG_VALIDATE_INDICES).close()
