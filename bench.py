@@ -69,6 +69,8 @@ def parse_args():
                     help="switch a mechanism off (Section 5.4): z = shared projections recomputed per expert, "
                          "launch = one gate/up and one down launch per work group")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flags", type=int, default=0,
+                    help="extra MOE_VQLR_FLAG_* bits for the handles of the main workload (A/B runs of the kernel paths)")
     return ap.parse_args()
 
 
@@ -454,7 +456,7 @@ def main():
     from paper_2609_21137_b200 import binding as _b
     ablate_flags = {"": 0, "z": _b.FLAG_ABLATE_Z_PER_EXPERT, "launch": _b.FLAG_ABLATE_PER_EXPERT_LAUNCH,
                     "both": _b.FLAG_ABLATE_Z_PER_EXPERT | _b.FLAG_ABLATE_PER_EXPERT_LAUNCH}[args.ablate]
-    wl = Workload(args.workload, args.mode, args.layers, device, flags=ablate_flags)
+    wl = Workload(args.workload, args.mode, args.layers, device, flags=ablate_flags | args.flags)
 
     # ---- the timed regions: W warm-up steps, then R regions of exactly K steps each -----------
     # A region of few steps lasts well under a millisecond and one sample of it is noisy, so the
@@ -558,7 +560,8 @@ def main():
                 "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
                 "data": "synthetic",
                 "config": {"workload": f"{args.workload} T={shp.T} mode={args.mode}"
-                                       + (f" ablate={args.ablate}" if args.ablate else ""),
+                                       + (f" ablate={args.ablate}" if args.ablate else "")
+                                       + (f" flags={args.flags}" if args.flags else ""),
                            "shape": f"H={shp.H} I={shp.I} E={shp.E} k={shp.k} S={shp.S} K={shp.K} r={shp.r}",
                            "distinct_layers": n_layers,
                            "l2": f"rotation over {n_layers} distinct layers touches "

@@ -121,7 +121,8 @@ enum {
   MOE_VQLR_FLAG_GENERIC_KERNELS = 256u,  /* only the generic CUDA-core kernels (one warp per output
                                          row), which otherwise serve the shapes the tensor-core
                                          kernels do not cover */
-  MOE_VQLR_FLAG_PROJECTION_CODE_BOOK = 512u, /* calls with two or more tokens evaluate the VQ term of
+  MOE_VQLR_FLAG_PROJECTION_CODE_BOOK = 512u, /* calls that run the chain of kernels (all of them with
+                                         MOE_VQLR_FLAG_NO_FUSED) evaluate the VQ term of
                                          gate / up through per-token projection code books
                                          T[b][k] = <x_b, codebook[k]> (Section 4.2; needs K <= 256 and
                                          vq_dim 8; measured slower than the reconstructing tensor-core

@@ -633,7 +633,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
   h->pcb_Q = 0;
   h->smem_lr = 0;
   {
-    const bool want_pcb = (cfg->flags & MOE_VQLR_FLAG_PROJECTION_CODE_BOOK) != 0;   // from two tokens on; off by default (measured slower than the tensor-core kernel)
+    const bool want_pcb = (cfg->flags & MOE_VQLR_FLAG_PROJECTION_CODE_BOOK) != 0;   // off by default (measured slower than the tensor-core kernels at every batch size)
     const bool gu_vq2 = P.gate.kind == MOE_VQLR_PROJ_VQLR && P.up.kind == MOE_VQLR_PROJ_VQLR;
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
     if (h->fast && gu_vq2 && !h->d4 && cfg->vq_dim == kD && h->idx_bytes == 1 && H % 16 == 0 && I % kPcbRows == 0 &&
@@ -646,7 +646,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
           raise_dyn_smem((const void*)k_gateup_pcb, (size_t)pcb_smem_bytes(K)) == cudaSuccess) {
         h->pcb = true;
         h->pcb_Q = (H / 8 + kPcbPiece - 1) / kPcbPiece;
-        h->pcb_min_T = 2;
+        h->pcb_min_T = 1;
       } else {
         cudaGetLastError();
       }

@@ -83,7 +83,14 @@ SHAPES: Dict[str, LayerShape] = {
                              mode="paper", per_projection_codebook=True),
     "qwen3_5bit": LayerShape("qwen3_5bit", H=2048, I=768, E=128, k=8, d=8, K=256, r=504, T=1,
                              mode="paper", per_projection_codebook=True),
-    # the (4, 256, 256) point on the OLMoE shape: four-value code words (generic kernels)
+    # ... and its d = 4 points: the index term alone is 2 bits per weight, r = 128 / 248 / 376
+    "qwen3_d4_3bit": LayerShape("qwen3_d4_3bit", H=2048, I=768, E=128, k=8, d=4, K=256, r=128, T=1,
+                                mode="paper", per_projection_codebook=True),
+    "qwen3_d4_4bit": LayerShape("qwen3_d4_4bit", H=2048, I=768, E=128, k=8, d=4, K=256, r=248, T=1,
+                                mode="paper", per_projection_codebook=True),
+    "qwen3_d4_5bit": LayerShape("qwen3_d4_5bit", H=2048, I=768, E=128, k=8, d=4, K=256, r=376, T=1,
+                                mode="paper", per_projection_codebook=True),
+    # the (4, 256, 256) point on the OLMoE shape: four-value code words
     # Nemotron-3-Nano-shaped layer at its deployed point (8, 256, 512): up-only ReLU^2 experts, bf16 down projection
     "nemotron_deployed": LayerShape("nemotron_deployed", H=2688, I=1856, E=128, k=6, d=8, K=256, r=512, T=1,
                                     mode="paper", per_projection_codebook=True, act="relu2"),

@@ -68,7 +68,7 @@ def test_more_slices_than_warps_b16():
 
 
 @pytest.mark.parametrize("name", ["qwen3_deployed", "qwen3_deployed_b16", "gemma4_deployed", "qwen3_3bit",
-                                  "qwen3_5bit"])
+                                  "qwen3_5bit", "qwen3_d4_3bit", "qwen3_d4_4bit", "qwen3_d4_5bit"])
 def test_papers_deployed_operating_points(name):
     # K = 256 / uint8, r = 384 (twelve low-rank parts), separate gate and up code books, bf16 down;
     # fewer experts than the real models to keep the oracle quick (routing width is unchanged)

@@ -240,6 +240,7 @@ def test_ablation_switches_keep_results(shp):
 
 @pytest.mark.parametrize("shp", [synth.shape("tiny", T=5), synth.shape("tiny", T=2, mode="paper", K=100),
                                  synth.shape("dsv2lite", E=16, T=8), synth.shape("qwen3_deployed", E=24, T=16),
+                                 synth.shape("dsv2lite", E=16, T=1), synth.shape("qwen3_deployed", E=24, T=1),
                                  synth.LayerShape("ragged_piece", H=8 * 48, I=128, E=6, k=2, S=1, d=8, K=256, r=40, T=3),
                                  synth.LayerShape("r0_books", H=1024, I=64, E=8, k=3, d=8, K=64, r=0, T=4,
                                                   per_projection_codebook=True)],

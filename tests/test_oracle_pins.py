@@ -216,9 +216,10 @@ def test_single_expert_is_plain_swiglu_mlp(d):
 
 
 def test_storage_rate_sweep_shapes_hit_their_rates():
-    # Section 5.5: K = 256, d = 8, r chosen for about 3, 4 and 5 bits per original weight
+    # Section 5.5: K = 256, d in {8, 4}, r chosen for about 3, 4 and 5 bits per original weight
     # (here r is a multiple of 8, which moves the 3-bit point 0.022 off its target)
-    for name, target in (("qwen3_3bit", 3.0), ("qwen3_4bit", 4.0), ("qwen3_5bit", 5.0)):
+    for name, target in (("qwen3_3bit", 3.0), ("qwen3_4bit", 4.0), ("qwen3_5bit", 5.0),
+                         ("qwen3_d4_3bit", 3.0), ("qwen3_d4_4bit", 4.0), ("qwen3_d4_5bit", 5.0)):
         s = synth.shape(name)
         bits = oracle.storage_bits_per_weight(s.d, s.K, s.r, s.H, s.I, s.E)
         closed = 8 / s.d + 16 * s.r / s.H + 16 * s.r / (s.E * s.I) + 16 * s.K * s.d / (s.E * s.H * s.I)
