@@ -1033,7 +1033,10 @@ struct Walk {
 };
 
 // Streams the bytes of the prefetch cursor's unit into the ring and advances that cursor.
-template <typename IdxT, bool DENSE>
+// SP ("special formats"): the kernel also handles experts without a gate projection and 12-bit
+// packed indices, at the price of run-time checks in its unit loop; the plain instantiation folds
+// them away.
+template <typename IdxT, bool DENSE, bool SP = false>
 __device__ __forceinline__ void gu_issue(const Params& P, const StagePlan& pl, const GuSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3, nb = pl.nb;
   uint4* ring = m.ring;
@@ -1041,12 +1044,13 @@ __device__ __forceinline__ void gu_issue(const Params& P, const StagePlan& pl, c
     const IdxT* idx_g = static_cast<const IdxT*>(P.gate.idx);
     const IdxT* idx_u = static_cast<const IdxT*>(P.up.idx);
     const size_t row = (size_t)m.R.grp_e[w.pf.grp] * P.I + w.pf.jt * 8 + g;
-    const bool up_only = P.act == 2;       // experts without a gate: its bytes are not requested
+    const bool up_only = SP && P.act == 2;       // experts without a gate: its bytes are not requested
+    const int idx12 = SP ? P.idx12 : 0;
     if (w.pf.part < pl.n_slices) {
       const int b = w.pf.part * 32 + 8 * c;
       if (b < nb) {
-        if (!up_only) cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_at(idx_g, row * nb + b, P.idx12), P.idx12);
-        cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 1) * 32, idx_at(idx_u, row * nb + b, P.idx12), P.idx12);
+        if (!up_only) cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 0) * 32, idx_at(idx_g, row * nb + b, idx12), idx12);
+        cp_async_idx8<IdxT>(ring + (w.pf_slot * 2 + 1) * 32, idx_at(idx_u, row * nb + b, idx12), idx12);
       }
     } else {
       const int rho = (w.pf.part - pl.n_slices) * 32 + 8 * c;
@@ -1062,7 +1066,7 @@ __device__ __forceinline__ void gu_issue(const Params& P, const StagePlan& pl, c
 
 // Start of the walk of warp `wid` out of `W` warps (needs the work groups): depth - 1 units are
 // requested, each as one cp.async group.
-template <typename IdxT, bool DENSE>
+template <typename IdxT, bool DENSE, bool SP = false>
 __device__ __forceinline__ void gu_tiles_begin(const Params& P, const StagePlan& pl, const GuSmem& m, int wid, int W, Walk& w) {
   const int per_grp = pl.n_parts * pl.tiles;
   int V = *m.R.n_grp * per_grp, v0 = 0;
@@ -1072,7 +1076,7 @@ __device__ __forceinline__ void gu_tiles_begin(const Params& P, const StagePlan&
   w.pf.set(w.n_my > 0 ? v0 + v_begin : 0, pl);
   w.cur = w.pf;
   w.pf_slot = 0; w.cur_slot = 0;
-  for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) gu_issue<IdxT, DENSE>(P, pl, m, w); cp_async_commit(); }
+  for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) gu_issue<IdxT, DENSE, SP>(P, pl, m, w); cp_async_commit(); }
   TRACE_STAMP(1, 7);
 }
 
@@ -1081,7 +1085,7 @@ __device__ __forceinline__ void gu_tiles_begin(const Params& P, const StagePlan&
 // ... besides its own blocks and no group is a part of its own (fewer, fatter units and fewer
 // partial tiles; with fewer groups than slices the units that carry one would lag the others).
 // LRF = 2: some slices carry two or more groups; the second one's bytes are requested early as well.
-template <typename IdxT, bool DENSE, bool D4 = false, int LRF = 0>
+template <typename IdxT, bool DENSE, bool D4 = false, int LRF = 0, bool SP = false>
 __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __restrict__ x, int T, const StagePlan& pl,
                                              const GuSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
@@ -1097,11 +1101,12 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
   const int n_pos = T * (P.k + P.S), n_my = w.n_my;
   Cursor& cur = w.cur;
   int& cur_slot = w.cur_slot;
-  auto issue = [&]() { gu_issue<IdxT, DENSE>(P, pl, m, w); };
+  auto issue = [&]() { gu_issue<IdxT, DENSE, SP>(P, pl, m, w); };
 
   uint4 fx[8];                       // activation fragments of the current (group, part)
   int frag_grp = -1, frag_part = -1;
-  const bool up_only = P.act == 2;   // experts without a gate projection: only the up products are formed
+  const bool up_only = SP && P.act == 2;   // experts without a gate projection: only the up products are formed
+  const int idx12 = SP ? P.idx12 : 0;
 
   for (int i = 0; i < n_my; ++i) {
     if (i + D - 1 < n_my) issue();
@@ -1169,8 +1174,8 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
           raw_u = ring_idx8<IdxT>(ring + (slot * 2 + 1) * 32);
         }
         uint32_t ig[8], iu[8];
-        slot_idx8<IdxT>(raw_g, P.idx12, ig);
-        slot_idx8<IdxT>(raw_u, P.idx12, iu);
+        slot_idx8<IdxT>(raw_g, idx12, ig);
+        slot_idx8<IdxT>(raw_u, idx12, iu);
         if (up_only) {                 // one projection: half the code-word reads and mma's
           if (D4) {
 #pragma unroll
@@ -1255,7 +1260,7 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
   TRACE_STAMP(0, 15);
 }
 
-template <typename IdxT, bool DENSE, bool D4 = false, int LRF = 0>
+template <typename IdxT, bool DENSE, bool D4 = false, int LRF = 0, bool SP = false>
 __global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
 k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {
   extern __shared__ uint4 s_u4[];
@@ -1269,11 +1274,11 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   TRACE_STAMP(0, 2);
   gu_route(P, T, pl, m, blockIdx.x == 0, want_dbg != 0);
   Walk w;
-  gu_tiles_begin<IdxT, DENSE>(P, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps, w);   // index bytes travel ...
+  gu_tiles_begin<IdxT, DENSE, SP>(P, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps, w);   // index bytes travel ...
   gu_finish_stage<DENSE>(P, pl, n_books, m, pl.depth - 1);                                     // ... while the stage settles
   pdl_launch();
   TRACE_STAMP(0, 3);
-  gu_tiles_run<IdxT, DENSE, D4, LRF>(P, x, T, pl, m, w);
+  gu_tiles_run<IdxT, DENSE, D4, LRF, SP>(P, x, T, pl, m, w);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1528,7 +1533,7 @@ struct DnSmem {
 };
 
 // Streams the bytes of the prefetch cursor's unit into the ring and advances that cursor.
-template <typename IdxT, bool DENSE, int TPU = 2>
+template <typename IdxT, bool DENSE, int TPU = 2, bool SP = false>
 __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, const DnSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3, nb = pl.nb;
   uint4* ring = m.ring;
@@ -1546,7 +1551,7 @@ __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, c
     for (int sub = 0; sub < TPU; ++sub) {
       const size_t rs = row + 8 * sub;
       uint4* slot = ring + (size_t)(w.pf_slot * TPU + sub) * 2 * 32;
-      if (b < nb) cp_async_idx8<IdxT>(slot, idx_at(idx_d, rs * nb + b, P.idx12), P.idx12);
+      if (b < nb) cp_async_idx8<IdxT>(slot, idx_at(idx_d, rs * nb + b, SP ? P.idx12 : 0), SP ? P.idx12 : 0);
       if (pf.part < pl.n_lr && rho < P.r) cp_async16(slot + 32, P.down.factor + rs * P.r + rho);
     }
   }
@@ -1555,7 +1560,7 @@ __device__ __forceinline__ void dn_issue(const Params& P, const StagePlan& pl, c
 }
 
 // Start of the walk of warp `wid` out of `W` warps (needs only the work groups, not p).
-template <typename IdxT, bool DENSE, int TPU = 2>
+template <typename IdxT, bool DENSE, int TPU = 2, bool SP = false>
 __device__ __forceinline__ void dn_tiles_begin(const Params& P, const StagePlan& pl, const DnSmem& m, int wid, int W, Walk& w) {
   const int per_grp = pl.n_parts * pl.tiles;
   int V = m.n_grp * per_grp, v0 = 0;
@@ -1565,12 +1570,12 @@ __device__ __forceinline__ void dn_tiles_begin(const Params& P, const StagePlan&
   w.pf.set(w.n_my > 0 ? v0 + v_begin : 0, pl);
   w.cur = w.pf;
   w.pf_slot = 0; w.cur_slot = 0;
-  for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) dn_issue<IdxT, DENSE, TPU>(P, pl, m, w); cp_async_commit(); }
+  for (int i = 0; i < pl.depth - 1; ++i) { if (i < w.n_my) dn_issue<IdxT, DENSE, TPU, SP>(P, pl, m, w); cp_async_commit(); }
   TRACE_STAMP(2, 3);
 }
 
 // The tile loop proper (needs p, z_d and the code book).
-template <typename IdxT, bool DENSE, bool D4 = false, int TPU = 2>
+template <typename IdxT, bool DENSE, bool D4 = false, int TPU = 2, bool SP = false>
 __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const StagePlan& pl, const DnSmem& m, Walk& w) {
   const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
   const int nb = pl.nb, D = pl.depth;
@@ -1581,7 +1586,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
   const int *s_grp_e = m.grp_e, *s_grp_off = m.grp_off, *s_grp_cnt = m.grp_cnt;
   Cursor& cur = w.cur;
   int& cur_slot = w.cur_slot;
-  auto issue = [&]() { dn_issue<IdxT, DENSE, TPU>(P, pl, m, w); };
+  auto issue = [&]() { dn_issue<IdxT, DENSE, TPU, SP>(P, pl, m, w); };
 
   uint4 fh[8], fl[8];
   uint4 zh = {0, 0, 0, 0}, zl = {0, 0, 0, 0};     // z_d fragments of the low-rank group this part carries
@@ -1633,7 +1638,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
       uint4 raw = {0, 0, 0, 0};
       if (b0 < nb) raw = ring_idx8<IdxT>(uslot);
       uint32_t id[8];
-      slot_idx8<IdxT>(raw, P.idx12, id);
+      slot_idx8<IdxT>(raw, SP ? P.idx12 : 0, id);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const uint4 w = D4 ? lookup_d4(s_cb, id[j], lane) : s_cb[pl.repl ? ((id[j] << 3) | (lane & 7)) : id[j]];
@@ -1670,7 +1675,7 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
   TRACE_STAMP(2, 15);
 }
 
-template <typename IdxT, bool DENSE, bool D4 = false, int TPU = 2>
+template <typename IdxT, bool DENSE, bool D4 = false, int TPU = 2, bool SP = false>
 __global__ void __launch_bounds__(kDownThreads, 1)
 k_down_mma(const Params P, int T, const StagePlan pl) {
   extern __shared__ uint4 s_u4[];
@@ -1704,7 +1709,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   m.cb = s_cb; m.ring = ring; m.slot_u4 = L.slot_u4;
   m.grp_e = s_grp_e; m.grp_off = s_grp_off; m.grp_cnt = s_grp_cnt; m.n_grp = n_grp;
   Walk w;
-  dn_tiles_begin<IdxT, DENSE, TPU>(P, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps, w);   // index bytes travel ...
+  dn_tiles_begin<IdxT, DENSE, TPU, SP>(P, pl, m, blockIdx.x * nwarps + warp, gridDim.x * nwarps, w);   // index bytes travel ...
   cp_async_wait_pending(D - 1);                                                                // ... the code book has landed
   __syncthreads();
   if (!DENSE && pl.repl) {
@@ -1718,7 +1723,7 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
     __syncthreads();
   }
   TRACE_STAMP(2, 2);
-  dn_tiles_run<IdxT, DENSE, D4, TPU>(P, T, pl, m, w);
+  dn_tiles_run<IdxT, DENSE, D4, TPU, SP>(P, T, pl, m, w);
 }
 
 // out[t][h] = sum over slots (in slot order) of affinity * y[t][slot][h], where y is the sum of

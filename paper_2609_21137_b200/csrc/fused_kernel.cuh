@@ -86,7 +86,9 @@ __global__ void k_relay_down_idx(const IdxT* __restrict__ src, IdxT* __restrict_
 
 // JD = k steps of the down product (a compile-time constant: the down loop is bound by
 // instruction issue, and with JD known its predicates and index unpacking fold away).
-template <typename IdxT, bool DN_DENSE, int JD, bool D4 = false>
+// SP: also experts without a gate projection and 12-bit packed indices (run-time checks in the unit
+// loop that the plain instantiation folds away).
+template <typename IdxT, bool DN_DENSE, int JD, bool D4 = false, bool SP = false>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePlan pg, const FusedPlan fp, int n_books,
                int want_dbg, const IdxT* __restrict__ idx_dp) {
@@ -165,7 +167,8 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     if (u.i == it.ns) { u.part = it.lp; u.tile = it.lt; }
     else if (++u.tile == it.tiles) { u.tile = 0; ++u.part; }
   };
-  const bool up_only = P.act == 2;     // experts without a gate: its bytes are not requested, its products not formed
+  const bool up_only = SP && P.act == 2;     // experts without a gate: its bytes are not requested, its products not formed
+  const int idx12 = SP ? P.idx12 : 0;
   int g_rq = 0, g_use = 0;             // gate/up ring: next slot to request into, next to consume
   bool requests_on = true;             // off: the request code runs (and warms the instruction cache) without asking for bytes
   auto gu_request = [&](const Item& it, UnitCur& rq) {                    // requests come in the order of use
@@ -177,8 +180,8 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
     if (part < pg.n_slices) {
       const int b = part * 32 + 8 * c;
       if (b < nb && requests_on) {
-        if (!up_only) cp_async_idx8<IdxT>(slot, idx_at(idx_g, row * nb + b, P.idx12), P.idx12);
-        cp_async_idx8<IdxT>(slot + 32, idx_at(idx_u, row * nb + b, P.idx12), P.idx12);
+        if (!up_only) cp_async_idx8<IdxT>(slot, idx_at(idx_g, row * nb + b, idx12), idx12);
+        cp_async_idx8<IdxT>(slot + 32, idx_at(idx_u, row * nb + b, idx12), idx12);
       }
     } else {
       const int rho = (part - pg.n_slices) * 32 + 8 * c;
@@ -292,8 +295,8 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
           uint4 raw_g = {0, 0, 0, 0}, raw_u = {0, 0, 0, 0};
           if (b0 < nb) { if (!up_only) raw_g = ring_idx8<IdxT>(slot); raw_u = ring_idx8<IdxT>(slot + 32); }
           uint32_t ig[8], iu[8];
-          slot_idx8<IdxT>(raw_g, P.idx12, ig);
-          slot_idx8<IdxT>(raw_u, P.idx12, iu);
+          slot_idx8<IdxT>(raw_g, idx12, ig);
+          slot_idx8<IdxT>(raw_u, idx12, iu);
           if (D4) {                   // four-value code words: two 8-byte reads per block
 #pragma unroll
             for (int j = 0; j < 8; ++j) mma_block(acc_u[j & 1], fx[j], lookup_d4(m.cb_u, iu[j], lane));

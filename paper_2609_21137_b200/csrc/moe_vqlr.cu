@@ -59,6 +59,7 @@ struct moe_vqlr_handle {
   signed char fused_xs[kMaxT + 1];                        // ... with the tokens staged in shared memory (else read from L2)
   StagePlan plan_gu_fused;
   bool per_expert_launch;   // ablation: gate/up and down run as one launch per work group
+  bool special;             // up-only experts or 12-bit indices: the tensor-core kernels' SP instantiations run
   bool d4;                  // four-value code words on the tensor-core paths (uint8 indices read as pairs)
   int idx_tc;               // bytes per index element as the tensor-core kernels read it (2 with d4)
   bool lrf;                 // chain gate/up: the low-rank groups ride on the slices (at least one per slice)
@@ -218,6 +219,63 @@ T* carve(char*& cur, size_t n) {
   return p;
 }
 
+// Launch through an untyped kernel pointer (the selectors below), as a link of the chain.
+cudaError_t launch_pdl_ptr(const void* kern, int grid, int block, size_t smem, cudaStream_t st, void** args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  const bool chain = st != nullptr && st != cudaStreamLegacy && st != cudaStreamPerThread;
+  cfg.attrs = at;
+  cfg.numAttrs = chain ? 1 : 0;
+  return cudaLaunchKernelExC(&cfg, kern, args);
+}
+
+// Which instantiation of a tensor-core kernel a handle runs.  SP = the instantiations that also
+// handle experts without a gate projection and 12-bit packed indices.
+template <bool SP>
+const void* gateup_kernel_sp(bool gu_dense, bool d4, int idx_bytes, bool lrf, bool lrf2) {
+  if (gu_dense) return (const void*)k_gateup_mma<uint16_t, true, false, 0, SP>;
+  if (d4) return lrf2 ? (const void*)k_gateup_mma<uint16_t, false, true, 2, SP> : lrf ? (const void*)k_gateup_mma<uint16_t, false, true, 1, SP>
+                                                                                       : (const void*)k_gateup_mma<uint16_t, false, true, 0, SP>;
+  if (idx_bytes == 1) return lrf2 ? (const void*)k_gateup_mma<uint8_t, false, false, 2, SP> : lrf ? (const void*)k_gateup_mma<uint8_t, false, false, 1, SP>
+                                                                                                   : (const void*)k_gateup_mma<uint8_t, false, false, 0, SP>;
+  return lrf2 ? (const void*)k_gateup_mma<uint16_t, false, false, 2, SP> : lrf ? (const void*)k_gateup_mma<uint16_t, false, false, 1, SP>
+                                                                               : (const void*)k_gateup_mma<uint16_t, false, false, 0, SP>;
+}
+template <bool SP>
+const void* down_kernel_sp(bool dn_dense, bool d4, int idx_bytes, int tpu) {
+  if (dn_dense) return (const void*)k_down_mma<uint16_t, true, false, 2, SP>;
+  if (d4) return tpu == 4 ? (const void*)k_down_mma<uint16_t, false, true, 4, SP> : (const void*)k_down_mma<uint16_t, false, true, 2, SP>;
+  if (idx_bytes == 1) return tpu == 4 ? (const void*)k_down_mma<uint8_t, false, false, 4, SP> : (const void*)k_down_mma<uint8_t, false, false, 2, SP>;
+  return tpu == 4 ? (const void*)k_down_mma<uint16_t, false, false, 4, SP> : (const void*)k_down_mma<uint16_t, false, false, 2, SP>;
+}
+template <typename IdxT, bool DENSE, bool D4V, bool SP>
+const void* fused_kernel_jd(int jd) {
+  return jd == 1 ? (const void*)k_expert_fused<IdxT, DENSE, 1, D4V, SP> : jd == 2 ? (const void*)k_expert_fused<IdxT, DENSE, 2, D4V, SP>
+       : jd == 3 ? (const void*)k_expert_fused<IdxT, DENSE, 3, D4V, SP> : (const void*)k_expert_fused<IdxT, DENSE, 4, D4V, SP>;
+}
+template <bool SP>
+const void* fused_kernel_sp(bool dn_dense, bool d4, int idx_bytes, int jd) {
+  if (d4) return dn_dense ? fused_kernel_jd<uint16_t, true, true, SP>(jd) : fused_kernel_jd<uint16_t, false, true, SP>(jd);
+  if (idx_bytes == 1) return dn_dense ? fused_kernel_jd<uint8_t, true, false, SP>(jd) : fused_kernel_jd<uint8_t, false, false, SP>(jd);
+  return dn_dense ? fused_kernel_jd<uint16_t, true, false, SP>(jd) : fused_kernel_jd<uint16_t, false, false, SP>(jd);
+}
+const void* gateup_kernel(const moe_vqlr_handle* h) {
+  return h->special ? gateup_kernel_sp<true>(h->gu_dense, h->d4, h->idx_bytes, h->lrf, h->lrf2)
+                    : gateup_kernel_sp<false>(h->gu_dense, h->d4, h->idx_bytes, h->lrf, h->lrf2);
+}
+const void* down_kernel(const moe_vqlr_handle* h, int tpu) {
+  return h->special ? down_kernel_sp<true>(h->dn_dense, h->d4, h->idx_bytes, tpu) : down_kernel_sp<false>(h->dn_dense, h->d4, h->idx_bytes, tpu);
+}
+const void* fused_kernel(const moe_vqlr_handle* h, int jd) {
+  return h->special ? fused_kernel_sp<true>(h->dn_dense, h->d4, h->idx_bytes, jd) : fused_kernel_sp<false>(h->dn_dense, h->d4, h->idx_bytes, jd);
+}
+
 // Enqueues the kernel of one stage (nothing for a stage this configuration does not have).
 cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, bf16* ob, cudaStream_t st, bool allow_coop) {
   const Params& P = h->P;
@@ -257,24 +315,14 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         StagePlan pgl = h->plan_gu_fused;
         pgl.x_smem = h->fused_xs[T];
         const size_t smem2 = fused_layout(P.K, h->n_books, T, P.H, P.r, pgl, fpl, h->dn_dense, h->idx_tc, P.E, P.k, P.S).total;
-#define MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, JDV, D4V)                                                                  \
-  le = launch_pdl(k_expert_fused<IDXT, DENSE, JDV, D4V>, h->sm_count, kFusedThreads, smem2, st, P, xb, T, pgl, fpl, h->n_books, \
-                  h->want_dbg, static_cast<const IDXT*>(DENSE ? nullptr : h->idx_dp))
-#define MOE_VQLR_FUSED_JD(IDXT, DENSE, D4V)                                  \
-  switch (fpl.jd) {                                                          \
-    case 1: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 1, D4V); break;               \
-    case 2: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 2, D4V); break;               \
-    case 3: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 3, D4V); break;               \
-    default: MOE_VQLR_FUSED_LAUNCH(IDXT, DENSE, 4, D4V); break;              \
-  }
-        if (h->d4 && h->dn_dense) { MOE_VQLR_FUSED_JD(uint16_t, true, true) }
-        else if (h->d4) { MOE_VQLR_FUSED_JD(uint16_t, false, true) }
-        else if (h->dn_dense && h->idx_bytes == 1) { MOE_VQLR_FUSED_JD(uint8_t, true, false) }
-        else if (h->dn_dense) { MOE_VQLR_FUSED_JD(uint16_t, true, false) }
-        else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_JD(uint8_t, false, false) }
-        else { MOE_VQLR_FUSED_JD(uint16_t, false, false) }
-#undef MOE_VQLR_FUSED_JD
-#undef MOE_VQLR_FUSED_LAUNCH
+        {
+          Params Pa = P;
+          const bf16* xa = xb;
+          int Ta = T, nb_a = h->n_books, dbg_a = h->want_dbg;
+          const void* idp = h->dn_dense ? nullptr : h->idx_dp;
+          void* args[] = {&Pa, &xa, &Ta, &pgl, &fpl, &nb_a, &dbg_a, &idp};
+          le = launch_pdl_ptr(fused_kernel(h, fpl.jd), h->sm_count, kFusedThreads, smem2, st, args);
+        }
         ran = true;
         break;
       }
@@ -321,16 +369,11 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         for (int gi = 0; gi < n_launch && le == cudaSuccess; ++gi) {
           StagePlan pl = h->plan_gu;
           if (h->per_expert_launch) pl.only_grp = gi;
-          if (h->gu_dense) le = launch_pdl(k_gateup_mma<uint16_t, true>, h->sm_count, kDenseThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->d4 && h->lrf2) le = launch_pdl(k_gateup_mma<uint16_t, false, true, 2>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->d4 && h->lrf) le = launch_pdl(k_gateup_mma<uint16_t, false, true, 1>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->d4) le = launch_pdl(k_gateup_mma<uint16_t, false, true>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->idx_bytes == 1 && h->lrf2) le = launch_pdl(k_gateup_mma<uint8_t, false, false, 2>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->idx_bytes == 1 && h->lrf) le = launch_pdl(k_gateup_mma<uint8_t, false, false, 1>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->idx_bytes == 1) le = launch_pdl(k_gateup_mma<uint8_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->lrf2) le = launch_pdl(k_gateup_mma<uint16_t, false, false, 2>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else if (h->lrf) le = launch_pdl(k_gateup_mma<uint16_t, false, false, 1>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
-          else le = launch_pdl(k_gateup_mma<uint16_t, false>, h->sm_count, kFastThreads, smem, st, P, xb, T, pl, h->n_books, h->want_dbg);
+          Params Pa = P;
+          const bf16* xa = xb;
+          int Ta = T, nb_a = h->n_books, dbg_a = h->want_dbg;
+          void* args[] = {&Pa, &xa, &Ta, &pl, &nb_a, &dbg_a};
+          le = launch_pdl_ptr(gateup_kernel(h), h->sm_count, h->gu_dense ? kDenseThreads : kFastThreads, smem, st, args);
         }
         h->launches += n_launch - 1;
         ran = true;
@@ -367,13 +410,10 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         for (int gi = 0; gi < n_launch && le == cudaSuccess; ++gi) {
           StagePlan pl = h->plan_dn;
           if (h->per_expert_launch) pl.only_grp = gi;
-          if (h->dn_dense) le = launch_pdl(k_down_mma<uint16_t, true>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else if (h->d4 && pl.tpu == 4) le = launch_pdl(k_down_mma<uint16_t, false, true, 4>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else if (h->d4) le = launch_pdl(k_down_mma<uint16_t, false, true, 2>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else if (h->idx_bytes == 1 && pl.tpu == 4) le = launch_pdl(k_down_mma<uint8_t, false, false, 4>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else if (h->idx_bytes == 1) le = launch_pdl(k_down_mma<uint8_t, false, false, 2>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else if (pl.tpu == 4) le = launch_pdl(k_down_mma<uint16_t, false, false, 4>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
-          else le = launch_pdl(k_down_mma<uint16_t, false, false, 2>, h->sm_count, kDownThreads, h->smem_fast_dn, st, P, T, pl);
+          Params Pa = P;
+          int Ta = T;
+          void* args[] = {&Pa, &Ta, &pl};
+          le = launch_pdl_ptr(down_kernel(h, pl.tpu), h->sm_count, kDownThreads, h->smem_fast_dn, st, args);
         }
         h->launches += n_launch - 1;
         ran = true;
@@ -605,23 +645,9 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
     h->idx_tc = h->d4 ? 2 : h->idx_bytes;
     if (ok) {
       cudaError_t e1 = cudaSuccess, e2 = cudaSuccess;
-      if (gu_dn) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, true>, (size_t)smem_gu);
-      else if (d4 && h->lrf2) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, true, 2>, (size_t)smem_gu);
-      else if (d4 && h->lrf) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, true, 1>, (size_t)smem_gu);
-      else if (d4) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, true>, (size_t)smem_gu);
-      else if (h->idx_bytes == 1 && h->lrf2) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint8_t, false, false, 2>, (size_t)smem_gu);
-      else if (h->idx_bytes == 1 && h->lrf) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint8_t, false, false, 1>, (size_t)smem_gu);
-      else if (h->idx_bytes == 1) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint8_t, false>, (size_t)smem_gu);
-      else if (h->lrf2) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, false, 2>, (size_t)smem_gu);
-      else if (h->lrf) e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false, false, 1>, (size_t)smem_gu);
-      else e1 = raise_dyn_smem((const void*)k_gateup_mma<uint16_t, false>, (size_t)smem_gu);
-      if (h->dn_dense) e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, true>, (size_t)h->smem_fast_dn);
-      else if (d4 && h->plan_dn.tpu == 4) e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, false, true, 4>, (size_t)h->smem_fast_dn);
-      else if (d4) e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, false, true, 2>, (size_t)h->smem_fast_dn);
-      else if (h->idx_bytes == 1 && h->plan_dn.tpu == 4) e2 = raise_dyn_smem((const void*)k_down_mma<uint8_t, false, false, 4>, (size_t)h->smem_fast_dn);
-      else if (h->idx_bytes == 1) e2 = raise_dyn_smem((const void*)k_down_mma<uint8_t, false, false, 2>, (size_t)h->smem_fast_dn);
-      else if (h->plan_dn.tpu == 4) e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, false, false, 4>, (size_t)h->smem_fast_dn);
-      else e2 = raise_dyn_smem((const void*)k_down_mma<uint16_t, false, false, 2>, (size_t)h->smem_fast_dn);
+      h->special = (P.act == 2 || P.idx12) && !gu_dn;
+      e1 = raise_dyn_smem(gateup_kernel(h), smem_gu);
+      e2 = raise_dyn_smem(down_kernel(h, h->plan_dn.tpu), h->smem_fast_dn);
       cudaError_t e3 = raise_dyn_smem((const void*)k_act_zdown, (size_t)((size_t)I * sizeof(float)));
       if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) { cudaGetLastError(); h->fast = false; }
     }
@@ -769,17 +795,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
           if (!fit) break;                         // more tokens need more room
           maxT_fit = t;
         }
-        const void* fn = nullptr;
-#define MOE_VQLR_FUSED_FN(IDXT, DENSE, D4V)                                                             \
-  fn = fp.jd == 1 ? (const void*)k_expert_fused<IDXT, DENSE, 1, D4V> : fp.jd == 2 ? (const void*)k_expert_fused<IDXT, DENSE, 2, D4V> \
-     : fp.jd == 3 ? (const void*)k_expert_fused<IDXT, DENSE, 3, D4V> : (const void*)k_expert_fused<IDXT, DENSE, 4, D4V>
-        if (h->d4 && h->dn_dense) { MOE_VQLR_FUSED_FN(uint16_t, true, true); }
-        else if (h->d4) { MOE_VQLR_FUSED_FN(uint16_t, false, true); }
-        else if (h->dn_dense && h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, true, false); }
-        else if (h->dn_dense) { MOE_VQLR_FUSED_FN(uint16_t, true, false); }
-        else if (h->idx_bytes == 1) { MOE_VQLR_FUSED_FN(uint8_t, false, false); }
-        else { MOE_VQLR_FUSED_FN(uint16_t, false, false); }
-#undef MOE_VQLR_FUSED_FN
+        const void* fn = fused_kernel(h, fp.jd);
         cudaError_t e1 = raise_dyn_smem((const void*)fn, (size_t)smem_max);
         const size_t cf_smem = ((size_t)(k + S) * (r > 0 ? r : 0) + (size_t)(k + S) * kCfCols * 2) * sizeof(float);
         if (e1 == cudaSuccess && cf_smem > 48 * 1024)
