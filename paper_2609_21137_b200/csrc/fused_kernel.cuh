@@ -501,6 +501,12 @@ k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePla
 // ---------------------------------------------------------------------------------------------
 constexpr int kCfCols = 8;
 constexpr int kCfThreads = 256;
+// For a single token the kernel's 128 blocks are asked to be ALONE on their SM: the launch requests
+// more than half an SM's shared memory.  Blocks of this kernel become resident one SM at a time as
+// the expert kernel's blocks leave; with two per SM the first SMs to empty took two blocks each and
+// those pairs shared one SM's path to memory for their cold rows of the down factor (measured: layer
+// 24.4 us with two blocks per SM, 23.8 us with one).
+constexpr size_t kCfAloneBytes = 120 * 1024;
 
 __global__ void __launch_bounds__(kCfThreads)
 k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr) {
@@ -512,12 +518,37 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
   const int units_per_tok = H2 / kCfCols;
   const int t = blockIdx.x / units_per_tok, h2 = (blockIdx.x - t * units_per_tok) * kCfCols + col;
   TRACE_STAMP(2, 8);
-  pdl_wait();
-  TRACE_STAMP(2, 9);
-  pdl_launch();
   // Every load of a thread is requested before the first one is used: the kernel is a handful of
   // dependent round trips long, not a loop of them.
   constexpr int kYv = 8, kAv = 4;      // slices / rank groups per thread held in registers (more: second pass)
+  // Before the wait: a block of this kernel becomes resident when an SM runs out of expert-kernel
+  // blocks, a microsecond or more before the LAST of them is done, and until now it sat out that
+  // time.  The rows of the down factor that it needs depend only on the routing, which the expert
+  // kernel published at its start: they are requested now, for the first trip over the slots, with
+  // the expert ids as they stand in memory.  Memory written by the preceding kernel is only
+  // guaranteed to be visible after the wait, so the ids are read again then and a thread whose id
+  // has changed asks again; the speculation costs nothing when it fails and a DRAM round trip less
+  // when it holds.
+  int e_spec = -1;
+  uint4 a0v[kAv], a1v[kAv];
+  if (lr && sl < n_slots) {
+    e_spec = sl < P.k ? __ldcg(P.topk_id + t * P.k + sl) : P.E + (sl - P.k);
+    if ((unsigned int)e_spec >= (unsigned int)(P.E + P.S)) e_spec = 0;        // whatever the memory held: stay in range
+    const uint4* a0 = reinterpret_cast<const uint4*>(P.down.factor + ((size_t)e_spec * P.H + 2 * h2) * r);
+    const uint4* a1 = reinterpret_cast<const uint4*>(P.down.factor + ((size_t)e_spec * P.H + 2 * h2 + 1) * r);
+#pragma unroll
+    for (int i = 0; i < kAv; ++i) {
+      const int rg = q + 4 * i;
+      a0v[i] = a1v[i] = make_uint4(0, 0, 0, 0);
+      if (rg < r / 8) {                  // volatile: these requests must leave before the wait below, not after it
+        asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a0v[i].x), "=r"(a0v[i].y), "=r"(a0v[i].z), "=r"(a0v[i].w) : "l"(a0 + rg));
+        asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a1v[i].x), "=r"(a1v[i].y), "=r"(a1v[i].z), "=r"(a1v[i].w) : "l"(a1 + rg));
+      }
+    }
+  }
+  pdl_wait();
+  TRACE_STAMP(2, 9);
+  pdl_launch();
   for (int s0 = 0; s0 < n_slots; s0 += kCfThreads / 32) {      // uniform trip count for the shuffles and barriers
     const int s = s0 + sl;
     const bool live = s < n_slots;
@@ -527,6 +558,7 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
       pos = __ldcg(P.inv_pos + t * n_slots + s);
       e = s < P.k ? __ldcg(P.topk_id + t * P.k + s) : P.E + (s - P.k);
     }
+    const bool spec_ok = s0 == 0 && e == e_spec;        // the rows requested before the wait are the right ones
     // the first two z_d entries of this thread (slot sj, rank rho): their positions travel with `pos`
     const int n_here = min(kCfThreads / 32, n_slots - s0);
     const int n_zd = lr ? n_here * r : 0;
@@ -539,7 +571,6 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
       zpj[u] = idx < n_zd ? __ldcg(P.inv_pos + t * n_slots + s0 + zsj[u]) : 0;
     }
     float2 yv[kYv];
-    uint4 a0v[kAv], a1v[kAv];
     const float* ysrc = P.ypart + (size_t)pos * P.H + 2 * h2;
     const uint4* a0 = reinterpret_cast<const uint4*>(P.down.factor + ((size_t)e * P.H + 2 * h2) * r);
     const uint4* a1 = reinterpret_cast<const uint4*>(P.down.factor + ((size_t)e * P.H + 2 * h2 + 1) * r);
@@ -553,8 +584,10 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
     for (int i = 0; i < kAv; ++i) {
       const int rg = q + 4 * i;
       const bool on = live && lr && rg < r / 8;
-      a0v[i] = on ? __ldg(a0 + rg) : make_uint4(0, 0, 0, 0);
-      a1v[i] = on ? __ldg(a1 + rg) : make_uint4(0, 0, 0, 0);
+      if (!spec_ok) {
+        a0v[i] = on ? __ldg(a0 + rg) : make_uint4(0, 0, 0, 0);
+        a1v[i] = on ? __ldg(a1 + rg) : make_uint4(0, 0, 0, 0);
+      }
     }
     if (lr) {                            // z_d of this trip's slots: sum of the slices' parts, ascending
       float zv[2][16];

@@ -328,7 +328,8 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
       }
       case 5: {
         const int lr = (!h->dn_dense && P.r > 0) ? 1 : 0;
-        const size_t smem = ((lr ? (size_t)(P.k + P.S) * P.r : 0) + (size_t)(P.k + P.S) * kCfCols * 2) * sizeof(float);
+        size_t smem = ((lr ? (size_t)(P.k + P.S) * P.r : 0) + (size_t)(P.k + P.S) * kCfCols * 2) * sizeof(float);
+        if (smem < kCfAloneBytes && T == 1) smem = kCfAloneBytes;      // one block per SM (see kCfAloneBytes)
         le = launch_pdl(k_combine_fused, T * (P.H / 2 / kCfCols), kCfThreads, smem, st, P, ob, T, h->fplan.n_sl, lr);
         ran = true;
         break;
@@ -797,7 +798,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
         }
         const void* fn = fused_kernel(h, fp.jd);
         cudaError_t e1 = raise_dyn_smem((const void*)fn, (size_t)smem_max);
-        const size_t cf_smem = ((size_t)(k + S) * (r > 0 ? r : 0) + (size_t)(k + S) * kCfCols * 2) * sizeof(float);
+        size_t cf_smem = ((size_t)(k + S) * (r > 0 ? r : 0) + (size_t)(k + S) * kCfCols * 2) * sizeof(float);
+        if (cf_smem < kCfAloneBytes) cf_smem = kCfAloneBytes;
         if (e1 == cudaSuccess && cf_smem > 48 * 1024)
           e1 = cf_smem <= limit ? raise_dyn_smem((const void*)k_combine_fused, (size_t)cf_smem) : cudaErrorInvalidValue;
         if (e1 == cudaSuccess && maxT_fit >= 1) {
