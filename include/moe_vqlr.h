@@ -10,7 +10,7 @@
  *   the k experts with the largest logits per token (ties: lower expert id), affinities a =
  *       softmax over the k selected logits (or over all E when renorm_topk == 0)
  *   grouping of the (token, slot) pairs by expert, so each activated expert's payload is read
- *       once per layer whatever the batch size (Section 5.5)
+ *       once per layer whatever the batch size (Section 5.6)
  *   per projection P in {gate, up, down}, per activated expert e (Eq. 1, stored transposed):
  *       W_P,e[o][b*d+j] = codebook_P[ idx_P[e][o][b] ][j] + sum_rho factor_P[e][o][rho]*basis_P[rho][b*d+j]
  *     evaluated without ever forming W: the VQ part by code-word lookups, the low-rank part as

@@ -120,7 +120,7 @@ void oracle_topk_affinity(const double* logits, int T, int E, int k, int renorm,
 }
 
 /* Grouping of the T*k (token, slot) pairs by expert so that each activated expert's payload
- * is used once per layer (Section 5.5, batch scaling).  Pairs of one expert keep ascending
+ * is used once per layer (Section 5.6, batch scaling).  Pairs of one expert keep ascending
  * token order. */
 void oracle_group_by_expert(const int32_t* ids, int T, int k, int E, int32_t* counts,
                             int32_t* offsets, int32_t* pair_token, int32_t* pair_slot) {

@@ -3,7 +3,7 @@
 Counts follow the paper's per-projection load table (Appendix "Exact engine-work counts"):
 shared loads of the code book (16 K d bits) and the basis (16 in r bits) once per token batch,
 expert-private loads of the index map ((in out / d) b_J bits) and coefficients (16 out r bits)
-once per distinct activated expert (Section 5.5: every batch size loads only the activated
+once per distinct activated expert (Section 5.6: every batch size loads only the activated
 experts), plus the router matrix, the dense bf16 projections where a projection is kept
 uncompressed (Section 3.1), and the token vectors in and out.
 """

@@ -3,8 +3,9 @@ same seeded layer and checks the acceptance bars.
 
 Bars: routing ids and grouping bit-exact; affinities to 2e-6; bf16 outputs against the fp64
 oracle with (i) elementwise |err| / max(|y|, 1e-3 * max|y|) <= 2e-2, (ii) max|err| / max|y| <=
-2e-2, (iii) mean |err| <= 1e-3 + mean|bf16(y) - y| (the second term is the rounding error any
-bf16 output carries).
+2e-2, (iii) mean |err| <= 1e-3 as stated -- except on layers whose OUTPUT FORMAT alone breaks that
+bar: where rounding the oracle's own result to bf16 already costs more than 1e-3 of mean error (the
+Mixtral-shaped layers: outputs of rms 2, 2.3e-3), the bar is 1e-3 on top of that rounding error.
 """
 import numpy as np
 import torch
@@ -33,8 +34,10 @@ def make_checked_layer(shp, seed=0, max_tries=20, tie=None, **oracle_kw):
         res = oracle.OracleLayer.from_synth(layer, **oracle_kw).decode_layer(layer.x)
         if tie is not None:
             return layer, res, s
-        if shp.k == shp.E or logit_gaps(res, shp.k) > MIN_LOGIT_GAP:
+        gap = np.inf if shp.k == shp.E else logit_gaps(res, shp.k)
+        if gap > MIN_LOGIT_GAP:
             return layer, res, s
+        print(f"[make_checked_layer] {shp.name} seed {s} rejected: smallest logit gap {gap:.3g} <= {MIN_LOGIT_GAP}")
     raise RuntimeError("no seed with separated logits")
 
 
@@ -57,7 +60,9 @@ def assert_output(out_gpu: np.ndarray, ref: np.ndarray, what=""):
     m = output_metrics(out_gpu, ref)
     assert m["max_rel"] <= REL_TOL, (what, m)
     assert m["norm_max"] <= REL_TOL, (what, m)
-    assert m["mae"] <= MAE_TOL + m["mae_format"], (what, m)
+    # the format term is granted only where the format by itself exceeds the bar (no correct bf16 output could pass)
+    mae_bar = MAE_TOL + m["mae_format"] if m["mae_format"] > MAE_TOL else MAE_TOL
+    assert m["mae"] <= mae_bar, (what, m)
     return m
 
 
