@@ -525,6 +525,9 @@ def main():
            "how": "moe_vqlr_decode_layer_host with pinned host buffers, one call after the other, wall clock around "
                   "the loop; every handle made one call before the clock started (its first call captures graphs)"}
     n_layers = len(wl.layers)
+    specialized = {"layers_with_kernels_compiled_for_their_shape": sum(1 for l in wl.layers if l.specialized()),
+                   "of": len(wl.layers),
+                   "note": next((l.specialization_note() for l in wl.layers if not l.specialized()), "")}
     wl.close()
 
     extras = []
@@ -567,6 +570,7 @@ def main():
                            "l2": f"rotation over {n_layers} distinct layers touches "
                                  f"{n_layers * wl.mean_bytes / 1e6:.0f} MB per pass, larger than the 126 MB L2",
                            "launch": "each rotation over the layers is one captured CUDA graph; kernels of a call are linked by programmatic dependent launch",
+                           "specialized": specialized,
                            "parallelism": "replicas only" if world > 1 else "single GPU"},
                 "tokens_per_s_per_layer": shp.T * world / (ms_per_step * 1e-3),
                 "hbm_gbs": layer_gbs, "hbm_frac_of_measured": layer_gbs / peak,

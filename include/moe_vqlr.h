@@ -118,6 +118,9 @@ enum {
                                          weighted sum (the default for calls whose work items fill
                                          at most one wave of blocks): always the chain of kernels */
   MOE_VQLR_FLAG_FORCE_FUSED = 128u,      /* ... or run every call that fits its shared memory that way */
+  MOE_VQLR_FLAG_NO_SPECIALIZE = 16384u,  /* do not compile the single-token kernels for this layer's
+                                         shape at create() (see moe_vqlr_specialized): the library's
+                                         precompiled kernels run */
   MOE_VQLR_FLAG_GENERIC_KERNELS = 256u,  /* only the generic CUDA-core kernels (one warp per output
                                          row), which otherwise serve the shapes the tensor-core
                                          kernels do not cover */
@@ -171,6 +174,9 @@ typedef struct {
   int32_t* pair_slot;  /* [T*k]                                                                */
 } moe_vqlr_debug;
 
+#ifndef __CUDACC_RTC__ /* host entry points (the library's run-time-compiled kernels include this
+                          file for the types and constants above) */
+
 /* Validates the configuration, allocates the handle and its device workspace on the CURRENT
  * CUDA device and returns the handle in *out (NULL on failure).  Synchronous.
  * Errors: INVALID_ARG, UNSUPPORTED (vq_dim not 8 or 4, H or I not a multiple of 8, K > 65536, k > 32,
@@ -201,6 +207,20 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
  * two pointers; other pointers re-capture it. */
 int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T, void* out_host,
                                void* cuda_stream);
+
+/* Shape specialisation.  Where a configuration's single-token calls run as router -> fused expert
+ * kernel -> weighted sum, create() compiles that path once more for exactly this layer (NVRTC; the
+ * library's own kernel source, found beside the library file, with the layer's sizes, expert count,
+ * top-k, rank, code-book size and work plan as compile-time constants: the GPU-side counterpart of
+ * the ahead-of-time, per-model mapping of Section 4).  Same arithmetic in the same order, so results
+ * are bitwise those of the precompiled kernels; a batch-1 call is shorter because its blocks fetch
+ * about half the instructions.  Costs a few seconds at the first create() of a shape (kept per
+ * process and device afterwards).  Needs libnvrtc and the CUDA headers under /usr/local/cuda; where
+ * they are missing, or with MOE_VQLR_FLAG_NO_SPECIALIZE, the precompiled kernels run.
+ * moe_vqlr_specialized: number of kernels of the handle that were compiled that way (0 if none);
+ * moe_vqlr_specialization_note: why not (empty string if they were), valid until destroy. */
+int moe_vqlr_specialized(const moe_vqlr_handle* h);
+const char* moe_vqlr_specialization_note(const moe_vqlr_handle* h);
 
 /* The status word of the handle: conditions that only the kernels can detect while a call runs.
  * Returns MOE_VQLR_OK, or the code a kernel of an earlier call recorded, and clears the word:
@@ -250,6 +270,8 @@ const char* moe_vqlr_last_error(const moe_vqlr_handle* h);
 int moe_vqlr_route_noalloc(const void* x, const void* router_w, const float* router_bias,
                            int32_t T, int32_t E, int32_t H, int32_t k, int32_t renorm_topk,
                            int32_t* topk_id, float* topk_w, void* cuda_stream);
+
+#endif /* !__CUDACC_RTC__ */
 
 #ifdef __cplusplus
 }

@@ -30,9 +30,11 @@ FLAG_PROJECTION_CODE_BOOK = 512
 FLAG_PHASE_CLOCKS = 1024
 FLAG_ACT_RELU2_UP_ONLY = 4096
 FLAG_IDX12 = 8192
+FLAG_NO_SPECIALIZE = 16384
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
-           "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_last_status", "moe_vqlr_launch_count",
+           "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_last_status", "moe_vqlr_specialized",
+           "moe_vqlr_specialization_note", "moe_vqlr_launch_count",
            "moe_vqlr_workspace_bytes", "moe_vqlr_set_profiling", "moe_vqlr_last_stage_times",
            "moe_vqlr_stage_count", "moe_vqlr_stage_name", "moe_vqlr_route_noalloc",
            "moe_vqlr_run_stage", "moe_vqlr_phase_clocks", "moe_vqlr_probe_lookup_rate"]
@@ -85,6 +87,10 @@ def _load():
     lib.moe_vqlr_last_error.argtypes = [C.c_void_p]
     lib.moe_vqlr_last_status.restype = C.c_int
     lib.moe_vqlr_last_status.argtypes = [C.c_void_p]
+    lib.moe_vqlr_specialized.restype = C.c_int
+    lib.moe_vqlr_specialized.argtypes = [C.c_void_p]
+    lib.moe_vqlr_specialization_note.restype = C.c_char_p
+    lib.moe_vqlr_specialization_note.argtypes = [C.c_void_p]
     lib.moe_vqlr_launch_count.restype = C.c_int64
     lib.moe_vqlr_launch_count.argtypes = [C.c_void_p]
     lib.moe_vqlr_workspace_bytes.restype = C.c_int64
@@ -282,6 +288,14 @@ class MoeVqlrLayer:
         """Status word of the handle (0, or the code a kernel recorded); reading clears it.
         Synchronize the stream of the calls in question first."""
         return int(_lib.moe_vqlr_last_status(self._h))
+
+    def specialized(self) -> int:
+        """Number of kernels of the single-token path that create() compiled for this layer's shape."""
+        return int(_lib.moe_vqlr_specialized(self._h))
+
+    def specialization_note(self) -> str:
+        """Why there are none (empty string if there are)."""
+        return _lib.moe_vqlr_specialization_note(self._h).decode()
 
     def set_profiling(self, on: bool) -> None:
         self._check(_lib.moe_vqlr_set_profiling(self._h, 1 if on else 0))

@@ -1,11 +1,13 @@
 // Shared definitions of the CUDA kernels: parameter block, bf16 helpers, warp reductions.
 #pragma once
 #include "moe_vqlr.h"
+#ifndef __CUDACC_RTC__       // the run-time compiler has the device built-ins and takes no host headers
 #include "moe_vqlr_bench.h"
-
-#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#endif
+#include <cuda_bf16.h>
+#include <math_constants.h>
 
 namespace {
 
@@ -74,6 +76,18 @@ struct Params {
   long long* clk;          // optional phase stamps [kernel 4][block][warp 16][stamp 16], or NULL
   int clk_blocks;
 };
+
+#ifdef MOE_VQLR_JIT
+// Run-time-compiled copies of the kernels know the layer: every integer of the parameter block is
+// a constant of the compilation (the pointers stay arguments, so one copy serves all layers of a
+// shape).
+#define MOE_VQLR_JIT_PARAMS(P)                                                                          \
+  do {                                                                                                  \
+    (P).H = J_H; (P).I = J_I; (P).E = J_E; (P).k = J_TOPK; (P).S = J_S; (P).K = J_K; (P).r = J_R;       \
+    (P).renorm = J_RENORM; (P).act = J_ACT; (P).d = J_D; (P).idx12 = J_IDX12; (P).z_repeat = J_ZREPEAT; \
+    (P).n_zrows = J_NZROWS; (P).gate.zslot = J_ZSLOT_G; (P).up.zslot = J_ZSLOT_U;                       \
+  } while (0)
+#endif
 
 // The model-specific expert activation phi applied to the gate output (Section 2.1):
 // p = phi(g) * u.  act is uniform over the launch.

@@ -198,7 +198,7 @@ __device__ __forceinline__ uint4 lookup_d4(const uint4* s_cb, uint32_t pair, int
 struct FastDiv {
   unsigned int mul, shr;      // mul == 0: divisor 1
 };
-__host__ inline FastDiv make_fastdiv(unsigned int d) {
+__host__ __device__ inline FastDiv make_fastdiv(unsigned int d) {
   FastDiv f = {0u, 0u};
   if (d <= 1u) return f;
   unsigned int L = 0;
@@ -380,7 +380,7 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
     float denom = ev;
     if (!P.renorm)
       for (int e = lane, j = 0; e < E; e += 32, ++j)
-        if (!((taken >> j) & 1u) && row[e] != -INFINITY) denom += expf(row[e] - lmax);
+        if (!((taken >> j) & 1u) && row[e] != -CUDART_INF_F) denom += expf(row[e] - lmax);
     denom = warp_sum(denom);
     const float aff = ev / denom;
     if (lane < k) {

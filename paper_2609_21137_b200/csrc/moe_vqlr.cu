@@ -17,6 +17,7 @@
 #include "coop_kernel.cuh"
 #include "fused_kernel.cuh"
 #include "pcb_kernel.cuh"
+#include "jit_host.cuh"
 
 #include <cstdarg>
 #include <cstdio>
@@ -68,6 +69,8 @@ struct moe_vqlr_handle {
   int pcb_min_T;            // ... and used from this many tokens on
   int pcb_Q;                // table pieces per token = ceil(H / 8 / 64)
   size_t smem_lr;           // dynamic shared memory of k_gateup_lr
+  const void* jit_fused;     // k_expert_fused compiled at create() for this layer's shape (single-token calls), or NULL
+  std::string jit_note;      // why there is none
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
   size_t workspace_bytes;
@@ -321,7 +324,8 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           int Ta = T, nb_a = h->n_books, dbg_a = h->want_dbg;
           const void* idp = h->dn_dense ? nullptr : h->idx_dp;
           void* args[] = {&Pa, &xa, &Ta, &pgl, &fpl, &nb_a, &dbg_a, &idp};
-          le = launch_pdl_ptr(fused_kernel(h, fpl.jd), h->sm_count, kFusedThreads, smem2, st, args);
+          const void* fn = (h->jit_fused && T == 1 && !h->want_dbg) ? h->jit_fused : fused_kernel(h, fpl.jd);
+          le = launch_pdl_ptr(fn, h->sm_count, kFusedThreads, smem2, st, args);
         }
         ran = true;
         break;
@@ -815,8 +819,46 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
     }
   }
 
-  // workspace
+  // The single-token path compiled for this layer's shape (see jit_host.cuh).
   const bool want_clk = (cfg->flags & MOE_VQLR_FLAG_PHASE_CLOCKS) != 0;
+  h->jit_fused = nullptr;
+  if (cfg->flags & MOE_VQLR_FLAG_NO_SPECIALIZE) h->jit_note = "switched off by MOE_VQLR_FLAG_NO_SPECIALIZE";
+  else if (!h->fused || h->fused_dg[1] == 0) h->jit_note = "single-token calls of this configuration do not run the fused kernel";
+  else if ((k + S) * h->fplan.n_sl > h->sm_count) h->jit_note = "a single token's work items exceed one wave";
+  else if (want_clk) h->jit_note = "phase clocks are recorded by the generic kernels";
+  else {
+    const FusedPlan& fp = h->fplan;
+    const StagePlan& pg = h->plan_gu_fused;
+    std::vector<std::string> defs;
+    auto def = [&](const char* name, long long v) { defs.push_back(std::string("-D") + name + "=" + std::to_string(v)); };
+    def("J_H", H); def("J_I", I); def("J_E", E); def("J_TOPK", k); def("J_S", S); def("J_K", K); def("J_R", r);
+    def("J_RENORM", P.renorm); def("J_ACT", P.act); def("J_D", P.d); def("J_IDX12", P.idx12); def("J_ZREPEAT", P.z_repeat);
+    def("J_NZROWS", P.n_zrows); def("J_ZSLOT_G", P.gate.zslot); def("J_ZSLOT_U", P.up.zslot);
+    def("J_NBOOKS", h->n_books); def("J_NB", pg.nb); def("J_NSLICES", pg.n_slices); def("J_NLR", pg.n_lr); def("J_NPARTS", pg.n_parts);
+    def("J_REPL", pg.repl); def("J_XSMEM", h->fused_xs[1]);
+    def("J_TPS", fp.tps); def("J_NSL", fp.n_sl); def("J_TLAST", fp.t_last); def("J_JD", fp.jd); def("J_RP_LOG2", fp.rp_log2);
+    def("J_DEPTH_G", h->fused_dg[1]); def("J_DEPTH_D", h->fused_dd[1]);
+    defs.push_back(std::string("-DJ_IDXT=") + ((h->d4 || h->idx_bytes == 2) ? "uint16_t" : "uint8_t"));
+    defs.push_back(std::string("-DJ_DENSE=") + (h->dn_dense ? "true" : "false"));
+    defs.push_back(std::string("-DJ_D4=") + (h->d4 ? "true" : "false"));
+    defs.push_back(std::string("-DJ_SP=") + (h->special ? "true" : "false"));
+    cudaLibrary_t lib = jit_library(defs, &h->jit_note);
+    if (lib) {
+      cudaKernel_t kern = nullptr;
+      FusedPlan fp1 = fp;
+      fp1.depth_g = h->fused_dg[1];
+      fp1.depth_d = h->fused_dd[1];
+      StagePlan pg1 = pg;
+      pg1.x_smem = h->fused_xs[1];
+      const size_t smem1 = fused_layout(K, h->n_books, 1, H, r, pg1, fp1, h->dn_dense, h->idx_tc, E, k, S).total;
+      cudaError_t je = cudaLibraryGetKernel(&kern, lib, "k_expert_fused_jit");
+      if (je == cudaSuccess) je = raise_dyn_smem((const void*)kern, smem1);
+      if (je == cudaSuccess) { h->jit_fused = (const void*)kern; h->jit_note.clear(); }
+      else { h->jit_note = std::string("loading the compiled kernel: ") + cudaGetErrorString(je); cudaGetLastError(); }
+    }
+  }
+
+  // workspace
   const size_t n_pos = (size_t)maxT * (k + S);
   unsigned int* idx_max = nullptr;      // scratch of the index validation
   auto plan = [&](char* base) {
@@ -1063,6 +1105,10 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
   if (ce != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "copy out: %s", cudaGetErrorString(ce));
   return take_status(h);
 }
+
+int moe_vqlr_specialized(const moe_vqlr_handle* h) { return (h && h->jit_fused) ? 1 : 0; }
+
+const char* moe_vqlr_specialization_note(const moe_vqlr_handle* h) { return h ? h->jit_note.c_str() : ""; }
 
 int moe_vqlr_last_status(moe_vqlr_handle* h) {
   if (!h) return MOE_VQLR_ERR_INVALID_ARG;

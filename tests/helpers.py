@@ -84,4 +84,11 @@ def run_gpu(layer, T=None, debug=True, **kw):
     x = binding.bits_to_device(layer.x if T is None else layer.x[:T], "cuda")
     result = mod.decode(x, debug=debug)
     torch.cuda.synchronize()
+    if debug and x.shape[0] == 1 and mod.specialized():
+        # a call that asks for the routing lists runs the precompiled kernels; the plain call runs the
+        # copies compiled for this shape, which must give the same bits
+        plain = mod.decode(x)
+        torch.cuda.synchronize()
+        assert torch.equal(plain.view(torch.int16), result[0].view(torch.int16)), \
+            "shape-specialised kernels differ from the precompiled ones"
     return mod, result
