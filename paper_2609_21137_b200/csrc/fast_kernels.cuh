@@ -779,7 +779,16 @@ __device__ __forceinline__ void router_z_unit_row8(const Params& P, const bf16* 
 // The weight row of a unit is requested BEFORE the wait for the previous kernel of the stream: the
 // weights never depend on it (only the tokens and the logits / z buffers do), so the DRAM round
 // trip of the row overlaps the previous kernel's tail.
-__global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
+// LEAN (the copy compiled per shape, see jit_host.cuh): a single token, the layer's sizes constants.
+template <bool LEAN>
+__device__ __forceinline__ void router_z_pdl_body(const Params& P_in, const bf16* __restrict__ x, int T_in) {
+  const int T = LEAN ? 1 : T_in;
+#ifdef MOE_VQLR_JIT
+  Params P = P_in;
+  MOE_VQLR_JIT_PARAMS(P);
+#else
+  const Params& P = P_in;
+#endif
   int unit = blockIdx.x * kRouterWarps + (threadIdx.x >> 5);
   const int base_units = router_z_units(P, T), lane = threadIdx.x & 31;
   const bool has = unit < router_z_units_launched(P, T);
@@ -805,6 +814,12 @@ __global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params
   TRACE_STAMP(0, 10);
 }
 
+#ifndef MOE_VQLR_JIT
+__global__ void __launch_bounds__(32 * kRouterWarps) k_router_z_pdl(const Params P, const bf16* __restrict__ x, int T) {
+  router_z_pdl_body<false>(P, x, T);
+}
+#endif
+
 // k_router_zmma_pdl: head of the chain for 9..16 tokens.  The shared projections z = basis * x
 // (Section 4.2) run on the tensor cores: one block per eight basis rows, each of its eight warps
 // takes an eighth of H with the tokens as the sixteen rows of the m16n8k16 tile (tokens 0..7 in
@@ -815,6 +830,7 @@ constexpr int kZmmaWarps = 8;
 
 __host__ __device__ __forceinline__ int zmma_blocks(const Params& P) { return P.n_zrows / 8 * P.z_repeat; }
 
+#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
 __global__ void __launch_bounds__(32 * kZmmaWarps) k_router_zmma_pdl(const Params P, const bf16* __restrict__ x, int T) {
   __shared__ float s_red[kZmmaWarps][128];
   pdl_wait();      // the previous call's kernels may still read logits / z
@@ -862,6 +878,7 @@ __global__ void __launch_bounds__(32 * kZmmaWarps) k_router_zmma_pdl(const Param
     if (tok < T) P.z[((size_t)tok * 2 + slot) * P.r + rho0 + row] = sum;
   }
 }
+#endif
 
 // Splits `total` units evenly over `parts` warps: first unit of warp `idx` = floor(total * idx / parts),
 // in 32-bit arithmetic (parts < 65536).
@@ -1361,15 +1378,18 @@ __device__ __forceinline__ void act_zdown_unit(const Params& P, int n_pos, int n
   }
 }
 
+#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
 __global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n_pos, int n_parts, int with_zd, int zsplit) {
   extern __shared__ float s_p[];                 // [I]
   pdl_launch();                                  // the down kernel may stage its code book meanwhile
   pdl_wait();
   act_zdown_unit(P, n_pos, n_parts, with_zd, zsplit, blockIdx.x, s_p);
 }
+#endif
 
 // The same link as two fully parallel kernels, for layers with few pairs or a long intermediate:
 // k_act (one thread per pair of p values) and k_zdown_pdl (one warp per z_d value).
+#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
 __global__ void __launch_bounds__(256) k_act(const Params P, int n_pos, int n_parts) {
   pdl_launch();
   pdl_wait();
@@ -1397,9 +1417,11 @@ __global__ void __launch_bounds__(256) k_act(const Params P, int n_pos, int n_pa
         __floats2bfloat162_rn(p0 - __low2float(hi), p1 - __high2float(hi));
   }
 }
+#endif
 
 // wpd warps share one z_d value (a long intermediate would otherwise be one warp's serial stream
 // of dependent loads); their partial sums meet in shared memory and are added in warp order.
+#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
 __global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos, int wpd) {
   __shared__ float s_part[8];
   pdl_launch();
@@ -1444,9 +1466,11 @@ __global__ void __launch_bounds__(256) k_zdown_pdl(const Params P, int n_pos, in
     P.zd[d] = sum;
   }
 }
+#endif
 
 // The same with four consecutive ranks per unit (many pairs: the pair's p values, two thirds of the
 // bytes of a dot product, are loaded once for four basis rows).
+#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
 __global__ void __launch_bounds__(256) k_zdown4_pdl(const Params P, int n_pos, int wpd) {
   // one unit = (pair, four consecutive ranks): the pair's p values are loaded once for the four rows
   __shared__ float s_part[8][4];
@@ -1501,6 +1525,7 @@ __global__ void __launch_bounds__(256) k_zdown4_pdl(const Params P, int n_pos, i
     P.zd[(size_t)pos * P.r + rho + lane] = sum;
   }
 }
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // k_down_mma: partial y tiles for every (work group, slice of I, 8-row tile of H); activations
@@ -1796,6 +1821,7 @@ __device__ __forceinline__ void combine_unit(const Params& P, bf16* __restrict__
   }
 }
 
+#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
 __global__ void __launch_bounds__(kCombineCols * kCombineSlots)
 k_combine(const Params P, bf16* __restrict__ out, int T, int n_parts) {
   __shared__ float2 s_y[kMaxK + 8][kCombineCols];       // affinity-weighted y per slot (k + S <= 40)
@@ -1803,5 +1829,6 @@ k_combine(const Params P, bf16* __restrict__ out, int T, int n_parts) {
   pdl_launch();
   combine_unit(P, out, T, n_parts, blockIdx.x, s_y);
 }
+#endif
 
 }  // namespace

@@ -540,8 +540,17 @@ constexpr int kCfThreads = 256;
 // 24.4 us with two blocks per SM, 23.8 us with one).
 constexpr size_t kCfAloneBytes = 120 * 1024;
 
-__global__ void __launch_bounds__(kCfThreads)
-k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr) {
+template <bool LEAN>
+__device__ __forceinline__ void combine_fused_body(const Params& P_in, bf16* __restrict__ out, int T_in, int n_sl_in, int lr_in) {
+#ifdef MOE_VQLR_JIT
+  constexpr int T = 1, n_sl = J_NSL, lr = J_LR;
+  Params P = P_in;
+  MOE_VQLR_JIT_PARAMS(P);
+  (void)T_in; (void)n_sl_in; (void)lr_in;
+#else
+  const int T = LEAN ? 1 : T_in, n_sl = n_sl_in, lr = lr_in;
+  const Params& P = P_in;
+#endif
   extern __shared__ float s_cf[];
   const int n_slots = P.k + P.S, H2 = P.H / 2, n_pos = T * n_slots, r = P.r;
   float* s_zd = s_cf;                                                        // [n_slots][r]
@@ -693,5 +702,12 @@ k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr)
   }
   TRACE_STAMP(2, 10);
 }
+
+#ifndef MOE_VQLR_JIT
+__global__ void __launch_bounds__(kCfThreads)
+k_combine_fused(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr) {
+  combine_fused_body<false>(P, out, T, n_sl, lr);
+}
+#endif
 
 }  // namespace

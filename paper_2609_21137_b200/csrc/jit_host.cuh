@@ -98,10 +98,16 @@ void nvrtc_open() {
 const char kJitSource[] =
     "#define MOE_VQLR_JIT 1\n"
     "#include \"fused_kernel.cuh\"\n"
+    "extern \"C\" __global__ void __launch_bounds__(32 * kRouterWarps)\n"
+    "k_router_z_jit(const Params P, const bf16* __restrict__ x, int T) { router_z_pdl_body<true>(P, x, T); }\n"
     "extern \"C\" __global__ void __launch_bounds__(kFusedThreads, 1)\n"
     "k_expert_fused_jit(const Params P, const bf16* __restrict__ x, int T, const StagePlan pg, const FusedPlan fp,\n"
     "                   int n_books, int want_dbg, const J_IDXT* __restrict__ idx_dp) {\n"
     "  expert_fused_body<J_IDXT, J_DENSE, J_JD, J_D4, J_SP, true>(P, x, T, pg, fp, n_books, want_dbg, idx_dp);\n"
+    "}\n"
+    "extern \"C\" __global__ void __launch_bounds__(kCfThreads)\n"
+    "k_combine_fused_jit(const Params P, bf16* __restrict__ out, int T, int n_sl, int lr) {\n"
+    "  combine_fused_body<true>(P, out, T, n_sl, lr);\n"
     "}\n";
 
 // NVRTC has no host headers; the public header asks for <stdint.h>.

@@ -70,6 +70,8 @@ struct moe_vqlr_handle {
   int pcb_Q;                // table pieces per token = ceil(H / 8 / 64)
   size_t smem_lr;           // dynamic shared memory of k_gateup_lr
   const void* jit_fused;     // k_expert_fused compiled at create() for this layer's shape (single-token calls), or NULL
+  const void* jit_router;    // ... and the kernels before and after it
+  const void* jit_combine;
   std::string jit_note;      // why there is none
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
@@ -306,7 +308,13 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         if (z_by_mma)
           le = launch_pdl(k_router_zmma_pdl, zmma_blocks(P) + (P.E * ((T + kTokGroup - 1) / kTokGroup) + kZmmaWarps - 1) / kZmmaWarps,
                           32 * kZmmaWarps, 0, st, P, xb, T);
-        else
+        else if (h->jit_router && T == 1) {
+          Params Pa = P;
+          const bf16* xa = xb;
+          int Ta = T;
+          void* args[] = {&Pa, &xa, &Ta};
+          le = launch_pdl_ptr(h->jit_router, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps, 32 * kRouterWarps, 0, st, args);
+        } else
           le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
                           32 * kRouterWarps, 0, st, P, xb, T);
         ran = true;
@@ -334,7 +342,14 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         const int lr = (!h->dn_dense && P.r > 0) ? 1 : 0;
         size_t smem = ((lr ? (size_t)(P.k + P.S) * P.r : 0) + (size_t)(P.k + P.S) * kCfCols * 2) * sizeof(float);
         if (smem < kCfAloneBytes && T == 1) smem = kCfAloneBytes;      // one block per SM (see kCfAloneBytes)
-        le = launch_pdl(k_combine_fused, T * (P.H / 2 / kCfCols), kCfThreads, smem, st, P, ob, T, h->fplan.n_sl, lr);
+        if (h->jit_combine && T == 1) {
+          Params Pa = P;
+          bf16* oa = ob;
+          int Ta = T, nsl_a = h->fplan.n_sl, lr_a = lr;
+          void* args[] = {&Pa, &oa, &Ta, &nsl_a, &lr_a};
+          le = launch_pdl_ptr(h->jit_combine, T * (P.H / 2 / kCfCols), kCfThreads, smem, st, args);
+        } else
+          le = launch_pdl(k_combine_fused, T * (P.H / 2 / kCfCols), kCfThreads, smem, st, P, ob, T, h->fplan.n_sl, lr);
         ran = true;
         break;
       }
@@ -821,7 +836,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
 
   // The single-token path compiled for this layer's shape (see jit_host.cuh).
   const bool want_clk = (cfg->flags & MOE_VQLR_FLAG_PHASE_CLOCKS) != 0;
-  h->jit_fused = nullptr;
+  h->jit_fused = h->jit_router = h->jit_combine = nullptr;
   if (cfg->flags & MOE_VQLR_FLAG_NO_SPECIALIZE) h->jit_note = "switched off by MOE_VQLR_FLAG_NO_SPECIALIZE";
   else if (!h->fused || h->fused_dg[1] == 0) h->jit_note = "single-token calls of this configuration do not run the fused kernel";
   else if ((k + S) * h->fplan.n_sl > h->sm_count) h->jit_note = "a single token's work items exceed one wave";
@@ -838,6 +853,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
     def("J_REPL", pg.repl); def("J_XSMEM", h->fused_xs[1]);
     def("J_TPS", fp.tps); def("J_NSL", fp.n_sl); def("J_TLAST", fp.t_last); def("J_JD", fp.jd); def("J_RP_LOG2", fp.rp_log2);
     def("J_DEPTH_G", h->fused_dg[1]); def("J_DEPTH_D", h->fused_dd[1]);
+    def("J_LR", (!h->dn_dense && r > 0) ? 1 : 0);
     defs.push_back(std::string("-DJ_IDXT=") + ((h->d4 || h->idx_bytes == 2) ? "uint16_t" : "uint8_t"));
     defs.push_back(std::string("-DJ_DENSE=") + (h->dn_dense ? "true" : "false"));
     defs.push_back(std::string("-DJ_D4=") + (h->d4 ? "true" : "false"));
@@ -851,10 +867,23 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
       StagePlan pg1 = pg;
       pg1.x_smem = h->fused_xs[1];
       const size_t smem1 = fused_layout(K, h->n_books, 1, H, r, pg1, fp1, h->dn_dense, h->idx_tc, E, k, S).total;
+      cudaKernel_t kern_r = nullptr, kern_c = nullptr;
+      size_t cf_smem = ((size_t)(k + S) * (r > 0 ? r : 0) + (size_t)(k + S) * kCfCols * 2) * sizeof(float);
+      if (cf_smem < kCfAloneBytes) cf_smem = kCfAloneBytes;
       cudaError_t je = cudaLibraryGetKernel(&kern, lib, "k_expert_fused_jit");
+      if (je == cudaSuccess) je = cudaLibraryGetKernel(&kern_r, lib, "k_router_z_jit");
+      if (je == cudaSuccess) je = cudaLibraryGetKernel(&kern_c, lib, "k_combine_fused_jit");
       if (je == cudaSuccess) je = raise_dyn_smem((const void*)kern, smem1);
-      if (je == cudaSuccess) { h->jit_fused = (const void*)kern; h->jit_note.clear(); }
-      else { h->jit_note = std::string("loading the compiled kernel: ") + cudaGetErrorString(je); cudaGetLastError(); }
+      if (je == cudaSuccess) je = raise_dyn_smem((const void*)kern_c, cf_smem);
+      if (je == cudaSuccess) {
+        h->jit_fused = (const void*)kern;
+        h->jit_router = (const void*)kern_r;
+        h->jit_combine = (const void*)kern_c;
+        h->jit_note.clear();
+      } else {
+        h->jit_note = std::string("loading the compiled kernels: ") + cudaGetErrorString(je);
+        cudaGetLastError();
+      }
     }
   }
 
@@ -1106,7 +1135,9 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
   return take_status(h);
 }
 
-int moe_vqlr_specialized(const moe_vqlr_handle* h) { return (h && h->jit_fused) ? 1 : 0; }
+int moe_vqlr_specialized(const moe_vqlr_handle* h) {
+  return h ? (h->jit_router ? 1 : 0) + (h->jit_fused ? 1 : 0) + (h->jit_combine ? 1 : 0) : 0;
+}
 
 const char* moe_vqlr_specialization_note(const moe_vqlr_handle* h) { return h ? h->jit_note.c_str() : ""; }
 
