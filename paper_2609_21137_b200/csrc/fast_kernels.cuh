@@ -232,6 +232,22 @@ struct StagePlan {
   FastDiv d_per_grp, d_per_chunk, d_chunk, d_tail, d_W;   // n_parts*tiles, n_parts*chunk, chunk, tail, W
 };
 
+#ifdef MOE_VQLR_JIT
+// Run-time-compiled copies (jit_host.cuh): the integers of a work plan as constants, X = GU or DN.
+#define MOE_VQLR_JIT_PLAN(pl, X)                                                                          \
+  do {                                                                                                    \
+    (pl).nb = J_##X##_NB; (pl).n_slices = J_##X##_NSLICES; (pl).n_lr = J_##X##_NLR;                       \
+    (pl).n_parts = J_##X##_NPARTS; (pl).tiles = J_##X##_TILES; (pl).depth = J_##X##_DEPTH;                \
+    (pl).chunk = J_##X##_CHUNK; (pl).x_smem = J_##X##_XSMEM; (pl).repl = J_##X##_REPL; (pl).W = J_##X##_W; \
+    (pl).only_grp = -1; (pl).tpu = J_##X##_TPU; (pl).tail = J_##X##_TAIL;                                 \
+    (pl).d_per_grp = make_fastdiv((unsigned int)(J_##X##_NPARTS * J_##X##_TILES));                        \
+    (pl).d_per_chunk = make_fastdiv((unsigned int)(J_##X##_NPARTS * J_##X##_CHUNK));                      \
+    (pl).d_chunk = make_fastdiv((unsigned int)J_##X##_CHUNK);                                             \
+    (pl).d_tail = make_fastdiv((unsigned int)(J_##X##_TAIL > 0 ? J_##X##_TAIL : 1));                      \
+    (pl).d_W = make_fastdiv((unsigned int)J_##X##_W);                                                     \
+  } while (0)
+#endif
+
 // Position in the flattened work list of a stage.  Units are ordered (group, chunk of `chunk`
 // row tiles, part, tile inside the chunk): a warp's contiguous range then mixes cheap low-rank
 // parts with lookup-heavy slice parts instead of drawing only one kind, while consecutive tiles
@@ -830,8 +846,13 @@ constexpr int kZmmaWarps = 8;
 
 __host__ __device__ __forceinline__ int zmma_blocks(const Params& P) { return P.n_zrows / 8 * P.z_repeat; }
 
-#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
-__global__ void __launch_bounds__(32 * kZmmaWarps) k_router_zmma_pdl(const Params P, const bf16* __restrict__ x, int T) {
+__device__ __forceinline__ void router_zmma_pdl_body(const Params& P_in, const bf16* __restrict__ x, int T) {
+#ifdef MOE_VQLR_JIT
+  Params P = P_in;
+  MOE_VQLR_JIT_PARAMS(P);
+#else
+  const Params& P = P_in;
+#endif
   __shared__ float s_red[kZmmaWarps][128];
   pdl_wait();      // the previous call's kernels may still read logits / z
   pdl_launch();
@@ -877,6 +898,11 @@ __global__ void __launch_bounds__(32 * kZmmaWarps) k_router_zmma_pdl(const Param
     const int tok = (l2 >> 2) + ((i & 2) ? 8 : 0), row = 2 * (l2 & 3) + (i & 1);
     if (tok < T) P.z[((size_t)tok * 2 + slot) * P.r + rho0 + row] = sum;
   }
+}
+
+#ifndef MOE_VQLR_JIT
+__global__ void __launch_bounds__(32 * kZmmaWarps) k_router_zmma_pdl(const Params P, const bf16* __restrict__ x, int T) {
+  router_zmma_pdl_body(P, x, T);
 }
 #endif
 
@@ -1277,9 +1303,21 @@ __device__ __forceinline__ void gu_tiles_run(const Params& P, const bf16* __rest
   TRACE_STAMP(0, 15);
 }
 
-template <typename IdxT, bool DENSE, bool D4 = false, int LRF = 0, bool SP = false>
-__global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
-k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {
+template <typename IdxT, bool DENSE, bool D4, int LRF, bool SP>
+__device__ __forceinline__ void gateup_mma_body(const Params& P_in, const bf16* __restrict__ x, int T, const StagePlan& pl_in,
+                                                int n_books_in, int want_dbg) {
+#ifdef MOE_VQLR_JIT_CHAIN      // the chain compiled for one layer shape: see jit_host.cuh
+  Params P = P_in;
+  MOE_VQLR_JIT_PARAMS(P);
+  StagePlan pl = pl_in;
+  MOE_VQLR_JIT_PLAN(pl, GU);
+  constexpr int n_books = J_NBOOKS;
+  (void)n_books_in;
+#else
+  const Params& P = P_in;
+  const StagePlan& pl = pl_in;
+  const int n_books = n_books_in;
+#endif
   extern __shared__ uint4 s_u4[];
   const int nwarps = blockDim.x >> 5, warp = threadIdx.x >> 5;
   const GuLayout L = gu_layout(P.K, n_books, T, P.H, P.r, pl, nwarps, P.E, P.k, P.S);
@@ -1296,6 +1334,12 @@ k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan 
   pdl_launch();
   TRACE_STAMP(0, 3);
   gu_tiles_run<IdxT, DENSE, D4, LRF, SP>(P, x, T, pl, m, w);
+}
+
+template <typename IdxT, bool DENSE, bool D4 = false, int LRF = 0, bool SP = false>
+__global__ void __launch_bounds__(DENSE ? kDenseThreads : kFastThreads, 1)
+k_gateup_mma(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {
+  gateup_mma_body<IdxT, DENSE, D4, LRF, SP>(P, x, T, pl, n_books, want_dbg);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1378,12 +1422,22 @@ __device__ __forceinline__ void act_zdown_unit(const Params& P, int n_pos, int n
   }
 }
 
-#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
-__global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n_pos, int n_parts, int with_zd, int zsplit) {
+__device__ __forceinline__ void act_zdown_body(const Params& P_in, int n_pos, int n_parts, int with_zd, int zsplit) {
+#ifdef MOE_VQLR_JIT
+  Params P = P_in;
+  MOE_VQLR_JIT_PARAMS(P);
+#else
+  const Params& P = P_in;
+#endif
   extern __shared__ float s_p[];                 // [I]
   pdl_launch();                                  // the down kernel may stage its code book meanwhile
   pdl_wait();
   act_zdown_unit(P, n_pos, n_parts, with_zd, zsplit, blockIdx.x, s_p);
+}
+
+#ifndef MOE_VQLR_JIT
+__global__ void __launch_bounds__(kActThreads) k_act_zdown(const Params P, int n_pos, int n_parts, int with_zd, int zsplit) {
+  act_zdown_body(P, n_pos, n_parts, with_zd, zsplit);
 }
 #endif
 
@@ -1700,9 +1754,17 @@ __device__ __forceinline__ void dn_tiles_run(const Params& P, int T, const Stage
   TRACE_STAMP(2, 15);
 }
 
-template <typename IdxT, bool DENSE, bool D4 = false, int TPU = 2, bool SP = false>
-__global__ void __launch_bounds__(kDownThreads, 1)
-k_down_mma(const Params P, int T, const StagePlan pl) {
+template <typename IdxT, bool DENSE, bool D4, int TPU, bool SP>
+__device__ __forceinline__ void down_mma_body(const Params& P_in, int T, const StagePlan& pl_in) {
+#ifdef MOE_VQLR_JIT_CHAIN
+  Params P = P_in;
+  MOE_VQLR_JIT_PARAMS(P);
+  StagePlan pl = pl_in;
+  MOE_VQLR_JIT_PLAN(pl, DN);
+#else
+  const Params& P = P_in;
+  const StagePlan& pl = pl_in;
+#endif
   extern __shared__ uint4 s_u4[];
   char* s_base = reinterpret_cast<char*>(s_u4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1749,6 +1811,12 @@ k_down_mma(const Params P, int T, const StagePlan pl) {
   }
   TRACE_STAMP(2, 2);
   dn_tiles_run<IdxT, DENSE, D4, TPU, SP>(P, T, pl, m, w);
+}
+
+template <typename IdxT, bool DENSE, bool D4 = false, int TPU = 2, bool SP = false>
+__global__ void __launch_bounds__(kDownThreads, 1)
+k_down_mma(const Params P, int T, const StagePlan pl) {
+  down_mma_body<IdxT, DENSE, D4, TPU, SP>(P, T, pl);
 }
 
 // out[t][h] = sum over slots (in slot order) of affinity * y[t][slot][h], where y is the sum of
@@ -1821,13 +1889,23 @@ __device__ __forceinline__ void combine_unit(const Params& P, bf16* __restrict__
   }
 }
 
-#ifndef MOE_VQLR_JIT      // not part of the single-token path that is compiled per shape
-__global__ void __launch_bounds__(kCombineCols * kCombineSlots)
-k_combine(const Params P, bf16* __restrict__ out, int T, int n_parts) {
+__device__ __forceinline__ void combine_body(const Params& P_in, bf16* __restrict__ out, int T, int n_parts) {
+#ifdef MOE_VQLR_JIT
+  Params P = P_in;
+  MOE_VQLR_JIT_PARAMS(P);
+#else
+  const Params& P = P_in;
+#endif
   __shared__ float2 s_y[kMaxK + 8][kCombineCols];       // affinity-weighted y per slot (k + S <= 40)
   pdl_wait();
   pdl_launch();
   combine_unit(P, out, T, n_parts, blockIdx.x, s_y);
+}
+
+#ifndef MOE_VQLR_JIT
+__global__ void __launch_bounds__(kCombineCols * kCombineSlots)
+k_combine(const Params P, bf16* __restrict__ out, int T, int n_parts) {
+  combine_body(P, out, T, n_parts);
 }
 #endif
 

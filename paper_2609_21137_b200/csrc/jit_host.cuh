@@ -19,6 +19,7 @@
 #include <nvrtc.h>      // types only: the library itself is opened at run time
 
 #include <cstdio>
+#include <cstdlib>
 #include <map>
 #include <mutex>
 #include <string>
@@ -110,15 +111,37 @@ const char kJitSource[] =
     "  combine_fused_body<true>(P, out, T, n_sl, lr);\n"
     "}\n";
 
+// The chain of kernels for calls of several tokens, compiled for one layer shape: the same constants
+// (the token count stays an argument), plus the two work plans of the gate/up and down kernels.
+// Only the three kernels that gain from it: the router and the activation kernel measured SLOWER as
+// per-shape copies at 4-16 tokens (router 4.4 -> 5.6 us, activation + z_d 5.6 -> 7.2 us on the Qwen3
+// shape at batch 16: with constant trip counts the compiler unrolls their loops into long straight-line
+// code, which is exactly what a kernel that runs once per call should not be).
+const char kJitChainSource[] =
+    "#define MOE_VQLR_JIT 1\n"
+    "#define MOE_VQLR_JIT_CHAIN 1\n"
+    "#include \"fast_kernels.cuh\"\n"
+    "extern \"C\" __global__ void __launch_bounds__(J_GU_DENSE ? kDenseThreads : kFastThreads, 1)\n"
+    "k_gateup_mma_jit(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {\n"
+    "  gateup_mma_body<J_GU_IDXT, J_GU_DENSE, J_GU_D4, J_LRF, J_SP>(P, x, T, pl, n_books, want_dbg);\n"
+    "}\n"
+    "extern \"C\" __global__ void __launch_bounds__(kDownThreads, 1)\n"
+    "k_down_mma_jit(const Params P, int T, const StagePlan pl) {\n"
+    "  down_mma_body<J_DN_IDXT, J_DN_DENSE, J_DN_D4, J_DN_TPUT, J_SP>(P, T, pl);\n"
+    "}\n"
+    "extern \"C\" __global__ void __launch_bounds__(kCombineCols * kCombineSlots)\n"
+    "k_combine_jit(const Params P, bf16* __restrict__ out, int T, int n_parts) { combine_body(P, out, T, n_parts); }\n";
+
 // NVRTC has no host headers; the public header asks for <stdint.h>.
 const char kJitStdint[] =
     "typedef signed char int8_t; typedef short int16_t; typedef int int32_t; typedef long long int64_t;\n"
     "typedef unsigned char uint8_t; typedef unsigned short uint16_t; typedef unsigned int uint32_t;\n"
     "typedef unsigned long long uint64_t;\n";
 
-// Compiles (or finds) the specialised kernels for `defs` on the current device.  Returns the loaded
+// Compiles (or finds) the specialised kernels of `source` (kJitSource or kJitChainSource) for `defs`
+// on the current device.  Returns the loaded
 // library or nullptr with *why set.
-cudaLibrary_t jit_library(const std::vector<std::string>& defs, std::string* why) {
+cudaLibrary_t jit_library(const char* source, const std::vector<std::string>& defs, std::string* why) {
   std::lock_guard<std::mutex> lock(g_jit_mu);
   nvrtc_open();
   NvrtcApi& a = g_nvrtc;
@@ -130,7 +153,25 @@ cudaLibrary_t jit_library(const std::vector<std::string>& defs, std::string* why
   snprintf(arch, sizeof arch, "--gpu-architecture=sm_%d%d%s", prop.major, prop.minor, prop.major >= 9 ? "a" : "");
   std::vector<std::string> opts = {arch, "-std=c++17", "-I" + a.src_dir, "-I" + a.api_include, "-I" + a.cuda_include};
   opts.insert(opts.end(), defs.begin(), defs.end());
-  std::string key = std::to_string(dev);
+#ifdef MOE_VQLR_JIT_EXTRA_ENV      // development builds only: extra options for A/B runs of kernel variants
+  if (const char* extra = getenv("MOE_VQLR_JIT_EXTRA")) {
+    std::string e(extra);
+    size_t at = 0;
+    while (at < e.size()) {
+      size_t sp = e.find(' ', at);
+      if (sp == std::string::npos) sp = e.size();
+      if (sp > at) opts.push_back(e.substr(at, sp - at));
+      at = sp + 1;
+    }
+  }
+#endif
+#ifdef MOE_VQLR_TRACE
+  opts.push_back("-DMOE_VQLR_TRACE");
+#ifdef MOE_VQLR_TRACE_GLOBAL
+  opts.push_back("-DMOE_VQLR_TRACE_GLOBAL");
+#endif
+#endif
+  std::string key = std::to_string(dev) + (source == kJitChainSource ? "|chain" : "|single");
   for (const std::string& o : opts) { key += '|'; key += o; }
   auto hit = g_jit_cache.find(key);
   if (hit != g_jit_cache.end()) {
@@ -142,7 +183,7 @@ cudaLibrary_t jit_library(const std::vector<std::string>& defs, std::string* why
   nvrtcProgram prog = nullptr;
   const char* hdr_names[] = {"stdint.h"};
   const char* hdr_src[] = {kJitStdint};
-  nvrtcResult r = a.create_program(&prog, kJitSource, "moe_vqlr_jit.cu", 1, hdr_src, hdr_names);
+  nvrtcResult r = a.create_program(&prog, source, "moe_vqlr_jit.cu", 1, hdr_src, hdr_names);
   if (r != NVRTC_SUCCESS) { *why = std::string("nvrtcCreateProgram: ") + a.error_string(r); return nullptr; }
   std::vector<const char*> argv;
   for (const std::string& o : opts) argv.push_back(o.c_str());

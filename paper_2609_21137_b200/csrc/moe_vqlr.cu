@@ -72,6 +72,8 @@ struct moe_vqlr_handle {
   const void* jit_fused;     // k_expert_fused compiled at create() for this layer's shape (single-token calls), or NULL
   const void* jit_router;    // ... and the kernels before and after it
   const void* jit_combine;
+  // the chain of kernels (calls of several tokens) compiled for this layer's shape, or NULL each
+  const void *jit_c_gateup, *jit_c_down, *jit_c_combine;      // (its router and activation kernels measured slower that way)
   std::string jit_note;      // why there is none
   void* idx_dp;              // down index map re-laid per slice (inside the workspace)
   void* workspace;
@@ -281,6 +283,22 @@ const void* fused_kernel(const moe_vqlr_handle* h, int jd) {
   return h->special ? fused_kernel_sp<true>(h->dn_dense, h->d4, h->idx_bytes, jd) : fused_kernel_sp<false>(h->dn_dense, h->d4, h->idx_bytes, jd);
 }
 
+// Head of both chains: for a single token the copy compiled for this layer's shape where there is
+// one, else the precompiled kernel.
+cudaError_t launch_router(const moe_vqlr_handle* h, const bf16* xb, int T, bool z_by_mma, cudaStream_t st) {
+  const Params& P = h->P;
+  Params Pa = P;
+  const bf16* xa = xb;
+  int Ta = T;
+  void* args[] = {&Pa, &xa, &Ta};
+  if (z_by_mma) {
+    return launch_pdl_ptr((const void*)k_router_zmma_pdl, zmma_blocks(P) + (P.E * ((T + kTokGroup - 1) / kTokGroup) + kZmmaWarps - 1) / kZmmaWarps,
+                          32 * kZmmaWarps, 0, st, args);
+  }
+  const void* fn = (T == 1 && h->jit_router) ? h->jit_router : (const void*)k_router_z_pdl;
+  return launch_pdl_ptr(fn, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps, 32 * kRouterWarps, 0, st, args);
+}
+
 // Enqueues the kernel of one stage (nothing for a stage this configuration does not have).
 cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, bf16* ob, cudaStream_t st, bool allow_coop) {
   const Params& P = h->P;
@@ -305,18 +323,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
     // one wave of (work group, slice) items at most: with more, the chain's finer parts balance better
     switch (stage) {
       case 0:
-        if (z_by_mma)
-          le = launch_pdl(k_router_zmma_pdl, zmma_blocks(P) + (P.E * ((T + kTokGroup - 1) / kTokGroup) + kZmmaWarps - 1) / kZmmaWarps,
-                          32 * kZmmaWarps, 0, st, P, xb, T);
-        else if (h->jit_router && T == 1) {
-          Params Pa = P;
-          const bf16* xa = xb;
-          int Ta = T;
-          void* args[] = {&Pa, &xa, &Ta};
-          le = launch_pdl_ptr(h->jit_router, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps, 32 * kRouterWarps, 0, st, args);
-        } else
-          le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
-                          32 * kRouterWarps, 0, st, P, xb, T);
+        le = launch_router(h, xb, T, z_by_mma, st);
         ran = true;
         break;
       case 2: {
@@ -358,12 +365,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
   } else if (h->fast) {
     switch (stage) {
       case 0:
-        if (z_by_mma)
-          le = launch_pdl(k_router_zmma_pdl, zmma_blocks(P) + (P.E * ((T + kTokGroup - 1) / kTokGroup) + kZmmaWarps - 1) / kZmmaWarps,
-                          32 * kZmmaWarps, 0, st, P, xb, T);
-        else
-          le = launch_pdl(k_router_z_pdl, (router_z_units_launched(P, T) + kRouterWarps - 1) / kRouterWarps,
-                          32 * kRouterWarps, 0, st, P, xb, T);
+        le = launch_router(h, xb, T, z_by_mma, st);
         ran = true;
         break;
       case 2: {
@@ -393,7 +395,8 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           const bf16* xa = xb;
           int Ta = T, nb_a = h->n_books, dbg_a = h->want_dbg;
           void* args[] = {&Pa, &xa, &Ta, &pl, &nb_a, &dbg_a};
-          le = launch_pdl_ptr(gateup_kernel(h), h->sm_count, h->gu_dense ? kDenseThreads : kFastThreads, smem, st, args);
+          const void* fn = (h->jit_c_gateup && !h->per_expert_launch) ? h->jit_c_gateup : gateup_kernel(h);
+          le = launch_pdl_ptr(fn, h->sm_count, h->gu_dense ? kDenseThreads : kFastThreads, smem, st, args);
         }
         h->launches += n_launch - 1;
         ran = true;
@@ -406,8 +409,10 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         if (P.I <= 4096) {                                // one fused block per pair (times zsplit)
           int zsplit = 1;
           if (with_zd) while (n_pos * zsplit * 2 <= 3 * h->sm_count && zsplit * 2 <= 8 && zsplit * 2 <= P.r) zsplit *= 2;
-          le = launch_pdl(k_act_zdown, n_pos * zsplit, kActThreads, (size_t)P.I * sizeof(float), st, P, n_pos,
-                          gu_parts, with_zd, zsplit);
+          Params Pa = P;
+          int np_a = n_pos, parts_a = gu_parts, zd_a = with_zd, zs_a = zsplit;
+          void* args[] = {&Pa, &np_a, &parts_a, &zd_a, &zs_a};
+          le = launch_pdl_ptr((const void*)k_act_zdown, n_pos * zsplit, kActThreads, (size_t)P.I * sizeof(float), st, args);
         } else {                                          // few pairs or a long intermediate: two wide kernels
           int grid = (n_pos * (P.I / 2) + 255) / 256;
           if (grid > 4 * h->sm_count) grid = 4 * h->sm_count;
@@ -433,7 +438,8 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           Params Pa = P;
           int Ta = T;
           void* args[] = {&Pa, &Ta, &pl};
-          le = launch_pdl_ptr(down_kernel(h, pl.tpu), h->sm_count, kDownThreads, h->smem_fast_dn, st, args);
+          const void* fn = (h->jit_c_down && !h->per_expert_launch) ? h->jit_c_down : down_kernel(h, pl.tpu);
+          le = launch_pdl_ptr(fn, h->sm_count, kDownThreads, h->smem_fast_dn, st, args);
         }
         h->launches += n_launch - 1;
         ran = true;
@@ -441,7 +447,11 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
       }
       case 5: {
         const int grid = T * ((P.H / 2 + kCombineCols - 1) / kCombineCols);
-        le = launch_pdl(k_combine, grid, kCombineCols * kCombineSlots, 0, st, P, ob, T, h->plan_dn.n_parts);
+        Params Pa = P;
+        bf16* oa = ob;
+        int Ta = T, parts_a = h->plan_dn.n_parts;
+        void* args[] = {&Pa, &oa, &Ta, &parts_a};
+        le = launch_pdl_ptr(h->jit_c_combine ? h->jit_c_combine : (const void*)k_combine, grid, kCombineCols * kCombineSlots, 0, st, args);
         ran = true;
         break;
       }
@@ -834,31 +844,41 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
     }
   }
 
-  // The single-token path compiled for this layer's shape (see jit_host.cuh).
+  // The single-token path and the chain of kernels compiled for this layer's shape (see jit_host.cuh).
   const bool want_clk = (cfg->flags & MOE_VQLR_FLAG_PHASE_CLOCKS) != 0;
   h->jit_fused = h->jit_router = h->jit_combine = nullptr;
-  if (cfg->flags & MOE_VQLR_FLAG_NO_SPECIALIZE) h->jit_note = "switched off by MOE_VQLR_FLAG_NO_SPECIALIZE";
-  else if (!h->fused || h->fused_dg[1] == 0) h->jit_note = "single-token calls of this configuration do not run the fused kernel";
-  else if ((k + S) * h->fplan.n_sl > h->sm_count) h->jit_note = "a single token's work items exceed one wave";
-  else if (want_clk) h->jit_note = "phase clocks are recorded by the generic kernels";
-  else {
-    const FusedPlan& fp = h->fplan;
-    const StagePlan& pg = h->plan_gu_fused;
-    std::vector<std::string> defs;
-    auto def = [&](const char* name, long long v) { defs.push_back(std::string("-D") + name + "=" + std::to_string(v)); };
+  h->jit_c_gateup = h->jit_c_down = h->jit_c_combine = nullptr;
+  std::vector<std::string> base_defs;        // the integers of the parameter block
+  {
+    auto def = [&](const char* name, long long v) { base_defs.push_back(std::string("-D") + name + "=" + std::to_string(v)); };
     def("J_H", H); def("J_I", I); def("J_E", E); def("J_TOPK", k); def("J_S", S); def("J_K", K); def("J_R", r);
     def("J_RENORM", P.renorm); def("J_ACT", P.act); def("J_D", P.d); def("J_IDX12", P.idx12); def("J_ZREPEAT", P.z_repeat);
     def("J_NZROWS", P.n_zrows); def("J_ZSLOT_G", P.gate.zslot); def("J_ZSLOT_U", P.up.zslot);
-    def("J_NBOOKS", h->n_books); def("J_NB", pg.nb); def("J_NSLICES", pg.n_slices); def("J_NLR", pg.n_lr); def("J_NPARTS", pg.n_parts);
+    def("J_NBOOKS", h->n_books);
+    def("J_LR", (!h->dn_dense && r > 0) ? 1 : 0);
+    base_defs.push_back(std::string("-DJ_SP=") + (h->special ? "true" : "false"));
+  }
+  bool want_single = false;
+  if (cfg->flags & MOE_VQLR_FLAG_NO_SPECIALIZE) h->jit_note = "switched off by MOE_VQLR_FLAG_NO_SPECIALIZE";
+  else if (!h->fused || h->fused_dg[1] == 0) h->jit_note = "single-token calls of this configuration do not run the fused kernel";
+  else if ((k + S) * h->fplan.n_sl > h->sm_count) h->jit_note = "a single token's work items exceed one wave";
+#ifndef MOE_VQLR_TRACE
+  else if (want_clk) h->jit_note = "phase clocks are recorded by the generic kernels";
+#endif
+  else want_single = true;
+  if (want_single) {
+    const FusedPlan& fp = h->fplan;
+    const StagePlan& pg = h->plan_gu_fused;
+    std::vector<std::string> defs = base_defs;
+    auto def = [&](const char* name, long long v) { defs.push_back(std::string("-D") + name + "=" + std::to_string(v)); };
+    def("J_NB", pg.nb); def("J_NSLICES", pg.n_slices); def("J_NLR", pg.n_lr); def("J_NPARTS", pg.n_parts);
     def("J_REPL", pg.repl); def("J_XSMEM", h->fused_xs[1]);
     def("J_TPS", fp.tps); def("J_NSL", fp.n_sl); def("J_TLAST", fp.t_last); def("J_JD", fp.jd); def("J_RP_LOG2", fp.rp_log2);
     def("J_DEPTH_G", h->fused_dg[1]); def("J_DEPTH_D", h->fused_dd[1]);
-    def("J_LR", (!h->dn_dense && r > 0) ? 1 : 0);
     defs.push_back(std::string("-DJ_IDXT=") + ((h->d4 || h->idx_bytes == 2) ? "uint16_t" : "uint8_t"));
     defs.push_back(std::string("-DJ_DENSE=") + (h->dn_dense ? "true" : "false"));
     defs.push_back(std::string("-DJ_D4=") + (h->d4 ? "true" : "false"));
-    defs.push_back(std::string("-DJ_SP=") + (h->special ? "true" : "false"));
-    cudaLibrary_t lib = jit_library(defs, &h->jit_note);
+    cudaLibrary_t lib = jit_library(kJitSource, defs, &h->jit_note);
     if (lib) {
       cudaKernel_t kern = nullptr;
       FusedPlan fp1 = fp;
@@ -884,6 +904,49 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
         h->jit_note = std::string("loading the compiled kernels: ") + cudaGetErrorString(je);
         cudaGetLastError();
       }
+    }
+  }
+  // The chain, for the calls that run it: several tokens, or every call where the fused kernel is not used.
+  const bool chain_runs = h->fast && (maxT > 1 || !h->jit_fused);
+  if (chain_runs && !(cfg->flags & MOE_VQLR_FLAG_NO_SPECIALIZE) && !h->per_expert_launch && !h->pcb && !want_clk) {
+    std::vector<std::string> defs = base_defs;
+    auto def = [&](const std::string& name, long long v) { defs.push_back("-D" + name + "=" + std::to_string(v)); };
+    auto def_plan = [&](const std::string& x, const StagePlan& pl) {
+      def("J_" + x + "_NB", pl.nb); def("J_" + x + "_NSLICES", pl.n_slices); def("J_" + x + "_NLR", pl.n_lr);
+      def("J_" + x + "_NPARTS", pl.n_parts); def("J_" + x + "_TILES", pl.tiles); def("J_" + x + "_DEPTH", pl.depth);
+      def("J_" + x + "_CHUNK", pl.chunk); def("J_" + x + "_XSMEM", pl.x_smem); def("J_" + x + "_REPL", pl.repl);
+      def("J_" + x + "_W", pl.W); def("J_" + x + "_TPU", pl.tpu); def("J_" + x + "_TAIL", pl.tail);
+    };
+    def_plan("GU", h->plan_gu);
+    def_plan("DN", h->plan_dn);
+    const bool gu_d4 = !h->gu_dense && h->d4, dn_d4 = !h->dn_dense && h->d4;
+    defs.push_back(std::string("-DJ_GU_IDXT=") + ((h->gu_dense || h->d4 || h->idx_bytes == 2) ? "uint16_t" : "uint8_t"));
+    defs.push_back(std::string("-DJ_DN_IDXT=") + ((h->dn_dense || h->d4 || h->idx_bytes == 2) ? "uint16_t" : "uint8_t"));
+    defs.push_back(std::string("-DJ_GU_DENSE=") + (h->gu_dense ? "true" : "false"));
+    defs.push_back(std::string("-DJ_DN_DENSE=") + (h->dn_dense ? "true" : "false"));
+    defs.push_back(std::string("-DJ_GU_D4=") + (gu_d4 ? "true" : "false"));
+    defs.push_back(std::string("-DJ_DN_D4=") + (dn_d4 ? "true" : "false"));
+    def("J_LRF", h->gu_dense ? 0 : h->lrf2 ? 2 : h->lrf ? 1 : 0);
+    def("J_DN_TPUT", (!h->dn_dense && h->plan_dn.tpu == 4) ? 4 : 2);
+    std::string why;
+    cudaLibrary_t lib = jit_library(kJitChainSource, defs, &why);
+    if (lib) {
+      cudaKernel_t kg = nullptr, kd = nullptr, kc = nullptr;
+      cudaError_t je = cudaLibraryGetKernel(&kg, lib, "k_gateup_mma_jit");
+      if (je == cudaSuccess) je = cudaLibraryGetKernel(&kd, lib, "k_down_mma_jit");
+      if (je == cudaSuccess) je = cudaLibraryGetKernel(&kc, lib, "k_combine_jit");
+      const int gu_warps2 = (h->gu_dense ? kDenseThreads : kFastThreads) / 32;
+      if (je == cudaSuccess) je = raise_dyn_smem((const void*)kg, gu_layout(K, h->n_books, maxT, H, r, h->plan_gu, gu_warps2, E, k, S).total);
+      if (je == cudaSuccess) je = raise_dyn_smem((const void*)kd, h->smem_fast_dn);
+      if (je == cudaSuccess) {
+        h->jit_c_gateup = (const void*)kg; h->jit_c_down = (const void*)kd; h->jit_c_combine = (const void*)kc;
+        if (!want_single) h->jit_note.clear();
+      } else {
+        cudaGetLastError();
+        if (h->jit_note.empty()) h->jit_note = std::string("loading the compiled chain: ") + cudaGetErrorString(je);
+      }
+    } else if (h->jit_note.empty() || !want_single) {
+      h->jit_note = "chain: " + why;
     }
   }
 
@@ -1136,7 +1199,11 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
 }
 
 int moe_vqlr_specialized(const moe_vqlr_handle* h) {
-  return h ? (h->jit_router ? 1 : 0) + (h->jit_fused ? 1 : 0) + (h->jit_combine ? 1 : 0) : 0;
+  if (!h) return 0;
+  const void* all[] = {h->jit_router, h->jit_fused, h->jit_combine, h->jit_c_gateup, h->jit_c_down, h->jit_c_combine};
+  int n = 0;
+  for (const void* k : all) n += k ? 1 : 0;
+  return n;
 }
 
 const char* moe_vqlr_specialization_note(const moe_vqlr_handle* h) { return h ? h->jit_note.c_str() : ""; }
