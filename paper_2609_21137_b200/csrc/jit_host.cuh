@@ -8,7 +8,8 @@
 // The paper's system also compiles one mapping per model (Section 4); this is that step on a GPU.
 //
 // The copy is the SAME source (fused_kernel.cuh and what it includes, read from the directory this
-// library was loaded from) given to NVRTC with -DMOE_VQLR_JIT and one -DJ_* per constant, the
+// library was loaded from; a static_assert on the sizes of the argument structures refuses files
+// that no longer match the library) given to NVRTC with -DMOE_VQLR_JIT and one -DJ_* per constant, the
 // result loaded through the runtime's library API and launched like any other kernel.  NVRTC is
 // opened with dlopen at the first create() that wants it; without it, or when anything on the way
 // fails, the handle keeps the generic kernels (moe_vqlr_specialized() tells which, the reason is
@@ -99,6 +100,8 @@ void nvrtc_open() {
 const char kJitSource[] =
     "#define MOE_VQLR_JIT 1\n"
     "#include \"fused_kernel.cuh\"\n"
+    "static_assert(sizeof(Params) == J_SZ_PARAMS && sizeof(StagePlan) == J_SZ_PLAN && sizeof(FusedPlan) == J_SZ_FPLAN,\n"
+    "              \"the kernel sources beside the library are not the ones it was built from\");\n"
     "extern \"C\" __global__ void __launch_bounds__(32 * kRouterWarps)\n"
     "k_router_z_jit(const Params P, const bf16* __restrict__ x, int T) { router_z_pdl_body<true>(P, x, T); }\n"
     "extern \"C\" __global__ void __launch_bounds__(kFusedThreads, 1)\n"
@@ -121,6 +124,8 @@ const char kJitChainSource[] =
     "#define MOE_VQLR_JIT 1\n"
     "#define MOE_VQLR_JIT_CHAIN 1\n"
     "#include \"fast_kernels.cuh\"\n"
+    "static_assert(sizeof(Params) == J_SZ_PARAMS && sizeof(StagePlan) == J_SZ_PLAN,\n"
+    "              \"the kernel sources beside the library are not the ones it was built from\");\n"
     "extern \"C\" __global__ void __launch_bounds__(J_GU_DENSE ? kDenseThreads : kFastThreads, 1)\n"
     "k_gateup_mma_jit(const Params P, const bf16* __restrict__ x, int T, const StagePlan pl, int n_books, int want_dbg) {\n"
     "  gateup_mma_body<J_GU_IDXT, J_GU_DENSE, J_GU_D4, J_LRF, J_SP>(P, x, T, pl, n_books, want_dbg);\n"

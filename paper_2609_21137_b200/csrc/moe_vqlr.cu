@@ -857,6 +857,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
     def("J_NBOOKS", h->n_books);
     def("J_LR", (!h->dn_dense && r > 0) ? 1 : 0);
     base_defs.push_back(std::string("-DJ_SP=") + (h->special ? "true" : "false"));
+    def("J_SZ_PARAMS", (long long)sizeof(Params)); def("J_SZ_PLAN", (long long)sizeof(StagePlan)); def("J_SZ_FPLAN", (long long)sizeof(FusedPlan));
   }
   bool want_single = false;
   if (cfg->flags & MOE_VQLR_FLAG_NO_SPECIALIZE) h->jit_note = "switched off by MOE_VQLR_FLAG_NO_SPECIALIZE";
@@ -908,7 +909,12 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
   }
   // The chain, for the calls that run it: several tokens, or every call where the fused kernel is not used.
   const bool chain_runs = h->fast && (maxT > 1 || !h->jit_fused);
-  if (chain_runs && !(cfg->flags & MOE_VQLR_FLAG_NO_SPECIALIZE) && !h->per_expert_launch && !h->pcb && !want_clk) {
+#ifdef MOE_VQLR_TRACE      // a tracing build compiles the phase stamps into the per-shape copies as well
+  const bool clk_ok = true;
+#else
+  const bool clk_ok = !want_clk;
+#endif
+  if (chain_runs && !(cfg->flags & MOE_VQLR_FLAG_NO_SPECIALIZE) && !h->per_expert_launch && !h->pcb && clk_ok) {
     std::vector<std::string> defs = base_defs;
     auto def = [&](const std::string& name, long long v) { defs.push_back("-D" + name + "=" + std::to_string(v)); };
     auto def_plan = [&](const std::string& x, const StagePlan& pl) {
