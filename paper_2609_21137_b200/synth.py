@@ -58,6 +58,10 @@ SHAPES: Dict[str, LayerShape] = {
     "qwen3": LayerShape("qwen3", H=2048, I=768, E=128, k=8, d=8, K=4096, r=64, T=1),
     "qwen3_b16": LayerShape("qwen3_b16", H=2048, I=768, E=128, k=8, d=8, K=4096, r=64, T=16,
                             router_bias=True),
+    # the batch sizes between the two headline points (Section 5.6's batch axis)
+    "qwen3_b2": LayerShape("qwen3_b2", H=2048, I=768, E=128, k=8, d=8, K=4096, r=64, T=2),
+    "qwen3_b4": LayerShape("qwen3_b4", H=2048, I=768, E=128, k=8, d=8, K=4096, r=64, T=4),
+    "qwen3_b8": LayerShape("qwen3_b8", H=2048, I=768, E=128, k=8, d=8, K=4096, r=64, T=8),
     "dsv2lite": LayerShape("dsv2lite", H=2048, I=1408, E=64, k=6, S=2, d=8, K=256, r=32, T=1),
     "dsv2lite_b8": LayerShape("dsv2lite_b8", H=2048, I=1408, E=64, k=6, S=2, d=8, K=256, r=32,
                               T=8),
