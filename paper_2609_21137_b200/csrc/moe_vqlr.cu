@@ -86,6 +86,7 @@ struct moe_vqlr_handle {
   cudaGraphExec_t io_graph[kMaxT + 1];     // the same with both host copies inside, for the host buffers below
   const void* io_x[kMaxT + 1];
   void* io_out[kMaxT + 1];
+  bool io_stage_in[kMaxT + 1];             // ... whose tokens come in through k_stage_in (one more kernel per call)
   bool io_graph_failed;                    // host buffers that cannot be captured (pageable): copies stay outside
   int host_graph_launches;                 // kernels in one such graph
   int64_t launches;
@@ -125,6 +126,16 @@ cudaError_t raise_dyn_smem(const void* fn, size_t bytes) {
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Tokens from the caller's pinned host buffer into the staging buffer, 16 bytes per thread: as a
+// kernel of the programmatic-launch chain it costs less than a copy node of the graph, and the
+// router's weight rows (requested before its dependency wait) travel meanwhile.
+__global__ void __launch_bounds__(256) k_stage_in(const uint4* __restrict__ src_host, uint4* __restrict__ dst, int n16) {
+  pdl_wait();        // the previous call's kernels may still read the staging buffer
+  pdl_launch();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n16) dst[i] = src_host[i];
+}
 
 
 template <typename... KArgs, typename... Args>
@@ -1162,9 +1173,20 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
       cudaError_t ge = pinned ? cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal) : cudaErrorNotSupported;
       if (ge == cudaSuccess) {
         const int64_t before = h->launches;
-        cudaError_t c1 = cudaMemcpyAsync(h->x_stage, x_host, bytes, cudaMemcpyHostToDevice, h->cap_stream);
-        const int rc = c1 == cudaSuccess ? moe_vqlr_decode_layer(h, h->x_stage, T, h->out_stage, nullptr, h->cap_stream) : MOE_VQLR_ERR_CUDA;
-        cudaError_t c2 = cudaMemcpyAsync(out_host, h->out_stage, bytes, cudaMemcpyDeviceToHost, h->cap_stream);
+        // The result goes straight into the caller's pinned buffer where the device can address it (the
+        // last kernel's 2 H bytes per token are posted writes over the bus, visible after the stream
+        // synchronisation below): one graph node and one hand-off less than a copy out of the staging
+        // buffer.  The tokens come in through k_stage_in (every block of the first two kernels reads them, so
+        // they are staged on the device once).
+        void* out_dev = (ao.devicePointer && aligned16(ao.devicePointer)) ? ao.devicePointer : nullptr;
+        const void* x_dev = (ax.devicePointer && aligned16(ax.devicePointer)) ? ax.devicePointer : nullptr;
+        cudaError_t c1;
+        if (x_dev) c1 = launch_pdl(k_stage_in, (int)((bytes / 16 + 255) / 256), 256, 0, h->cap_stream, static_cast<const uint4*>(x_dev),
+                                   reinterpret_cast<uint4*>(h->x_stage), (int)(bytes / 16));
+        else c1 = cudaMemcpyAsync(h->x_stage, x_host, bytes, cudaMemcpyHostToDevice, h->cap_stream);
+        const int rc = c1 == cudaSuccess ? moe_vqlr_decode_layer(h, h->x_stage, T, out_dev ? out_dev : h->out_stage, nullptr, h->cap_stream)
+                                         : MOE_VQLR_ERR_CUDA;
+        cudaError_t c2 = out_dev ? cudaSuccess : cudaMemcpyAsync(out_host, h->out_stage, bytes, cudaMemcpyDeviceToHost, h->cap_stream);
         h->launches = before;
         ge = cudaStreamEndCapture(h->cap_stream, &graph);
         if ((rc != MOE_VQLR_OK || c1 != cudaSuccess || c2 != cudaSuccess) && ge == cudaSuccess) ge = cudaErrorUnknown;
@@ -1178,13 +1200,14 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
       } else {
         h->io_x[T] = x_host;
         h->io_out[T] = out_host;
+        h->io_stage_in[T] = ax.devicePointer && aligned16(ax.devicePointer);
       }
     }
     if (h->io_graph[T]) {
       cudaError_t ce2 = cudaGraphLaunch(h->io_graph[T], st);
       if (ce2 == cudaSuccess) ce2 = cudaStreamSynchronize(st);
       if (ce2 != cudaSuccess) return fail(h, MOE_VQLR_ERR_CUDA, "graph launch with copies: %s", cudaGetErrorString(ce2));
-      h->launches += h->host_graph_launches;
+      h->launches += h->host_graph_launches + (h->io_stage_in[T] ? 1 : 0);
       return take_status(h);
     }
   }
