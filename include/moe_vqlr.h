@@ -202,9 +202,12 @@ int moe_vqlr_decode_layer(moe_vqlr_handle* h, const void* x, int32_t T, void* ou
  * asynchronous up to the final wait; pageable memory works but is slower.  Weights stay on
  * the device.  Synchronous on return.  The first call for each T captures the kernel chain into
  * a CUDA graph owned by the handle (later calls replay it), so that first call is slower and
- * must not itself run inside a stream capture.  With pinned host buffers the two copies are part
+ * must not itself run inside a stream capture.  With pinned host buffers the transfers are part
  * of the graph too (one launch and one wait per call) for as long as the caller passes the same
- * two pointers; other pointers re-capture it. */
+ * two pointers; other pointers re-capture it.  Pinned buffers that the device can address (16-byte
+ * aligned; cudaHostAlloc / cudaHostRegister memory under unified addressing) are read and written
+ * by the kernels themselves: a staging kernel fetches the tokens and the last kernel of the layer
+ * stores out_host directly, so out_host is complete only when the call has returned. */
 int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T, void* out_host,
                                void* cuda_stream);
 
