@@ -12,8 +12,8 @@
 // that no longer match the library) given to NVRTC with -DMOE_VQLR_JIT and one -DJ_* per constant, the
 // result loaded through the runtime's library API and launched like any other kernel.  NVRTC is
 // opened with dlopen at the first create() that wants it; without it, or when anything on the way
-// fails, the handle keeps the generic kernels (moe_vqlr_specialized() tells which, the reason is
-// kept for moe_vqlr_last_error()).  Compiled kernels are cached per process, device and option
+// fails, the handle keeps the precompiled kernels (moe_vqlr_specialized() tells how many were compiled,
+// moe_vqlr_specialization_note() why not).  Compiled kernels are cached per process, device and option
 // string: the layers of a model share one compilation.
 #pragma once
 #include <dlfcn.h>
