@@ -81,3 +81,31 @@ def test_layers_of_one_shape_share_a_compilation():
     assert t[2] < 0.5 * max(t[0], 0.5), t         # no second compilation (the first takes about a second)
     for m in mods:
         m.close()
+
+
+ALLOWED_NOTES = ("do not run the fused kernel", "exceed one wave")
+
+
+@pytest.mark.parametrize("mode", ["full", "paper", "dense"])
+def test_every_named_workload_compiles_for_its_shape(mode):
+    """Every workload of the tables, in every mode: the run-time compilation must succeed for its
+    combination of index type, code-word length, code books, activation and work plan.  A compile
+    error would otherwise only show as a slower layer (the precompiled kernels take over)."""
+    from dataclasses import replace
+    from paper_2609_21137_b200 import binding, devsynth
+    seen = set()
+    for name, shp in synth.SHAPES.items():
+        key = (shp.H, shp.I, shp.k, shp.S, shp.d, shp.K, shp.r, shp.T, shp.act, shp.idx12, shp.per_projection_codebook, shp.router_bias)
+        if key in seen or (shp.idx12 and mode == "dense"):
+            continue
+        seen.add(key)
+        small = replace(shp, E=max(shp.k, min(shp.E, 8)), mode=mode)
+        kw = devsynth.make_device_layer(small, seed=0, device="cuda")
+        kw.pop("x")
+        mod = binding.MoeVqlrLayer(**kw)
+        note = mod.specialization_note()
+        assert mod.specialized() > 0, f"{name} {mode}: {note}"
+        assert note == "" or any(a in note for a in ALLOWED_NOTES), f"{name} {mode}: {note}"
+        mod.close()
+        del kw
+        torch.cuda.empty_cache()
