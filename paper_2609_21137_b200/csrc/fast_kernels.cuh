@@ -854,14 +854,24 @@ __device__ __forceinline__ void router_zmma_pdl_body(const Params& P_in, const b
   const Params& P = P_in;
 #endif
   __shared__ float s_red[kZmmaWarps][128];
-  pdl_wait();      // the previous call's kernels may still read logits / z
-  pdl_launch();
+  // As in k_router_z_pdl, the weights of a unit (they never depend on the previous kernel) are
+  // requested before the dependency wait: a router row of up to 2048 values, or the first half of a
+  // z block's basis rows.
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int n_units = P.E * ((T + kTokGroup - 1) / kTokGroup), n_logit_blocks = (n_units + kZmmaWarps - 1) / kZmmaWarps;
   if ((int)blockIdx.x < n_logit_blocks) {      // the logits blocks come first: their FMA chains take longest
     const int unit = (int)blockIdx.x * kZmmaWarps + warp;
-    if (unit >= n_units) return;
-    if (P.H <= 2048) router_z_unit_row8(P, x, T, unit, lane);
+    const bool has = unit < n_units, early = has && P.H <= 2048;
+    RouterRow u;
+    uint4 wv[8];
+    if (early) {
+      u = router_z_row(P, T, unit);
+      router_z_load8(u, 0, P.H / 8, lane, wv);
+    }
+    pdl_wait();      // the previous call's kernels may still read logits / z; the tokens are its output
+    pdl_launch();
+    if (!has) return;
+    if (early) router_z_finish_row8(P, u, x, lane, wv);
     else router_z_unit(P, x, T, unit, lane);
     return;
   }
@@ -874,13 +884,18 @@ __device__ __forceinline__ void router_zmma_pdl_body(const Params& P_in, const b
   const uint4* xa4 = reinterpret_cast<const uint4*>(x + (size_t)g * P.H) + warp * per + c;
   const uint4* xb4 = reinterpret_cast<const uint4*>(x + (size_t)(g + 8) * P.H) + warp * per + c;
   const bool live_a = g < T, live_b = g + 8 < T;
+  uint4 wv0[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) wv0[u] = 4 * u < per ? __ldg(w4 + 4 * u) : make_uint4(0, 0, 0, 0);
+  pdl_wait();
+  pdl_launch();
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
   for (int s = 0; s < per; s += 16) {                              // four steps of 32 values with their loads in flight
     uint4 wv[4], av[4], bv[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const bool in = s + 4 * u < per;
-      wv[u] = in ? __ldg(w4 + s + 4 * u) : make_uint4(0, 0, 0, 0);
+      wv[u] = s == 0 ? wv0[u] : in ? __ldg(w4 + s + 4 * u) : make_uint4(0, 0, 0, 0);
       av[u] = (in && live_a) ? __ldg(xa4 + s + 4 * u) : make_uint4(0, 0, 0, 0);
       bv[u] = (in && live_b) ? __ldg(xb4 + s + 4 * u) : make_uint4(0, 0, 0, 0);
     }
