@@ -9,7 +9,8 @@ import torch
 import oracle
 from paper_2609_21137_b200 import synth
 
-from helpers import (assert_output, assert_routing, bf16_tensor_to_f64, logit_gaps, MIN_LOGIT_GAP)
+from helpers import (assert_output, assert_routing, bf16_tensor_to_f64, logit_gaps, MIN_LOGIT_GAP,
+                     toolkit_for_specialisation)
 
 pytestmark = pytest.mark.gpu
 
@@ -33,7 +34,8 @@ def _sampled_check(shp, rows, seed=0):
     plain = mod.decode(x)
     torch.cuda.synchronize()
     assert torch.equal(plain.view(torch.int16), out.view(torch.int16))
-    assert mod.specialized() > 0, mod.specialization_note()
+    if toolkit_for_specialisation():
+        assert mod.specialized() > 0, mod.specialization_note()
     mod.close()
     del layer
     return m

@@ -6,9 +6,10 @@ import pytest
 import torch
 
 from paper_2609_21137_b200 import synth
-from tests.helpers import make_checked_layer, assert_output, bf16_tensor_to_f64
+from tests.helpers import make_checked_layer, assert_output, bf16_tensor_to_f64, toolkit_for_specialisation
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu,
+              pytest.mark.skipif(not toolkit_for_specialisation(), reason="no NVRTC / CUDA headers: the precompiled kernels run")]
 
 SHAPES = [
     synth.shape("qwen3", E=16),                                   # 16-bit indices, one 64 KB book, compressed down
