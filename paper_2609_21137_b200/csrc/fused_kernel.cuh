@@ -42,8 +42,10 @@ struct FusedLayout {
   int dn_slot_bytes;
 };
 
+// gu_halves: 2 = partial tiles of gate and up, 1 = of up alone (experts without a gate projection).
 __host__ __device__ inline FusedLayout fused_layout(int K, int n_books, int T, int H, int r, const StagePlan& pg,
-                                                    const FusedPlan& fp, bool dn_dense, int idx_bytes, int E, int k, int S) {
+                                                    const FusedPlan& fp, bool dn_dense, int idx_bytes, int E, int k, int S,
+                                                    int gu_halves = 2) {
   FusedLayout L;
   const size_t cb_bytes = (size_t)K * 16 * (pg.repl ? 8 : 1);
   L.cb_u = n_books == 2 ? cb_bytes : 0;
@@ -54,7 +56,7 @@ __host__ __device__ inline FusedLayout fused_layout(int K, int n_books, int T, i
   L.ring_d = o;  o += (size_t)kFusedWarps * fp.depth_d * L.dn_slot_bytes;
   L.z = o;       o += (size_t)2 * T * 2 * ((r + 7) / 8) * 16;
   L.route = o;   o += route_smem_bytes(T, E, k, S);
-  L.parts = o;   o += (size_t)fp.tps * pg.n_parts * 2 * 64 * 4;      // [part][tile][gate|up][token 8][row 8]
+  L.parts = o;   o += (size_t)fp.tps * pg.n_parts * gu_halves * 64 * 4;      // [part][tile][gate|up][token 8][row 8]
   L.pf = o;      o += (size_t)8 * 8 * fp.tps * 4;                    // p as fp32 [token 8][row]
   L.ph = o;      o += (size_t)8 * 4 * fp.jd * 16;                    // p as bf16 hi blocks [token 8][4 jd]
   L.pl = o;      o += (size_t)8 * 4 * fp.jd * 16;                    // ... and the bf16 remainder
@@ -120,7 +122,8 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
   char* s_base = reinterpret_cast<char*>(s_u4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, c = lane & 3;
   const int nb = pg.nb, xs = nb + 1, rb = (P.r + 7) / 8, Dg = fp.depth_g, Dd = fp.depth_d;
-  const FusedLayout L = fused_layout(P.K, n_books, T, P.H, P.r, pg, fp, DN_DENSE, (int)sizeof(IdxT), P.E, P.k, P.S);
+  const int gu_halves = (SP && P.act == 2) ? 1 : 2;      // up-only experts keep no gate tiles
+  const FusedLayout L = fused_layout(P.K, n_books, T, P.H, P.r, pg, fp, DN_DENSE, (int)sizeof(IdxT), P.E, P.k, P.S, gu_halves);
   GuSmem m;
   m.cb_g = s_u4;
   m.cb_u = reinterpret_cast<uint4*>(s_base + L.cb_u);
@@ -360,9 +363,9 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
           acc_u[0][0] += acc_u[0][2]; acc_u[0][1] += acc_u[0][3];
         }
         // partial tile of this unit: token g, rows 2c and 2c+1 of the tile
-        float* dst = s_parts + ((size_t)(part * fp.tps + tile) * 2) * 64 + g * 8 + 2 * c;
-        *reinterpret_cast<float2*>(dst) = make_float2(acc_g[0][0] + acc_g[1][0], acc_g[0][1] + acc_g[1][1]);
-        *reinterpret_cast<float2*>(dst + 64) = make_float2(acc_u[0][0] + acc_u[1][0], acc_u[0][1] + acc_u[1][1]);
+        float* dst = s_parts + ((size_t)(part * fp.tps + tile) * gu_halves) * 64 + g * 8 + 2 * c;
+        if (!up_only) *reinterpret_cast<float2*>(dst) = make_float2(acc_g[0][0] + acc_g[1][0], acc_g[0][1] + acc_g[1][1]);
+        *reinterpret_cast<float2*>(dst + (up_only ? 0 : 64)) = make_float2(acc_u[0][0] + acc_u[1][0], acc_u[0][1] + acc_u[1][1]);
         if (i < 2) TRACE_STAMP(3, 11 + 2 * i);
       }
     }
@@ -390,9 +393,9 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
         const int tile = row >> 3, rr = row & 7;
         float gs = 0.f, us = 0.f;
         for (int part = 0; part < pg.n_parts; ++part) {
-          const float* src = s_parts + ((size_t)(part * fp.tps + tile) * 2) * 64 + tk * 8 + rr;
-          gs += src[0];
-          us += src[64];
+          const float* src = s_parts + ((size_t)(part * fp.tps + tile) * gu_halves) * 64 + tk * 8 + rr;
+          if (!up_only) gs += src[0];
+          us += src[up_only ? 0 : 64];
         }
         const float pv = gated_act(gs, us, P.act);
         s_pf[tk * R_max + row] = pv;

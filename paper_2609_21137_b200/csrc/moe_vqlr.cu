@@ -290,6 +290,8 @@ const void* gateup_kernel(const moe_vqlr_handle* h) {
 const void* down_kernel(const moe_vqlr_handle* h, int tpu) {
   return h->special ? down_kernel_sp<true>(h->dn_dense, h->d4, h->idx_bytes, tpu) : down_kernel_sp<false>(h->dn_dense, h->d4, h->idx_bytes, tpu);
 }
+// Partial tiles the fused kernel keeps per unit: gate and up, or up alone for experts without a gate.
+int fused_gu_halves(const moe_vqlr_handle* h) { return (h->special && h->P.act == 2) ? 1 : 2; }
 const void* fused_kernel(const moe_vqlr_handle* h, int jd) {
   return h->special ? fused_kernel_sp<true>(h->dn_dense, h->d4, h->idx_bytes, jd) : fused_kernel_sp<false>(h->dn_dense, h->d4, h->idx_bytes, jd);
 }
@@ -343,7 +345,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         fpl.depth_d = h->fused_dd[T];
         StagePlan pgl = h->plan_gu_fused;
         pgl.x_smem = h->fused_xs[T];
-        const size_t smem2 = fused_layout(P.K, h->n_books, T, P.H, P.r, pgl, fpl, h->dn_dense, h->idx_tc, P.E, P.k, P.S).total;
+        const size_t smem2 = fused_layout(P.K, h->n_books, T, P.H, P.r, pgl, fpl, h->dn_dense, h->idx_tc, P.E, P.k, P.S, fused_gu_halves(h)).total;
         {
           Params Pa = P;
           const bf16* xa = xb;
@@ -799,7 +801,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
           for (int dg = 3; dg >= 2 && !found; --dg) {
             fp.depth_g = dg;
             fp.depth_d = dd;
-            found = fused_layout(K, h->n_books, 1, H, r, pg, fp, h->dn_dense, h->idx_tc, E, k, S).total <= limit;
+            found = fused_layout(K, h->n_books, 1, H, r, pg, fp, h->dn_dense, h->idx_tc, E, k, S, fused_gu_halves(h)).total <= limit;
           }
       }
       // many thin slices would turn the partial y into the dominant traffic: leave those shapes to the chain
@@ -824,7 +826,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
                 pgt.x_smem = xsm;
                 fp.depth_g = dg;
                 fp.depth_d = dd;
-                const size_t need = fused_layout(K, h->n_books, t, H, r, pgt, fp, h->dn_dense, h->idx_tc, E, k, S).total;
+                const size_t need = fused_layout(K, h->n_books, t, H, r, pgt, fp, h->dn_dense, h->idx_tc, E, k, S, fused_gu_halves(h)).total;
                 if (need <= limit) {
                   fit = true;
                   h->fused_dg[t] = (signed char)dg;
@@ -898,7 +900,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
       fp1.depth_d = h->fused_dd[1];
       StagePlan pg1 = pg;
       pg1.x_smem = h->fused_xs[1];
-      const size_t smem1 = fused_layout(K, h->n_books, 1, H, r, pg1, fp1, h->dn_dense, h->idx_tc, E, k, S).total;
+      const size_t smem1 = fused_layout(K, h->n_books, 1, H, r, pg1, fp1, h->dn_dense, h->idx_tc, E, k, S, fused_gu_halves(h)).total;
       cudaKernel_t kern_r = nullptr, kern_c = nullptr;
       size_t cf_smem = ((size_t)(k + S) * (r > 0 ? r : 0) + (size_t)(k + S) * kCfCols * 2) * sizeof(float);
       if (cf_smem < kCfAloneBytes) cf_smem = kCfAloneBytes;
