@@ -1,4 +1,5 @@
-// Run-time compilation of the single-token kernels for ONE layer shape.
+// Run-time compilation of the hot kernels for ONE layer shape: the three kernels of a single-token
+// call, and the gate/up, down and weighted-sum kernels of the chain that serves several tokens.
 //
 // At batch 1 every block of the router -> expert -> weighted-sum path runs most of its code once,
 // so the path costs what its instruction stream costs: the generic kernels carry every shape,
@@ -144,8 +145,7 @@ const char kJitStdint[] =
     "typedef unsigned long long uint64_t;\n";
 
 // Compiles (or finds) the specialised kernels of `source` (kJitSource or kJitChainSource) for `defs`
-// on the current device.  Returns the loaded
-// library or nullptr with *why set.
+// on the current device.  Returns the loaded library, or nullptr with *why set.
 cudaLibrary_t jit_library(const char* source, const std::vector<std::string>& defs, std::string* why) {
   std::lock_guard<std::mutex> lock(g_jit_mu);
   nvrtc_open();
