@@ -110,3 +110,48 @@ def test_every_named_workload_compiles_for_its_shape(mode):
         mod.close()
         del kw
         torch.cuda.empty_cache()
+
+
+def _drawn_shapes(n, seed):
+    """Shapes drawn from the ranges the tensor-core kernels cover (H a multiple of 64 so that rows
+    split into whole groups of eight blocks), with the odd values that constant folding could get
+    wrong: expert counts that are no multiple of 32, ranks that are no multiple of 32, a short
+    last slice of I, shared experts, either index width, one or two code books, every activation."""
+    import numpy as np
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        d = int(rng.choice([8, 8, 4]))
+        K = int(rng.choice([64, 256] if d == 4 else [100, 256, 512, 1000, 4096]))
+        if d == 4 and K % 2:
+            K += 1
+        mode = str(rng.choice(["full", "full", "paper"]))
+        # a compressed down projection contracts over whole groups of eight blocks of I
+        I = 64 * int(rng.integers(1, 13)) + (8 * int(rng.integers(0, 8)) if mode == "paper" else 0)
+        out.append(synth.LayerShape(
+            f"drawn{i}", H=64 * int(rng.integers(2, 20)), I=I,
+            E=int(rng.integers(4, 41)), k=int(rng.integers(1, 5)), S=int(rng.choice([0, 0, 1, 2])), d=d, K=K,
+            r=8 * int(rng.integers(0, 13)), T=int(rng.choice([1, 1, 2, 5, 9, 16])), router_bias=bool(rng.integers(0, 2)),
+            mode=mode, per_projection_codebook=bool(rng.integers(0, 2)),
+            act=str(rng.choice(["silu", "silu", "gelu_tanh", "relu2"]))))
+    return out
+
+
+@pytest.mark.parametrize("shp", _drawn_shapes(24, seed=20260921), ids=lambda s: f"{s.name}-H{s.H}-I{s.I}-E{s.E}-k{s.k}-S{s.S}-d{s.d}-K{s.K}-r{s.r}-T{s.T}-{s.mode}-{s.act}")
+def test_drawn_shapes_specialised_equals_precompiled(shp):
+    from paper_2609_21137_b200 import binding
+    layer, res, _ = make_checked_layer(shp, 0)
+    x = binding.bits_to_device(layer.x, "cuda")
+    spec = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+    plain = binding.MoeVqlrLayer.from_synth(layer, device="cuda", flags=binding.FLAG_NO_SPECIALIZE)
+    note = spec.specialization_note()
+    assert spec.specialized() > 0, note
+    assert "nvrtc" not in note.lower(), note
+    a = spec.decode(x)
+    b = plain.decode(x)
+    torch.cuda.synchronize()
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    assert_output(bf16_tensor_to_f64(a), res.out, what=shp.name)
+    assert spec.last_status() == 0
+    spec.close()
+    plain.close()
