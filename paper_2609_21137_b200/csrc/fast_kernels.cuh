@@ -445,27 +445,56 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
     return;
   }
   TRACE_STAMP(1, 2);
-  // ---- sort the pairs by (expert, token): four lanes share a pair and scan a quarter each ---
-  for (int q0 = 0; q0 < n_pairs; q0 += nthr >> 2) {       // uniform trip count for the shuffles
-    const int q = q0 + (tid >> 2);
-    const bool live = q < n_pairs;
-    const int e = live ? R.sel_id[q] : 0;
-    int lt = 0, eq_before = 0, eq_total = 0;
-    if (live)
-      for (int q2 = tid & 3; q2 < n_pairs; q2 += 4) {
-        const int e2 = R.sel_id[q2];
-        lt += e2 < e;
-        eq_total += e2 == e;
-        eq_before += (e2 == e) && (q2 < q);                // same expert: pair order = token order
+  // ---- pairs sorted by (expert, token) and cut into work groups, by counting -----------------
+  // Per expert a bit map of the tokens that selected it (a token selects an expert at most once, so
+  // OR-ing the bits does not depend on the order of the threads).  Population counts of the map give a
+  // pair's place inside its expert's run and the run's length; an exclusive scan over the experts by
+  // one warp gives the run's first pair position and first work group (a new group starts at every
+  // eighth pair of a run).  T >= 2 here, so the 2 E words fit where the logits were.
+  unsigned int* s_map = reinterpret_cast<unsigned int*>(R.logit);       // [E] tokens of the expert
+  unsigned int* s_off = s_map + E;                                       // [E] first pair position | first group << 16
+  for (int e = tid; e < E; e += nthr) s_map[e] = 0u;
+  __syncthreads();
+  for (int q = tid; q < n_pairs; q += nthr) atomicOr(&s_map[R.sel_id[q]], 1u << (q / k));
+  __syncthreads();
+  if (warp == 0) {
+    const int per = (E + 31) >> 5, e0 = lane * per;          // a contiguous run of experts per lane
+    unsigned int mine = 0u;                                   // pairs | groups << 16 (both at most 16 * 32)
+    for (int i = 0; i < per; ++i)
+      if (e0 + i < E) {
+        const unsigned int c = (unsigned int)__popc(s_map[e0 + i]);
+        mine += c | (((c + kGroupTokens - 1) / kGroupTokens) << 16);
       }
-    lt += __shfl_xor_sync(0xffffffffu, lt, 1);        lt += __shfl_xor_sync(0xffffffffu, lt, 2);
-    eq_before += __shfl_xor_sync(0xffffffffu, eq_before, 1);  eq_before += __shfl_xor_sync(0xffffffffu, eq_before, 2);
-    eq_total += __shfl_xor_sync(0xffffffffu, eq_total, 1);    eq_total += __shfl_xor_sync(0xffffffffu, eq_total, 2);
-    if (live && (tid & 3) == 0) {
-      const int pos = lt + eq_before, t = q / k, s = q - t * k;
-      R.sort_e[pos] = e; R.sort_j[pos] = eq_before; R.sort_c[pos] = eq_total;
-      R.pair_token[pos] = t;
-      if (write_global) { P.pair_token[pos] = t; P.pair_slot[pos] = s; P.pair_w[pos] = R.w[q]; P.inv_pos[t * (k + S) + s] = pos; }
+    unsigned int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    unsigned int run = incl - mine;
+    for (int i = 0; i < per; ++i)
+      if (e0 + i < E) {
+        s_off[e0 + i] = run;
+        const unsigned int c = (unsigned int)__popc(s_map[e0 + i]);
+        run += c | (((c + kGroupTokens - 1) / kGroupTokens) << 16);
+      }
+    if (lane == 31) R.warp_cnt[0] = (int)(incl >> 16);      // work groups of the routed experts
+  }
+  __syncthreads();
+  const int base = R.warp_cnt[0];
+  for (int q = tid; q < n_pairs; q += nthr) {
+    const int t = q / k, s = q - t * k, e = R.sel_id[q];
+    const unsigned int bm = s_map[e], o = s_off[e];
+    const int j = __popc(bm & ((1u << t) - 1u)), c = __popc(bm);      // same expert: pair order = token order
+    const int pos = (int)(o & 0xffffu) + j;
+    R.sort_e[pos] = e; R.sort_j[pos] = j; R.sort_c[pos] = c;
+    R.pair_token[pos] = t;
+    if (write_global) { P.pair_token[pos] = t; P.pair_slot[pos] = s; P.pair_w[pos] = R.w[q]; P.inv_pos[t * (k + S) + s] = pos; }
+    if (j % kGroupTokens == 0) {
+      const int gi = (int)(o >> 16) + j / kGroupTokens;
+      R.grp_e[gi] = e;
+      R.grp_off[gi] = pos;
+      R.grp_cnt[gi] = min(kGroupTokens, c - j);
     }
   }
   for (int q = tid; q < S * T; q += nthr) {                 // shared experts: every token, weight 1
@@ -475,27 +504,7 @@ __device__ void route_in_block(const Params& P, int T, const RouteSmem& R, bool 
       P.inv_pos[(q % T) * (k + S) + k + q / T] = n_pairs + q;
     }
   }
-  __syncthreads();
   TRACE_STAMP(1, 3);
-  // ---- work groups: a new group starts at every eighth pair of an expert's run -------------
-  int base = 0;
-  for (int p0 = 0; p0 < n_pairs; p0 += nthr) {
-    const int pos = p0 + tid;
-    const bool first = pos < n_pairs && (R.sort_j[pos] % kGroupTokens) == 0;
-    const unsigned int bal = __ballot_sync(0xffffffffu, first);
-    if (lane == 0) R.warp_cnt[warp] = __popc(bal);
-    __syncthreads();
-    int before = base;
-    for (int w = 0; w < warp; ++w) before += R.warp_cnt[w];
-    if (first) {
-      const int gi = before + __popc(bal & ((1u << lane) - 1u));
-      R.grp_e[gi] = R.sort_e[pos];
-      R.grp_off[gi] = pos;
-      R.grp_cnt[gi] = min(kGroupTokens, R.sort_c[pos] - R.sort_j[pos]);
-    }
-    for (int w = 0; w < nwarp; ++w) base += R.warp_cnt[w];
-    __syncthreads();
-  }
   const int sh_groups = (T + kGroupTokens - 1) / kGroupTokens;
   for (int q = tid; q < S * sh_groups; q += nthr) {
     const int s = q / sh_groups, pg = q - s * sh_groups;
