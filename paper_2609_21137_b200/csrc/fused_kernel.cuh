@@ -23,11 +23,11 @@
 
 namespace {
 
-constexpr int kFusedThreads = 384;
-constexpr int kFusedWarps = kFusedThreads / 32;
+constexpr int kFusedMaxThreads = 512;      // a block runs 16 warps where its shared memory allows, else 12 (FusedPlan::warps)
 constexpr int kFusedMaxJd = 4;       // k steps of the down product: at most 16 blocks per slice
 
 struct FusedPlan {
+  int warps;      // warps per block: 16, or 12 where the rings of 16 do not fit (more warps hide more of the read latency)
   int tps;        // row tiles of I per slice (the last slice of an expert may have fewer)
   int n_sl;       // slices per expert
   int t_last;     // row tiles of the last slice
@@ -51,9 +51,9 @@ __host__ __device__ inline FusedLayout fused_layout(int K, int n_books, int T, i
   L.cb_u = n_books == 2 ? cb_bytes : 0;
   size_t o = (size_t)n_books * cb_bytes;
   L.x = o;       o += pg.x_smem ? (size_t)T * (H / 8 + 1) * 16 : 0;
-  L.ring_g = o;  o += (size_t)kFusedWarps * fp.depth_g * 2 * 32 * 16;
+  L.ring_g = o;  o += (size_t)fp.warps * fp.depth_g * 2 * 32 * 16;
   L.dn_slot_bytes = dn_dense ? fp.jd * 32 * 16 : (32 * fp.jd * idx_bytes + 15) / 16 * 16;
-  L.ring_d = o;  o += (size_t)kFusedWarps * fp.depth_d * L.dn_slot_bytes;
+  L.ring_d = o;  o += (size_t)fp.warps * fp.depth_d * L.dn_slot_bytes;
   L.z = o;       o += (size_t)2 * T * 2 * ((r + 7) / 8) * 16;
   L.route = o;   o += route_smem_bytes(T, E, k, S);
   L.parts = o;   o += (size_t)fp.tps * pg.n_parts * gu_halves * 64 * 4;      // [part][tile][gate|up][token 8][row 8]
@@ -110,7 +110,7 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
   MOE_VQLR_JIT_PARAMS(P);
   pg.nb = J_NB; pg.n_slices = J_NSLICES; pg.n_lr = J_NLR; pg.n_parts = J_NPARTS; pg.repl = J_REPL; pg.x_smem = J_XSMEM;
   FusedPlan fp = fp_in;
-  fp.tps = J_TPS; fp.n_sl = J_NSL; fp.t_last = J_TLAST; fp.jd = JD; fp.depth_g = J_DEPTH_G; fp.depth_d = J_DEPTH_D; fp.rp_log2 = J_RP_LOG2;
+  fp.warps = J_WARPS; fp.tps = J_TPS; fp.n_sl = J_NSL; fp.t_last = J_TLAST; fp.jd = JD; fp.depth_g = J_DEPTH_G; fp.depth_d = J_DEPTH_D; fp.rp_log2 = J_RP_LOG2;
   (void)n_books_in;
 #else
   constexpr bool kShape = false;
@@ -121,6 +121,7 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
   extern __shared__ uint4 s_u4[];
   char* s_base = reinterpret_cast<char*>(s_u4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, c = lane & 3;
+  const int nw = fp.warps, nthr = nw * 32;       // = blockDim.x
   const int nb = pg.nb, xs = nb + 1, rb = (P.r + 7) / 8, Dg = fp.depth_g, Dd = fp.depth_d;
   const int gu_halves = (SP && P.act == 2) ? 1 : 2;      // up-only experts keep no gate tiles
   const FusedLayout L = fused_layout(P.K, n_books, T, P.H, P.r, pg, fp, DN_DENSE, (int)sizeof(IdxT), P.E, P.k, P.S, gu_halves);
@@ -165,9 +166,9 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
     const FastDiv d_tiles = last_sl ? fp.d_tlast : fp.d_tps;
     it.row0 = it.si * fp.tps * 8;
     const int Us = pg.n_slices * it.tiles, Ul = pg.n_lr * it.tiles;
-    const int s0 = Us * warp / kFusedWarps, l0 = Ul * warp / kFusedWarps;
-    it.ns = Us * (warp + 1) / kFusedWarps - s0;
-    it.n_my = it.ns + Ul * (warp + 1) / kFusedWarps - l0;
+    const int s0 = Us * warp / nw, l0 = Ul * warp / nw;
+    it.ns = Us * (warp + 1) / nw - s0;
+    it.n_my = it.ns + Ul * (warp + 1) / nw - l0;
     it.sp = kShape ? s0 / it.tiles : fdiv(s0, d_tiles); it.st = s0 - it.sp * it.tiles;
     const int lq = kShape ? l0 / it.tiles : fdiv(l0, d_tiles);
     it.lp = pg.n_slices + lq; it.lt = l0 - lq * it.tiles;
@@ -222,10 +223,10 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
   TRACE_STAMP(3, 0);
   gu_stage_async<false>(P, x, T, pg, n_books, m);
   const int n_pos = T * (P.k + P.S);
-  const int n_dn = (P.H / 8 - warp + kFusedWarps - 1) / kFusedWarps;    // down row tiles of this warp: warp, warp + 12, ...
+  const int n_dn = (P.H / 8 - warp + nw - 1) / nw;    // down row tiles of this warp: warp, warp + nw, ...
   // down tile warp + 12 i of the item -> slot `slot` of this warp's down ring
   auto dn_request = [&](const Item& it, int i, int slot_i) {
-    const int jt = warp + i * kFusedWarps;
+    const int jt = warp + i * nw;
     char* slot = ring_d + (size_t)slot_i * L.dn_slot_bytes;
     if (DN_DENSE) {
       const uint4* wd = reinterpret_cast<const uint4*>(P.down.dense + ((size_t)it.e * P.H + jt * 8 + g) * P.I + it.row0);
@@ -289,7 +290,7 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
       const char* src = reinterpret_cast<const char*>(idx_dp + (((size_t)it.e * fp.n_sl + si) * (P.H / 8) + warp) * 32 * JD) + lane * 16;
       char* dst = ring_d + lane * 16;
       if (lane * 16 < bytes)
-        for (int i = 0; i < n_dn; ++i) { cp_async16(dst, src); src += (size_t)kFusedWarps * bytes; dst += L.dn_slot_bytes; }
+        for (int i = 0; i < n_dn; ++i) { cp_async16(dst, src); src += (size_t)nw * bytes; dst += L.dn_slot_bytes; }
       cp_async_commit();
     }
     // ---- gate / up partial tiles into shared memory ------------------------------------------
@@ -387,7 +388,7 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
 
     // ---- p = phi(gate) * up for the slice's rows; parts added in ascending order -------------
     const int R_here = tiles_here * 8, R_max = fp.tps * 8, RP = 1 << fp.rp_log2;
-    for (int idx = tid; idx < cnt * RP; idx += kFusedThreads) {
+    for (int idx = tid; idx < cnt * RP; idx += nthr) {
       const int tk = idx >> fp.rp_log2, row = idx & (RP - 1);
       if (row < R_here) {
         const int tile = row >> 3, rr = row & 7;
@@ -409,7 +410,7 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
 
     // ---- partial z_d of the slice (compressed down projection with a low-rank term) -----------
     if (!DN_DENSE && P.r > 0) {
-      for (int idx = tid; idx < cnt * P.r; idx += kFusedThreads) {
+      for (int idx = tid; idx < cnt * P.r; idx += nthr) {
         const int tk = idx / P.r, rho = idx - tk * P.r;
         const uint4* b4 = reinterpret_cast<const uint4*>(P.down.basis + (size_t)rho * P.I + row0);
         const float* pv = s_pf + tk * R_max;
@@ -448,7 +449,7 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
           cp_async_wait_pending(Dd - 1);
           const uint4* slot = reinterpret_cast<const uint4*>(ring_d + (size_t)d_use * L.dn_slot_bytes) + lane;
           if (++d_use == Dd) d_use = 0;
-          const int jt = warp + i * kFusedWarps;
+          const int jt = warp + i * nw;
           float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};      // two chains; each: hi product | lo product
 #pragma unroll
           for (int j = 0; j < JD; ++j) {
@@ -503,7 +504,7 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
 #pragma unroll
           for (int u = 0; u < kU; ++u)
             if (ydst && i0 + u < n_dn)
-              *reinterpret_cast<float2*>(ydst + (warp + (i0 + u) * kFusedWarps) * 8) =
+              *reinterpret_cast<float2*>(ydst + (warp + (i0 + u) * nw) * 8) =
                   make_float2(acc[u][0] + acc[u][2], acc[u][1] + acc[u][3]);
         }
       }
@@ -521,7 +522,7 @@ __device__ __forceinline__ void expert_fused_body(const Params& P_in, const bf16
 }
 
 template <typename IdxT, bool DN_DENSE, int JD, bool D4 = false, bool SP = false>
-__global__ void __launch_bounds__(kFusedThreads, 1)
+__global__ void __launch_bounds__(kFusedMaxThreads, 1)
 k_expert_fused(const Params P, const bf16* __restrict__ x, int T, const StagePlan pg, const FusedPlan fp, int n_books,
                int want_dbg, const IdxT* __restrict__ idx_dp) {
   expert_fused_body<IdxT, DN_DENSE, JD, D4, SP, false>(P, x, T, pg, fp, n_books, want_dbg, idx_dp);

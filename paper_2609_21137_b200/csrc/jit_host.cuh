@@ -105,7 +105,7 @@ const char kJitSource[] =
     "              \"the kernel sources beside the library are not the ones it was built from\");\n"
     "extern \"C\" __global__ void __launch_bounds__(32 * kRouterWarps)\n"
     "k_router_z_jit(const Params P, const bf16* __restrict__ x, int T) { router_z_pdl_body<true>(P, x, T); }\n"
-    "extern \"C\" __global__ void __launch_bounds__(kFusedThreads, 1)\n"
+    "extern \"C\" __global__ void __launch_bounds__(32 * J_WARPS, 1)\n"
     "k_expert_fused_jit(const Params P, const bf16* __restrict__ x, int T, const StagePlan pg, const FusedPlan fp,\n"
     "                   int n_books, int want_dbg, const J_IDXT* __restrict__ idx_dp) {\n"
     "  expert_fused_body<J_IDXT, J_DENSE, J_JD, J_D4, J_SP, true>(P, x, T, pg, fp, n_books, want_dbg, idx_dp);\n"

@@ -57,6 +57,7 @@ struct moe_vqlr_handle {
   int fused_max_T;           // ... for calls of up to this many tokens (shared memory)
   FusedPlan fplan;
   signed char fused_dg[kMaxT + 1], fused_dd[kMaxT + 1];   // ring depths that fit for T tokens (0: the chain runs)
+  signed char fused_w[kMaxT + 1];                         // ... and with this many warps per block (16 where they fit, else 12)
   signed char fused_xs[kMaxT + 1];                        // ... with the tokens staged in shared memory (else read from L2)
   StagePlan plan_gu_fused;
   bool per_expert_launch;   // ablation: gate/up and down run as one launch per work group
@@ -343,6 +344,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
         FusedPlan fpl = h->fplan;
         fpl.depth_g = h->fused_dg[T];
         fpl.depth_d = h->fused_dd[T];
+        fpl.warps = h->fused_w[T];
         StagePlan pgl = h->plan_gu_fused;
         pgl.x_smem = h->fused_xs[T];
         const size_t smem2 = fused_layout(P.K, h->n_books, T, P.H, P.r, pgl, fpl, h->dn_dense, h->idx_tc, P.E, P.k, P.S, fused_gu_halves(h)).total;
@@ -353,7 +355,7 @@ cudaError_t launch_stage(moe_vqlr_handle* h, int stage, const bf16* xb, int T, b
           const void* idp = h->dn_dense ? nullptr : h->idx_dp;
           void* args[] = {&Pa, &xa, &Ta, &pgl, &fpl, &nb_a, &dbg_a, &idp};
           const void* fn = (h->jit_fused && T == 1 && !h->want_dbg) ? h->jit_fused : fused_kernel(h, fpl.jd);
-          le = launch_pdl_ptr(fn, h->sm_count, kFusedThreads, smem2, st, args);
+          le = launch_pdl_ptr(fn, h->sm_count, 32 * fpl.warps, smem2, st, args);
         }
         ran = true;
         break;
@@ -796,7 +798,8 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
         while ((1 << fp.rp_log2) < 8 * tps) ++fp.rp_log2;
         // compressed down projection: every index byte of a warp's down tiles is resident (one slot per
         // tile); dense: a ring as deep as fits, its bytes in flight are what hides the DRAM latency
-        const int dn_tiles_per_warp = (H / 8 + kFusedWarps - 1) / kFusedWarps;
+        fp.warps = 12;      // the slice plan is chosen for the smaller block; 16 warps are taken per token count below
+        const int dn_tiles_per_warp = (H / 8 + fp.warps - 1) / fp.warps;
         for (int dd = h->dn_dense ? 8 : dn_tiles_per_warp; dd >= (h->dn_dense ? 2 : dn_tiles_per_warp) && !found; --dd)
           for (int dg = 3; dg >= 2 && !found; --dg) {
             fp.depth_g = dg;
@@ -813,28 +816,33 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
         fp.d_tlast = make_fastdiv((unsigned int)fp.t_last);
         int maxT_fit = 0;
         size_t smem_max = 0;
-        const int dn_tiles_per_warp = (H / 8 + kFusedWarps - 1) / kFusedWarps;
         memset(h->fused_dg, 0, sizeof h->fused_dg);
         memset(h->fused_dd, 0, sizeof h->fused_dd);
         memset(h->fused_xs, 0, sizeof h->fused_xs);
-        for (int t = 1; t <= maxT; ++t) {          // staged tokens and the deepest rings that fit beside them
+        memset(h->fused_w, 0, sizeof h->fused_w);
+        for (int t = 1; t <= maxT; ++t) {          // staged tokens, the widest block and the deepest rings that fit beside them
           bool fit = false;
-          for (int xsm = 1; xsm >= 0 && !fit; --xsm)
-            for (int dd = h->dn_dense ? 8 : dn_tiles_per_warp; dd >= (h->dn_dense ? 3 : dn_tiles_per_warp) && !fit; --dd)
-              for (int dg = 3; dg >= 2 && !fit; --dg) {
-                StagePlan pgt = pg;
-                pgt.x_smem = xsm;
-                fp.depth_g = dg;
-                fp.depth_d = dd;
-                const size_t need = fused_layout(K, h->n_books, t, H, r, pgt, fp, h->dn_dense, h->idx_tc, E, k, S, fused_gu_halves(h)).total;
-                if (need <= limit) {
-                  fit = true;
-                  h->fused_dg[t] = (signed char)dg;
-                  h->fused_dd[t] = (signed char)dd;
-                  h->fused_xs[t] = (signed char)xsm;
-                  if (need > smem_max) smem_max = need;
+          for (int W = 16; W >= 12 && !fit; W -= 4) {
+            fp.warps = W;
+            const int dn_tiles_per_warp = (H / 8 + W - 1) / W;
+            for (int xsm = 1; xsm >= 0 && !fit; --xsm)
+              for (int dd = h->dn_dense ? 8 : dn_tiles_per_warp; dd >= (h->dn_dense ? 3 : dn_tiles_per_warp) && !fit; --dd)
+                for (int dg = 3; dg >= 2 && !fit; --dg) {
+                  StagePlan pgt = pg;
+                  pgt.x_smem = xsm;
+                  fp.depth_g = dg;
+                  fp.depth_d = dd;
+                  const size_t need = fused_layout(K, h->n_books, t, H, r, pgt, fp, h->dn_dense, h->idx_tc, E, k, S, fused_gu_halves(h)).total;
+                  if (need <= limit) {
+                    fit = true;
+                    h->fused_dg[t] = (signed char)dg;
+                    h->fused_dd[t] = (signed char)dd;
+                    h->fused_xs[t] = (signed char)xsm;
+                    h->fused_w[t] = (signed char)W;
+                    if (need > smem_max) smem_max = need;
+                  }
                 }
-              }
+          }
           if (!fit) break;                         // more tokens need more room
           maxT_fit = t;
         }
@@ -888,7 +896,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
     def("J_NB", pg.nb); def("J_NSLICES", pg.n_slices); def("J_NLR", pg.n_lr); def("J_NPARTS", pg.n_parts);
     def("J_REPL", pg.repl); def("J_XSMEM", h->fused_xs[1]);
     def("J_TPS", fp.tps); def("J_NSL", fp.n_sl); def("J_TLAST", fp.t_last); def("J_JD", fp.jd); def("J_RP_LOG2", fp.rp_log2);
-    def("J_DEPTH_G", h->fused_dg[1]); def("J_DEPTH_D", h->fused_dd[1]);
+    def("J_DEPTH_G", h->fused_dg[1]); def("J_DEPTH_D", h->fused_dd[1]); def("J_WARPS", h->fused_w[1]);
     defs.push_back(std::string("-DJ_IDXT=") + ((h->d4 || h->idx_bytes == 2) ? "uint16_t" : "uint8_t"));
     defs.push_back(std::string("-DJ_DENSE=") + (h->dn_dense ? "true" : "false"));
     defs.push_back(std::string("-DJ_D4=") + (h->d4 ? "true" : "false"));
@@ -898,6 +906,7 @@ int moe_vqlr_create(const moe_vqlr_config* cfg_in, moe_vqlr_handle** out) {
       FusedPlan fp1 = fp;
       fp1.depth_g = h->fused_dg[1];
       fp1.depth_d = h->fused_dd[1];
+      fp1.warps = h->fused_w[1];
       StagePlan pg1 = pg;
       pg1.x_smem = h->fused_xs[1];
       const size_t smem1 = fused_layout(K, h->n_books, 1, H, r, pg1, fp1, h->dn_dense, h->idx_tc, E, k, S, fused_gu_halves(h)).total;
