@@ -574,10 +574,15 @@ __device__ __forceinline__ void combine_fused_body(const Params& P_in, bf16* __r
   // guaranteed to be visible after the wait, so the ids are read again then and a thread whose id
   // has changed asks again; the speculation costs nothing when it fails and a DRAM round trip less
   // when it holds.
+  // A single token's pairs are positions 0 .. k+S-1, so the loop below can walk POSITIONS instead of
+  // slots: a position's partial results sit at addresses that do not depend on the routing lists (one
+  // dependent round trip less), its expert, slot and affinity are read beside them, and the product
+  // lands in its slot's place, so the final sum is still taken in slot order.
+  const bool pm = T == 1;
   int e_spec = -1;
   uint4 a0v[kAv], a1v[kAv];
   if (lr && sl < n_slots) {
-    e_spec = sl < P.k ? __ldcg(P.topk_id + t * P.k + sl) : P.E + (sl - P.k);
+    e_spec = pm ? __ldcg(P.grp_e + sl) : sl < P.k ? __ldcg(P.topk_id + t * P.k + sl) : P.E + (sl - P.k);
     if ((unsigned int)e_spec >= (unsigned int)(P.E + P.S)) e_spec = 0;        // whatever the memory held: stay in range
     const uint4* a0 = reinterpret_cast<const uint4*>(P.down.factor + ((size_t)e_spec * P.H + 2 * h2) * r);
     const uint4* a1 = reinterpret_cast<const uint4*>(P.down.factor + ((size_t)e_spec * P.H + 2 * h2 + 1) * r);
@@ -597,11 +602,17 @@ __device__ __forceinline__ void combine_fused_body(const Params& P_in, bf16* __r
   for (int s0 = 0; s0 < n_slots; s0 += kCfThreads / 32) {      // uniform trip count for the shuffles and barriers
     const int s = s0 + sl;
     const bool live = s < n_slots;
-    int pos = 0, e = 0;
+    int pos = 0, e = 0, slot = s;
     float w = 0.f;
     if (live) {
-      pos = __ldcg(P.inv_pos + t * n_slots + s);
-      e = s < P.k ? __ldcg(P.topk_id + t * P.k + s) : P.E + (s - P.k);
+      if (pm) {
+        pos = s;
+        e = __ldcg(P.grp_e + s);
+        slot = __ldcg(P.pair_slot + s);
+      } else {
+        pos = __ldcg(P.inv_pos + t * n_slots + s);
+        e = s < P.k ? __ldcg(P.topk_id + t * P.k + s) : P.E + (s - P.k);
+      }
     }
     const bool spec_ok = s0 == 0 && e == e_spec;        // the rows requested before the wait are the right ones
     // the first two z_d entries of this thread (slot sj, rank rho): their positions travel with `pos`
@@ -613,7 +624,7 @@ __device__ __forceinline__ void combine_fused_body(const Params& P_in, bf16* __r
       const int idx = tid + u * kCfThreads;
       zsj[u] = idx < n_zd ? idx / r : 0;
       zrho[u] = idx - zsj[u] * r;
-      zpj[u] = idx < n_zd ? __ldcg(P.inv_pos + t * n_slots + s0 + zsj[u]) : 0;
+      zpj[u] = idx >= n_zd ? 0 : pm ? s0 + zsj[u] : __ldcg(P.inv_pos + t * n_slots + s0 + zsj[u]);
     }
     float2 yv[kYv];
     const float* ysrc = P.ypart + (size_t)pos * P.H + 2 * h2;
@@ -655,7 +666,7 @@ __device__ __forceinline__ void combine_fused_body(const Params& P_in, bf16* __r
       }
       for (int idx = tid + 2 * kCfThreads; idx < n_zd; idx += kCfThreads) {
         const int sj = idx / r, rho = idx - sj * r;
-        const int pj = __ldcg(P.inv_pos + t * n_slots + s0 + sj);
+        const int pj = pm ? s0 + sj : __ldcg(P.inv_pos + t * n_slots + s0 + sj);
         const float* src = P.zd_part + (size_t)pj * n_sl * r + rho;
         float acc = 0.f;
         for (int si = 0; si < n_sl; ++si) acc += __ldcg(src + (size_t)si * r);
@@ -696,7 +707,7 @@ __device__ __forceinline__ void combine_fused_body(const Params& P_in, bf16* __r
     }
     y0 += __shfl_xor_sync(0xffffffffu, y0, 8);  y1 += __shfl_xor_sync(0xffffffffu, y1, 8);
     y0 += __shfl_xor_sync(0xffffffffu, y0, 16); y1 += __shfl_xor_sync(0xffffffffu, y1, 16);
-    if (live && q == 0) s_y[s * kCfCols + col] = make_float2(w * y0, w * y1);
+    if (live && q == 0) s_y[slot * kCfCols + col] = make_float2(w * y0, w * y1);
   }
   __syncthreads();
   if (tid < kCfCols) {
