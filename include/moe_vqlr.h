@@ -223,6 +223,11 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
  * moe_vqlr_specialized: number of kernels of the handle that were compiled that way (0 if none);
  * moe_vqlr_specialization_note: why not (empty string if they were), valid until destroy. */
 int moe_vqlr_specialized(const moe_vqlr_handle* h);
+/* Process-wide: where to find NVRTC (path of libnvrtc.so.12) and the CUDA headers (the directory
+ * that holds cuda_bf16.h) when they are not under /usr/local/cuda, e.g. the nvidia-cuda-nvrtc and
+ * nvidia-cuda-runtime packages of a Python environment.  NULL restores the default search.  Takes
+ * effect at the next create() of a shape that has not been compiled yet.  Returns MOE_VQLR_OK. */
+int moe_vqlr_set_jit_toolkit(const char* nvrtc_library, const char* cuda_include_dir);
 const char* moe_vqlr_specialization_note(const moe_vqlr_handle* h);
 
 /* The status word of the handle: conditions that only the kernels can detect while a call runs.

@@ -34,7 +34,7 @@ FLAG_NO_SPECIALIZE = 16384
 
 EXPORTS = ["moe_vqlr_create", "moe_vqlr_decode_layer", "moe_vqlr_decode_layer_host",
            "moe_vqlr_destroy", "moe_vqlr_last_error", "moe_vqlr_last_status", "moe_vqlr_specialized",
-           "moe_vqlr_specialization_note", "moe_vqlr_launch_count",
+           "moe_vqlr_specialization_note", "moe_vqlr_set_jit_toolkit", "moe_vqlr_launch_count",
            "moe_vqlr_workspace_bytes", "moe_vqlr_set_profiling", "moe_vqlr_last_stage_times",
            "moe_vqlr_stage_count", "moe_vqlr_stage_name", "moe_vqlr_route_noalloc",
            "moe_vqlr_run_stage", "moe_vqlr_phase_clocks", "moe_vqlr_probe_lookup_rate"]
@@ -91,6 +91,8 @@ def _load():
     lib.moe_vqlr_specialized.argtypes = [C.c_void_p]
     lib.moe_vqlr_specialization_note.restype = C.c_char_p
     lib.moe_vqlr_specialization_note.argtypes = [C.c_void_p]
+    lib.moe_vqlr_set_jit_toolkit.restype = C.c_int
+    lib.moe_vqlr_set_jit_toolkit.argtypes = [C.c_char_p, C.c_char_p]
     lib.moe_vqlr_launch_count.restype = C.c_int64
     lib.moe_vqlr_launch_count.argtypes = [C.c_void_p]
     lib.moe_vqlr_workspace_bytes.restype = C.c_int64
@@ -116,6 +118,35 @@ def _load():
 
 
 _lib = _load()
+
+
+def pip_toolkit():
+    """(libnvrtc path, CUDA include dir) of the nvidia-cuda-nvrtc / nvidia-cuda-runtime packages of this
+    Python environment, or (None, None)."""
+    try:
+        import nvidia
+    except ImportError:
+        return None, None
+    import glob
+    for base in list(getattr(nvidia, "__path__", [])):
+        libs = sorted(glob.glob(os.path.join(base, "cuda_nvrtc", "lib", "libnvrtc.so.12*")))
+        inc = os.path.join(base, "cuda_runtime", "include")
+        if libs and os.path.exists(os.path.join(inc, "cuda_bf16.h")):
+            return libs[0], inc
+    return None, None
+
+
+def set_jit_toolkit(nvrtc_library: Optional[str], cuda_include_dir: Optional[str]) -> None:
+    """Where create() finds NVRTC and the CUDA headers for the per-shape compilation (None: default)."""
+    _lib.moe_vqlr_set_jit_toolkit(None if nvrtc_library is None else nvrtc_library.encode(),
+                                  None if cuda_include_dir is None else cuda_include_dir.encode())
+
+
+# No CUDA toolkit in the usual place: point the library at the toolkit pieces of the Python environment.
+if not os.path.exists("/usr/local/cuda/include/cuda_bf16.h"):
+    _nvrtc, _inc = pip_toolkit()
+    if _nvrtc:
+        set_jit_toolkit(_nvrtc, _inc)
 
 
 def library():

@@ -12,7 +12,8 @@
 // library was loaded from; a static_assert on the sizes of the argument structures refuses files
 // that no longer match the library) given to NVRTC with -DMOE_VQLR_JIT and one -DJ_* per constant, the
 // result loaded through the runtime's library API and launched like any other kernel.  NVRTC is
-// opened with dlopen at the first create() that wants it; without it, or when anything on the way
+// opened with dlopen at the first create() that wants it (from the place moe_vqlr_set_jit_toolkit
+// names, else from the CUDA toolkit under /usr/local/cuda); without it, or when anything on the way
 // fails, the handle keeps the precompiled kernels (moe_vqlr_specialized() tells how many were compiled,
 // moe_vqlr_specialization_note() why not).  Compiled kernels are cached per process, device and option
 // string: the layers of a model share one compilation.
@@ -46,6 +47,7 @@ struct NvrtcApi {
 
 std::mutex g_jit_mu;
 NvrtcApi g_nvrtc;
+std::string g_jit_nvrtc_path, g_jit_include_dir;      // moe_vqlr_set_jit_toolkit: tried before the standard places
 std::map<std::string, cudaLibrary_t> g_jit_cache;     // "<device>|<options>" -> loaded library (never unloaded)
 
 bool file_exists(const std::string& p) {
@@ -73,6 +75,8 @@ void nvrtc_open() {
   }
   const char* roots[] = {"/usr/local/cuda", "/usr/local/cuda-12.9", "/usr/local/cuda-12", "/opt/cuda"};
   void* so = nullptr;
+  if (!g_jit_include_dir.empty() && file_exists(g_jit_include_dir + "/cuda_bf16.h")) a.cuda_include = g_jit_include_dir;
+  if (!g_jit_nvrtc_path.empty()) so = dlopen(g_jit_nvrtc_path.c_str(), RTLD_NOW | RTLD_LOCAL);
   for (const char* r : roots) {
     if (a.cuda_include.empty() && file_exists(std::string(r) + "/include/cuda_bf16.h")) a.cuda_include = std::string(r) + "/include";
     if (!so) so = dlopen((std::string(r) + "/lib64/libnvrtc.so.12").c_str(), RTLD_NOW | RTLD_LOCAL);

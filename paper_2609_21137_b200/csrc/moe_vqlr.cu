@@ -1238,6 +1238,14 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
   return take_status(h);
 }
 
+int moe_vqlr_set_jit_toolkit(const char* nvrtc_library, const char* cuda_include_dir) {
+  std::lock_guard<std::mutex> lock(g_jit_mu);
+  g_jit_nvrtc_path = nvrtc_library ? nvrtc_library : "";
+  g_jit_include_dir = cuda_include_dir ? cuda_include_dir : "";
+  g_nvrtc = NvrtcApi();          // the next create() looks again
+  return MOE_VQLR_OK;
+}
+
 int moe_vqlr_specialized(const moe_vqlr_handle* h) {
   if (!h) return 0;
   const void* all[] = {h->jit_router, h->jit_fused, h->jit_combine, h->jit_c_gateup, h->jit_c_down, h->jit_c_combine};

@@ -85,8 +85,11 @@ def toolkit_for_specialisation() -> bool:
     import glob
     import os
     roots = ["/usr/local/cuda", "/usr/local/cuda-12.9", "/usr/local/cuda-12", "/opt/cuda"]
-    return any(os.path.exists(r + "/include/cuda_bf16.h") for r in roots) and \
-        any(glob.glob(r + "/lib64/libnvrtc.so*") for r in roots)
+    if any(os.path.exists(r + "/include/cuda_bf16.h") for r in roots) and \
+            any(glob.glob(r + "/lib64/libnvrtc.so*") for r in roots):
+        return True
+    from paper_2609_21137_b200 import binding          # else the binding points the library at the pip packages
+    return binding.pip_toolkit()[0] is not None
 
 
 def run_gpu(layer, T=None, debug=True, **kw):

@@ -155,3 +155,25 @@ def test_drawn_shapes_specialised_equals_precompiled(shp):
     assert spec.last_status() == 0
     spec.close()
     plain.close()
+
+
+def test_toolkit_of_the_python_environment():
+    """moe_vqlr_set_jit_toolkit: NVRTC and the CUDA headers from the nvidia-* packages of the Python
+    environment instead of /usr/local/cuda give the same kernels (a new shape, so that it is compiled)."""
+    from paper_2609_21137_b200 import binding
+    nvrtc, inc = binding.pip_toolkit()
+    if nvrtc is None:
+        pytest.skip("no nvidia-cuda-nvrtc / nvidia-cuda-runtime packages in this environment")
+    shp = synth.LayerShape("toolkit", H=512, I=320, E=12, k=3, d=8, K=256, r=24, T=1)
+    layer, res, _ = make_checked_layer(shp, 0)
+    x = binding.bits_to_device(layer.x, "cuda")
+    binding.set_jit_toolkit(nvrtc, inc)
+    try:
+        mod = binding.MoeVqlrLayer.from_synth(layer, device="cuda")
+        assert mod.specialized() > 0, mod.specialization_note()
+        out = mod.decode(x)
+        torch.cuda.synchronize()
+        assert_output(bf16_tensor_to_f64(out), res.out, what="toolkit of the Python environment")
+        mod.close()
+    finally:
+        binding.set_jit_toolkit(None, None)
