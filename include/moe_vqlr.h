@@ -218,8 +218,9 @@ int moe_vqlr_decode_layer_host(moe_vqlr_handle* h, const void* x_host, int32_t T
  * the ahead-of-time, per-model mapping of Section 4).  Same arithmetic in the same order, so results
  * are bitwise those of the precompiled kernels; a batch-1 call is shorter because its blocks fetch
  * about half the instructions.  Costs a few seconds at the first create() of a shape (kept per
- * process and device afterwards).  Needs libnvrtc and the CUDA headers under /usr/local/cuda; where
- * they are missing, or with MOE_VQLR_FLAG_NO_SPECIALIZE, the precompiled kernels run.
+ * process and device afterwards).  Needs libnvrtc and the CUDA headers (under /usr/local/cuda, or where
+ * moe_vqlr_set_jit_toolkit points); where they are missing, or with MOE_VQLR_FLAG_NO_SPECIALIZE, the
+ * precompiled kernels run.
  * moe_vqlr_specialized: number of kernels of the handle that were compiled that way (0 if none);
  * moe_vqlr_specialization_note: why not (empty string if they were), valid until destroy. */
 int moe_vqlr_specialized(const moe_vqlr_handle* h);
